@@ -1,0 +1,142 @@
+/*
+ * goq.h - C ABI of libgoq: the linear-layer inner product against dual-basis Power-of-Two
+ * (PoT) weights of GoQuant (arxiv 2605.26092), hand-written CUDA for sm_100a.
+ *
+ * A weight row is cut into macro-blocks ("groups") of `group` consecutive input channels
+ * (paper Section 3.1, N = 128 there). Each group is stored as
+ *      w_hat = c1 * b1 + c2 * b2,   <b1, b2> = 0                        (Section 3.1)
+ *   b1  one `wbits`-bit PoT code per weight on the asymmetric lattice of Section 3.2
+ *       (code c: sign = c >> (wbits-1), e = c & emax, emax = 2^(wbits-1) - 1,
+ *        value = (-1)^sign 2^-e, except c == emax which is 0);
+ *   b2  never stored: a 6-bit record per 8 weights (2-bit pattern s-1, four pair-sign flags)
+ *       tells how to derive it from b1 by the Strided Dual-Exchange of Section 3.3, Theorem 1:
+ *       for each pair (i, j = i XOR s), i < j:  y_i = -eta x_j,  y_j = eta x_i.
+ *       Record byte: bits[1:0] = s-1; bit 2+p = 1 iff eta of the p-th pair (pairs in ascending
+ *       order of their lower index) is -1;
+ *   c1, c2  one fp16 pair per (row, group) (Section 3.4).
+ *
+ * The layer itself is Eq. 4 of Section 3.5 read per group:
+ *      y[m,n] = sum_j ( c1[n,j] * sum_{k in j} b1[n,k] x[m,k] + c2[n,j] * sum_{k in j} b2[n,k] x[m,k] )
+ * The two inner sums use PoT operands only; the coefficient multiply sits outside them.
+ *
+ * Conventions for every call
+ *   - W is [n_out][k_in] (row n = output channel). k_in % group == 0, group % 8 == 0.
+ *   - All pointers are DEVICE pointers unless a parameter says "host". The caller owns every
+ *     buffer; the library allocates nothing, frees nothing and keeps no pointer after return.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream). Calls enqueue work
+ *     and return; they do not synchronise.
+ *   - Argument errors are found on the host before any launch and returned as a status; nothing
+ *     is printed, nothing aborts. A failed launch returns GOQ_ERR_CUDA.
+ *   - The library runs on compute capability 10.x only (GOQ_ERR_ARCH otherwise). There is no
+ *     CPU path.
+ */
+#ifndef GOQ_H
+#define GOQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GOQ_OK = 0,
+    GOQ_ERR_INVALID_ARG = 1,    /* NULL pointer, bad size, bad enum */
+    GOQ_ERR_UNSUPPORTED = 2,    /* valid request this build has no kernel for */
+    GOQ_ERR_ALIGNMENT = 3,      /* pointer not aligned as documented */
+    GOQ_ERR_WORKSPACE = 4,      /* workspace or output buffer too small */
+    GOQ_ERR_OVERFLOW_BOUND = 5, /* integer path: static int32 bound k_in*127*127*2^emax exceeded */
+    GOQ_ERR_ARCH = 6,           /* current device is not sm_100 */
+    GOQ_ERR_CUDA = 7,           /* CUDA runtime reported an error */
+    GOQ_ERR_TIMEOUT = 8         /* a bounded device-side wait expired (reported through a status word) */
+} goq_status;
+
+typedef enum { GOQ_BF16 = 0, GOQ_F32 = 1, GOQ_I8 = 2 } goq_dtype;
+typedef enum { GOQ_OP_GEMV = 0, GOQ_OP_GEMM = 1 } goq_op;
+
+#define GOQ_LAYOUT_TILE16 1 /* the only packed layout so far; see goq_pack */
+
+typedef struct {
+    int32_t n_out;  /* output channels N */
+    int32_t k_in;   /* input channels K */
+    int32_t group;  /* macro-block size g: multiple of 8 that divides 128, or 128 (8,16,32,64,128) */
+    int32_t wbits;  /* 2, 3 or 4 */
+    int32_t layout; /* GOQ_LAYOUT_TILE16 */
+} goq_desc;
+
+/* Text for a status code (static string, never NULL). */
+const char* goq_status_string(goq_status s);
+
+/* Bytes of the packed buffer for this descriptor; 0 if the descriptor is invalid.
+ * Storage arithmetic of Section 3.3 step 3 (6 record bits per 8 weights) plus codes and coefficients. */
+size_t goq_packed_bytes(const goq_desc* desc);
+
+/* Algorithmic bytes of the same weights: n_out*k_in*(wbits + 0.75)/8 + n_out*(k_in/group)*4.
+ * This is the figure roofline numbers are quoted against; the packed buffer may be larger. */
+size_t goq_algorithmic_bytes(const goq_desc* desc);
+
+/* Scratch bytes goq_gemv / goq_gemm need for `m` activation rows (may be 0). */
+size_t goq_workspace_bytes(const goq_desc* desc, int op, int m);
+
+/* goq_pack - re-tile quantizer output into the layout the kernels stream (Sections 3.2-3.4 give
+ * the fields; the layout is this library's own).
+ *   codes     [n_out][k_in] uint8, one code per weight, value < 2^wbits
+ *   meta      [n_out][k_in/8] uint8, 6-bit exchange record per micro-block
+ *   coef_f16  [n_out][k_in/group][2] IEEE fp16 bit patterns (c1, c2)
+ *   packed    out, goq_packed_bytes(desc) bytes, 128-byte aligned
+ * Layout GOQ_LAYOUT_TILE16: rows padded to a multiple of 16 and k to a multiple of 128 with
+ * zero-valued weights; one 32-bit word per micro-block (8 nibbles = 8 codes, record bits in the
+ * nibbles' spare top bits for wbits <= 3, in a side byte plane for wbits = 4); words ordered so
+ * that the 32 lanes of a warp read 512 contiguous bytes per 128-bit load; coefficient pairs in a
+ * second plane, 64 contiguous bytes per (16-row tile, group). */
+goq_status goq_pack(const goq_desc* desc, const uint8_t* codes, const uint8_t* meta,
+                    const uint16_t* coef_f16, void* packed, size_t packed_bytes, void* stream);
+
+/* goq_unpack - inverse of goq_pack plus the in-register derivation of b2, for tests.
+ *   codes_b1  out [n_out][k_in] uint8: the stored code of b1
+ *   codes_b2  out [n_out][k_in] uint8: b2 as (sign << 3) | e, or 0x80 for a zero (b2 can take the
+ *             value +2^-emax that b1's code cannot express; Section 3.3 on separate sign and magnitude)
+ *   coef_f16  out [n_out][k_in/group][2]
+ * Any output pointer may be NULL to skip it. */
+goq_status goq_unpack(const goq_desc* desc, const void* packed, uint8_t* codes_b1, uint8_t* codes_b2,
+                      uint16_t* coef_f16, void* stream);
+
+/* goq_gemv - decode-time layer for a small batch (Eq. 4, float activations).
+ *   x_bf16   [batch][k_in] bf16, 16-byte aligned, batch in 1..16
+ *   y        out [batch][n_out], y_dtype GOQ_BF16 or GOQ_F32
+ *   ws       scratch of goq_workspace_bytes(desc, GOQ_OP_GEMV, batch) bytes (may be NULL if that is 0)
+ * Each PoT term is applied to the activation as an exponent shift; sums are fp32. */
+goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16, int batch, void* y,
+                    int y_dtype, void* ws, size_t ws_bytes, void* stream);
+
+/* goq_gemm - the same layer for m activation rows.
+ *  x_dtype GOQ_BF16: x [m][k_in] bf16; y out [m][n_out] (GOQ_BF16 or GOQ_F32); sx, cq, sc, acc unused (NULL).
+ *  x_dtype GOQ_I8 (Eq. 4 with integer X~ and c~; left shifts x~ << (emax-e), exact int32):
+ *      x    [m][k_in] int8         sx [m] fp32 per-token scale
+ *      cq   [n_out][k_in/group][2] int8 integer coefficients,  sc [n_out][2] fp32 their per-channel scales
+ *      acc  out, optional: [2][m][n_out] int32, ACC_b[m][n] = sum_j cq[n][j][b] * sum_{k in j} x[m][k] * (2^emax b_b[n][k])
+ *      y    out, optional: [m][n_out] = sx[m] * 2^-emax * (sc[n][0]*ACC_1 + sc[n][1]*ACC_2)
+ *    At least one of acc, y must be given. Returns GOQ_ERR_OVERFLOW_BOUND if k_in*127*127*2^emax >= 2^31. */
+goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int m, int x_dtype,
+                    const float* sx, const int8_t* cq, const float* sc, void* y, int y_dtype,
+                    int32_t* acc, void* ws, size_t ws_bytes, void* stream);
+
+/* goq_gemv_host - goq_gemv for callers whose activations live in host memory (Eq. 4, as goq_gemv).
+ *   x_host   HOST [batch][k_in] bf16 (pinned memory makes the copy asynchronous)
+ *   y_host   HOST out [batch][n_out]
+ *   x_stage, y_stage  DEVICE staging buffers of batch*k_in*2 and batch*n_out*sizeof(y_dtype) bytes
+ * Enqueues copy-in, the kernel and copy-out on `stream`; the caller synchronises the stream
+ * before reading y_host. */
+goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x_host, int batch,
+                         void* y_host, int y_dtype, void* x_stage, void* y_stage, void* ws,
+                         size_t ws_bytes, void* stream);
+
+/* Force a kernel variant (benchmarks and tests only): 0 = automatic, 1 = scalar exponent-add
+ * kernel, 2 = tensor-core fragment kernel. Process-wide. Returns the previous value. */
+int goq_set_gemv_variant(int variant);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GOQ_H */

@@ -1,0 +1,159 @@
+// C ABI of libgoq: argument checks on the host, then one launcher per call.
+#include <atomic>
+#include <cstdlib>
+#include "goq_common.cuh"
+#include "goq_internal.h"
+
+using goq::Geometry;
+
+namespace {
+
+std::atomic<int> g_gemv_variant{0};
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// compute capability 10.x of the current device, cached per device index
+goq_status check_arch() {
+    static std::atomic<int> cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GOQ_ERR_CUDA;
+    if (dev >= 0 && dev < 64) {
+        int c = cached[dev].load(std::memory_order_relaxed);
+        if (c == 1) return GOQ_OK;
+        if (c == 2) return GOQ_ERR_ARCH;
+    }
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return GOQ_ERR_CUDA;
+    const bool ok = (major == 10);
+    if (dev >= 0 && dev < 64) cached[dev].store(ok ? 1 : 2, std::memory_order_relaxed);
+    return ok ? GOQ_OK : GOQ_ERR_ARCH;
+}
+
+goq_status from_cuda(cudaError_t e) { return e == cudaSuccess ? GOQ_OK : GOQ_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+const char* goq_status_string(goq_status s) {
+    switch (s) {
+        case GOQ_OK: return "ok";
+        case GOQ_ERR_INVALID_ARG: return "invalid argument";
+        case GOQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case GOQ_ERR_ALIGNMENT: return "misaligned pointer";
+        case GOQ_ERR_WORKSPACE: return "buffer too small";
+        case GOQ_ERR_OVERFLOW_BOUND: return "int32 accumulator bound exceeded";
+        case GOQ_ERR_ARCH: return "device is not sm_100";
+        case GOQ_ERR_CUDA: return "CUDA runtime error";
+        case GOQ_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+size_t goq_packed_bytes(const goq_desc* desc) {
+    Geometry g;
+    return goq::make_geometry(desc, &g) ? g.total_bytes : 0;
+}
+
+size_t goq_algorithmic_bytes(const goq_desc* desc) {
+    Geometry g;
+    if (!goq::make_geometry(desc, &g)) return 0;
+    // (wbits + 0.75) bits per weight = (4*wbits + 3) / 32 bytes
+    return (size_t)g.n_out * g.k_in * (4 * g.wbits + 3) / 32 + (size_t)g.n_out * (g.k_in / g.group) * 4;
+}
+
+size_t goq_workspace_bytes(const goq_desc* desc, int op, int m) {
+    Geometry g;
+    if (!goq::make_geometry(desc, &g) || m <= 0) return 0;
+    (void)op;
+    return 0;
+}
+
+goq_status goq_pack(const goq_desc* desc, const uint8_t* codes, const uint8_t* meta, const uint16_t* coef_f16,
+                    void* packed, size_t packed_bytes, void* stream) {
+    Geometry g;
+    if (!goq::make_geometry(desc, &g) || !codes || !meta || !coef_f16 || !packed) return GOQ_ERR_INVALID_ARG;
+    if (!aligned(packed, 128) || !aligned(coef_f16, 2)) return GOQ_ERR_ALIGNMENT;
+    if (packed_bytes < g.total_bytes) return GOQ_ERR_WORKSPACE;
+    if (goq_status s = check_arch()) return s;
+    return from_cuda(goq::launch_pack(g, codes, meta, coef_f16, packed, (cudaStream_t)stream));
+}
+
+goq_status goq_unpack(const goq_desc* desc, const void* packed, uint8_t* codes_b1, uint8_t* codes_b2,
+                      uint16_t* coef_f16, void* stream) {
+    Geometry g;
+    if (!goq::make_geometry(desc, &g) || !packed) return GOQ_ERR_INVALID_ARG;
+    if (!codes_b1 && !codes_b2 && !coef_f16) return GOQ_ERR_INVALID_ARG;
+    if (!aligned(packed, 128) || !aligned(coef_f16, 2)) return GOQ_ERR_ALIGNMENT;
+    if (goq_status s = check_arch()) return s;
+    return from_cuda(goq::launch_unpack(g, packed, codes_b1, codes_b2, coef_f16, (cudaStream_t)stream));
+}
+
+goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16, int batch, void* y, int y_dtype,
+                    void* ws, size_t ws_bytes, void* stream) {
+    Geometry g;
+    if (!goq::make_geometry(desc, &g) || !packed || !x_bf16 || !y) return GOQ_ERR_INVALID_ARG;
+    if (batch < 1 || batch > 16) return GOQ_ERR_INVALID_ARG;
+    if (y_dtype != GOQ_BF16 && y_dtype != GOQ_F32) return GOQ_ERR_INVALID_ARG;
+    if (!aligned(packed, 128) || !aligned(x_bf16, 16) || !aligned(y, y_dtype == GOQ_F32 ? 4 : 2))
+        return GOQ_ERR_ALIGNMENT;
+    (void)ws;
+    (void)ws_bytes;
+    if (goq_status s = check_arch()) return s;
+    const int variant = g_gemv_variant.load(std::memory_order_relaxed);
+    bool use_mma = goq::linear_mma_supported(g);
+    if (variant == 1) use_mma = false;
+    if (variant == 2 && !use_mma) return GOQ_ERR_UNSUPPORTED;
+    if (use_mma) return from_cuda(goq::launch_linear_mma(g, packed, x_bf16, batch, y, y_dtype, (cudaStream_t)stream));
+    return from_cuda(goq::launch_gemv_scalar(g, packed, x_bf16, batch, y, y_dtype, (cudaStream_t)stream));
+}
+
+goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int m, int x_dtype, const float* sx,
+                    const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, void* ws, size_t ws_bytes,
+                    void* stream) {
+    Geometry g;
+    if (!goq::make_geometry(desc, &g) || !packed || !x || m < 1) return GOQ_ERR_INVALID_ARG;
+    if (y && y_dtype != GOQ_BF16 && y_dtype != GOQ_F32) return GOQ_ERR_INVALID_ARG;
+    if (!aligned(packed, 128) || !aligned(x, 16)) return GOQ_ERR_ALIGNMENT;
+    if (y && !aligned(y, y_dtype == GOQ_F32 ? 4 : 2)) return GOQ_ERR_ALIGNMENT;
+    (void)ws;
+    (void)ws_bytes;
+    if (x_dtype == GOQ_BF16) {
+        if (!y) return GOQ_ERR_INVALID_ARG;
+        if (!goq::linear_mma_supported(g)) return GOQ_ERR_UNSUPPORTED;
+        if (goq_status s = check_arch()) return s;
+        return from_cuda(goq::launch_linear_mma(g, packed, x, m, y, y_dtype, (cudaStream_t)stream));
+    }
+    if (x_dtype == GOQ_I8) {
+        if (!cq || (!y && !acc)) return GOQ_ERR_INVALID_ARG;
+        if (y && (!sx || !sc)) return GOQ_ERR_INVALID_ARG;
+        if (!aligned(acc, 4) || !aligned(sx, 4) || !aligned(sc, 4)) return GOQ_ERR_ALIGNMENT;
+        if (g.wbits > 3 || g.group < 16 || (g.k_in % 16)) return GOQ_ERR_UNSUPPORTED;
+        // |ACC| <= k_in * 127 (x~) * 127 (c~) * 2^emax must stay below 2^31
+        const long long bound = (long long)g.k_in * 127 * 127 * (1ll << ((1 << (g.wbits - 1)) - 1));
+        if (bound >= (1ll << 31)) return GOQ_ERR_OVERFLOW_BOUND;
+        if (goq_status s = check_arch()) return s;
+        return from_cuda(goq::launch_gemm_a8(g, packed, (const int8_t*)x, m, sx, cq, sc, y, y_dtype, acc,
+                                             (cudaStream_t)stream));
+    }
+    return GOQ_ERR_INVALID_ARG;
+}
+
+goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x_host, int batch, void* y_host,
+                         int y_dtype, void* x_stage, void* y_stage, void* ws, size_t ws_bytes, void* stream) {
+    Geometry g;
+    if (!goq::make_geometry(desc, &g) || !x_host || !y_host || !x_stage || !y_stage) return GOQ_ERR_INVALID_ARG;
+    if (batch < 1 || batch > 16) return GOQ_ERR_INVALID_ARG;
+    if (y_dtype != GOQ_BF16 && y_dtype != GOQ_F32) return GOQ_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t xb = (size_t)batch * g.k_in * 2, yb = (size_t)batch * g.n_out * (y_dtype == GOQ_F32 ? 4 : 2);
+    if (cudaMemcpyAsync(x_stage, x_host, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return GOQ_ERR_CUDA;
+    goq_status s = goq_gemv(desc, packed, x_stage, batch, y_stage, y_dtype, ws, ws_bytes, stream);
+    if (s != GOQ_OK) return s;
+    if (cudaMemcpyAsync(y_host, y_stage, yb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GOQ_ERR_CUDA;
+    return GOQ_OK;
+}
+
+int goq_set_gemv_variant(int variant) { return g_gemv_variant.exchange(variant); }
+
+}  // extern "C"

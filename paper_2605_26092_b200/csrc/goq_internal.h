@@ -1,0 +1,25 @@
+// Internal launcher declarations shared by the translation units of libgoq.
+#pragma once
+#include <cuda_runtime.h>
+#include "goq_common.cuh"
+
+namespace goq {
+
+cudaError_t launch_pack(const Geometry& g, const uint8_t* codes, const uint8_t* meta, const uint16_t* coef,
+                        void* packed, cudaStream_t st);
+cudaError_t launch_unpack(const Geometry& g, const void* packed, uint8_t* b1, uint8_t* b2, uint16_t* coef,
+                          cudaStream_t st);
+
+// Float-activation layer, scalar exponent-add kernel (any group size, batch <= 16).
+cudaError_t launch_gemv_scalar(const Geometry& g, const void* packed, const void* x_bf16, int batch, void* y,
+                               int y_dtype, cudaStream_t st);
+// Float-activation layer, tensor-core fragment kernel (group >= 32); m may exceed 16.
+cudaError_t launch_linear_mma(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y,
+                              int y_dtype, cudaStream_t st);
+bool linear_mma_supported(const Geometry& g);
+
+// Integer-activation layer.
+cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* x, int m, const float* sx,
+                           const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, cudaStream_t st);
+
+}  // namespace goq

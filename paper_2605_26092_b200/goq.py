@@ -1,0 +1,139 @@
+"""ctypes binding of libgoq.so with the same names as include/goq.h.
+
+Arguments are torch CUDA tensors (device memory) or plain integers; the functions pass
+`tensor.data_ptr()` and the current CUDA stream to the C ABI and raise GoqError on a non-zero
+status. No arithmetic of the method happens here.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, c_char_p, c_int, c_int32, c_size_t, c_void_p
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libgoq.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_OVERFLOW_BOUND, ERR_ARCH, ERR_CUDA, \
+    ERR_TIMEOUT = range(9)
+BF16, F32, I8 = 0, 1, 2
+OP_GEMV, OP_GEMM = 0, 1
+LAYOUT_TILE16 = 1
+
+EXPORTS = (
+    "goq_status_string", "goq_packed_bytes", "goq_algorithmic_bytes", "goq_workspace_bytes", "goq_pack",
+    "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant",
+)
+
+
+class GoqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+class Desc(Structure):
+    _fields_ = [("n_out", c_int32), ("k_in", c_int32), ("group", c_int32), ("wbits", c_int32), ("layout", c_int32)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libgoq.so (built in-tree by build.py). Raises if it is missing: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} not found: run `python -m paper_2605_26092_b200.build` first")
+        L = ctypes.CDLL(_LIB_PATH)
+        L.goq_status_string.restype = c_char_p
+        L.goq_status_string.argtypes = [c_int]
+        for name in ("goq_packed_bytes", "goq_algorithmic_bytes"):
+            getattr(L, name).restype = c_size_t
+            getattr(L, name).argtypes = [POINTER(Desc)]
+        L.goq_workspace_bytes.restype = c_size_t
+        L.goq_workspace_bytes.argtypes = [POINTER(Desc), c_int, c_int]
+        L.goq_pack.restype = c_int
+        L.goq_pack.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.goq_unpack.restype = c_int
+        L.goq_unpack.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.goq_gemv.restype = c_int
+        L.goq_gemv.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p, c_size_t, c_void_p]
+        L.goq_gemm.restype = c_int
+        L.goq_gemm.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p,
+                               c_void_p, c_int, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.goq_gemv_host.restype = c_int
+        L.goq_gemv_host.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p,
+                                    c_void_p, c_size_t, c_void_p]
+        L.goq_set_gemv_variant.restype = c_int
+        L.goq_set_gemv_variant.argtypes = [c_int]
+        _lib = L
+    return _lib
+
+
+def desc(n_out: int, k_in: int, group: int, wbits: int, layout: int = LAYOUT_TILE16) -> Desc:
+    return Desc(n_out, k_in, group, wbits, layout)
+
+
+def status_string(status: int) -> str:
+    return lib().goq_status_string(int(status)).decode()
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr() if hasattr(t, "data_ptr") else int(t))
+
+
+def _stream(stream=None):
+    if stream is not None:
+        return c_void_p(int(stream))
+    import torch
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise GoqError(status, where)
+
+
+def packed_bytes(d: Desc) -> int:
+    return lib().goq_packed_bytes(ctypes.byref(d))
+
+
+def algorithmic_bytes(d: Desc) -> int:
+    return lib().goq_algorithmic_bytes(ctypes.byref(d))
+
+
+def workspace_bytes(d: Desc, op: int, m: int) -> int:
+    return lib().goq_workspace_bytes(ctypes.byref(d), op, m)
+
+
+def set_gemv_variant(variant: int) -> int:
+    return lib().goq_set_gemv_variant(variant)
+
+
+def pack(d: Desc, codes, meta, coef_f16, packed, stream=None):
+    _check(lib().goq_pack(ctypes.byref(d), _ptr(codes), _ptr(meta), _ptr(coef_f16), _ptr(packed),
+                          packed.numel() * packed.element_size(), _stream(stream)), "goq_pack")
+
+
+def unpack(d: Desc, packed, codes_b1=None, codes_b2=None, coef_f16=None, stream=None):
+    _check(lib().goq_unpack(ctypes.byref(d), _ptr(packed), _ptr(codes_b1), _ptr(codes_b2), _ptr(coef_f16),
+                            _stream(stream)), "goq_unpack")
+
+
+def gemv(d: Desc, packed, x_bf16, batch: int, y, y_dtype: int, ws=None, stream=None):
+    wsb = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(lib().goq_gemv(ctypes.byref(d), _ptr(packed), _ptr(x_bf16), batch, _ptr(y), y_dtype, _ptr(ws), wsb,
+                          _stream(stream)), "goq_gemv")
+
+
+def gemm(d: Desc, packed, x, m: int, x_dtype: int, y=None, y_dtype: int = F32, sx=None, cq=None, sc=None,
+         acc=None, ws=None, stream=None):
+    wsb = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(lib().goq_gemm(ctypes.byref(d), _ptr(packed), _ptr(x), m, x_dtype, _ptr(sx), _ptr(cq), _ptr(sc),
+                          _ptr(y), y_dtype, _ptr(acc), _ptr(ws), wsb, _stream(stream)), "goq_gemm")
+
+
+def gemv_host(d: Desc, packed, x_host, batch: int, y_host, y_dtype: int, x_stage, y_stage, ws=None, stream=None):
+    wsb = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(lib().goq_gemv_host(ctypes.byref(d), _ptr(packed), _ptr(x_host), batch, _ptr(y_host), y_dtype,
+                               _ptr(x_stage), _ptr(y_stage), _ptr(ws), wsb, _stream(stream)), "goq_gemv_host")

@@ -1,0 +1,289 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs.
+
+Tolerances: float-activation outputs within 2e-3 normwise relative error of the fp64 oracle (the stated
+bar); the fp32-accumulating kernels are expected far inside it, so a second, tight bound (2e-5) guards
+against errors that the loose bar would hide. Integer accumulators: bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+import synth_inputs as si
+from oracle import goq_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3
+TIGHT = 2e-5
+
+
+@pytest.fixture(scope="module")
+def goq():
+    from paper_2605_26092_b200 import build
+    build.build()
+    from paper_2605_26092_b200 import goq as g
+    g.lib()
+    assert torch.cuda.is_available()
+    return g
+
+
+def b2_reference_bytes(codes, meta, b):
+    """Oracle b2 values in the byte format goq_unpack emits: (sign << 3) | e, 0x80 for zero."""
+    b2 = O.decode_b2(codes, meta, b)
+    out = np.full(b2.shape, 0x80, dtype=np.uint8)
+    nz = b2 != 0
+    e = np.zeros(b2.shape, dtype=np.int64)
+    e[nz] = np.round(-np.log2(np.abs(b2[nz]))).astype(np.int64)
+    out[nz] = (((b2[nz] < 0).astype(np.uint8) << 3) | e[nz].astype(np.uint8))
+    return out
+
+
+# ------------------------------------------------------------------------------------- pack / unpack
+@pytest.mark.parametrize("n,k,g,b", [(256, 256, 64, 3), (40, 192, 64, 3), (17, 384, 128, 3), (33, 256, 32, 2),
+                                     (24, 128, 16, 4), (16, 128, 8, 3)])
+def test_pack_unpack_roundtrip_and_b2_derivation(goq, n, k, g, b):
+    from tests.gpu_util import pack_weights
+    w = si.gaussian_weights(n, k, seed=n + k)
+    codes, meta, coef = O.quantize_geo(w, g, b)
+    d, packed = pack_weights(n, k, g, b, codes, meta, coef)
+    b1 = torch.full((n, k), 0xEE, dtype=torch.uint8, device="cuda")
+    b2 = torch.full((n, k), 0xEE, dtype=torch.uint8, device="cuda")
+    cf = torch.zeros((n, k // g, 2), dtype=torch.int16, device="cuda")
+    goq.unpack(d, packed, b1, b2, cf)
+    torch.cuda.synchronize()
+    assert np.array_equal(b1.cpu().numpy(), codes)
+    assert np.array_equal(b2.cpu().numpy(), b2_reference_bytes(codes, meta, b))
+    assert np.array_equal(cf.cpu().numpy().view(np.uint16), coef.view(np.uint16))
+
+
+def test_unpack_covers_all_64_records_and_all_codes(goq):
+    from tests.gpu_util import pack_weights
+    rng = np.random.default_rng(0)
+    n, k = 64, 512
+    codes = rng.integers(0, 8, size=(n, k), dtype=np.uint8)
+    meta = (np.arange(n * k // 8) % 64).astype(np.uint8).reshape(n, k // 8)
+    coef = rng.standard_normal((n, k // 128, 2)).astype(np.float16)
+    d, packed = pack_weights(n, k, 128, 3, codes, meta, coef)
+    b2 = torch.empty((n, k), dtype=torch.uint8, device="cuda")
+    goq.unpack(d, packed, None, b2, None)
+    torch.cuda.synchronize()
+    assert np.array_equal(b2.cpu().numpy(), b2_reference_bytes(codes, meta, 3))
+
+
+# ------------------------------------------------------------------------------------- decode GEMV
+def _quantized(n, k, g, b, seed, outliers=False):
+    w = si.weights_with_outlier_channels(n, k, seed=seed) if outliers else si.gaussian_weights(n, k, seed=seed)
+    return O.quantize_geo(w, g, b)
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("batch", [1, 8])
+def test_config1_single_layer_256(goq, variant, batch):
+    """K = N = 256, W3, group 64, fp16 coefficients, bf16 activations, batch 1 and 8, seed 0."""
+    from tests.gpu_util import pack_weights, run_gemv
+    codes, meta, coef = _quantized(256, 256, 64, 3, seed=0)
+    d, packed = pack_weights(256, 256, 64, 3, codes, meta, coef)
+    xb = si.bf16_activations(batch, 256, seed=0)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 64, 3)
+    y = run_gemv(d, packed, xb, goq.F32, variant)
+    err = O.normwise_rel_err(y, y_ref)
+    assert err <= TOL and err <= TIGHT, err
+    y16 = run_gemv(d, packed, xb, goq.BF16, variant)
+    assert O.normwise_rel_err(y16, y_ref) <= 4e-3  # one extra bf16 rounding of the output (2^-9 per element)
+    assert O.normwise_rel_err(y16, y_ref) > 0
+
+
+@pytest.mark.parametrize("n,k,g,b,batch,variant", [
+    (40, 192, 64, 3, 3, 1), (40, 192, 64, 3, 3, 2), (17, 384, 128, 3, 16, 2), (17, 384, 128, 3, 16, 1),
+    (33, 256, 32, 2, 5, 2), (33, 256, 32, 2, 5, 1), (24, 128, 16, 4, 2, 1), (16, 128, 8, 3, 1, 1),
+    (48, 256, 64, 4, 9, 2), (48, 256, 64, 4, 9, 1), (16, 128, 128, 3, 1, 2), (300, 1152, 128, 3, 12, 2),
+])
+def test_gemv_ragged_shapes_bit_widths_and_groups(goq, n, k, g, b, batch, variant):
+    from tests.gpu_util import pack_weights, run_gemv
+    codes, meta, coef = _quantized(n, k, g, b, seed=n * 7 + k, outliers=True)
+    d, packed = pack_weights(n, k, g, b, codes, meta, coef)
+    xb = si.bf16_activations(batch, k, seed=k)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), g, b)
+    y = run_gemv(d, packed, xb, goq.F32, variant)
+    err = O.normwise_rel_err(y, y_ref)
+    assert err <= TIGHT, err
+
+
+def test_two_kernel_variants_agree_closely_and_runs_are_deterministic(goq):
+    from tests.gpu_util import pack_weights, run_gemv
+    codes, meta, coef = si.random_quantized(512, 1024, 128, 3, seed=3)
+    d, packed = pack_weights(512, 1024, 128, 3, codes, meta, coef)
+    xb = si.bf16_activations(4, 1024, seed=4)
+    y1 = run_gemv(d, packed, xb, goq.F32, 1)
+    y2 = run_gemv(d, packed, xb, goq.F32, 2)
+    assert O.normwise_rel_err(y1, y2) < 1e-5
+    for v in (1, 2):
+        a = run_gemv(d, packed, xb, goq.F32, v)
+        b = run_gemv(d, packed, xb, goq.F32, v)
+        assert np.array_equal(a, b)
+
+
+def test_extreme_activations_keep_exponent_arithmetic_right(goq):
+    """Zeros, tiny and huge bf16 values: the exponent-shift product must equal the true product."""
+    from tests.gpu_util import pack_weights, run_gemv
+    codes, meta, coef = si.random_quantized(32, 256, 64, 3, seed=5)
+    d, packed = pack_weights(32, 256, 64, 3, codes, meta, coef)
+    x = si.bf16_bits_to_f64(si.bf16_activations(2, 256, seed=6))
+    x[0, ::3] = 0.0
+    x[0, 1::7] *= 2.0 ** -120
+    x[1, ::5] *= 2.0 ** 100
+    xb = si.f32_to_bf16_bits(x.astype(np.float32))
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 64, 3)
+    for v in (1, 2):
+        assert O.normwise_rel_err(run_gemv(d, packed, xb, goq.F32, v), y_ref) <= TIGHT
+
+
+@pytest.mark.parametrize("name,n,k", si.LLAMA2_7B_LINEARS[3:])
+@pytest.mark.parametrize("batch", [1, 4, 16])
+def test_config2_llama7b_shapes_sampled_rows(goq, name, n, k, batch):
+    """7B-shaped linears, W3 group 128, full-size launch; the oracle evaluates a seeded sample of rows."""
+    from tests.gpu_util import pack_weights, run_gemv
+    codes, meta, coef = si.random_quantized(n, k, 128, 3, seed=n + k)
+    rows = si.sample_rows(n, 96, seed=1)
+    # rows quantized by the oracle from outlier-channel weights replace the random fields in the sample
+    w = si.weights_with_outlier_channels(len(rows), k, seed=7)
+    codes[rows], meta[rows], coef[rows] = O.quantize_geo(w, 128, 3)
+    d, packed = pack_weights(n, k, 128, 3, codes, meta, coef)
+    xb = si.bf16_activations(batch, k, seed=batch)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 128, 3, rows=rows)
+    y = run_gemv(d, packed, xb, goq.F32)
+    err = O.normwise_rel_err(y[:, rows], y_ref)
+    assert err <= TOL and err <= TIGHT, err
+
+
+# ------------------------------------------------------------------------------------- prefill GEMM
+def test_gemm_bf16_small_full_parity(goq):
+    from tests.gpu_util import pack_weights, run_gemm_bf16
+    codes, meta, coef = _quantized(80, 384, 128, 3, seed=11, outliers=True)
+    d, packed = pack_weights(80, 384, 128, 3, codes, meta, coef)
+    xb = si.bf16_activations(150, 384, seed=12)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 128, 3)
+    y = run_gemm_bf16(d, packed, xb)
+    assert O.normwise_rel_err(y, y_ref) <= TOL
+
+
+def test_config4_prefill_2048_tokens_sampled_rows(goq):
+    from tests.gpu_util import pack_weights, run_gemm_bf16
+    n, k, m = 4096, 4096, 2048
+    codes, meta, coef = si.random_quantized(n, k, 128, 3, seed=21)
+    rows = si.sample_rows(n, 64, seed=2)
+    w = si.gaussian_weights(len(rows), k, seed=22)
+    codes[rows], meta[rows], coef[rows] = O.quantize_geo(w, 128, 3)
+    d, packed = pack_weights(n, k, 128, 3, codes, meta, coef)
+    xb = si.bf16_activations(m, k, seed=23)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 128, 3, rows=rows)
+    y = run_gemm_bf16(d, packed, xb)
+    assert O.normwise_rel_err(y[:, rows], y_ref) <= TOL
+
+
+# ------------------------------------------------------------------------------------- integer path
+@pytest.mark.parametrize("n,k,g,b,m", [(48, 256, 64, 3, 200), (20, 192, 32, 2, 130), (16, 128, 128, 3, 1)])
+def test_int8_path_bit_exact_small(goq, n, k, g, b, m):
+    from tests.gpu_util import pack_weights, run_gemm_i8
+    codes, meta, coef = _quantized(n, k, g, b, seed=31)
+    cq, sc = O.quantize_coefficients_int8(coef)
+    xq, sx = O.quantize_activations_int8(si.f32_activations(m, k, seed=32))
+    d, packed = pack_weights(n, k, g, b, codes, meta, coef)
+    acc, y = run_gemm_i8(d, packed, xq, sx, cq, sc)
+    a1, a2, y_ref = O.linear_i32(codes, meta, cq, sc, xq, sx, g, b)
+    assert np.array_equal(acc[0], a1) and np.array_equal(acc[1], a2)
+    assert O.normwise_rel_err(y, y_ref) <= TIGHT
+
+
+@pytest.mark.parametrize("name,n,k", si.VIT_B16_LINEARS)
+def test_config3_vit_b16_int8_bit_exact(goq, name, n, k):
+    """ViT-B/16-shaped linears, 197 x 64 tokens, W3 group 64, per-token int8 activations:
+    full-size launch, int32 accumulators compared bit for bit on a seeded sample of output channels
+    (all tokens) - and on every channel for the extreme activations of the first 64 tokens."""
+    from tests.gpu_util import pack_weights, run_gemm_i8
+    m = si.VIT_B16_TOKENS
+    w = si.gaussian_weights(n, k, seed=n + k)
+    codes, meta, coef = O.quantize_geo(w, 64, 3)
+    cq, sc = O.quantize_coefficients_int8(coef)
+    xq, sx = O.quantize_activations_int8(si.f32_activations(m, k, seed=41))
+    xq[:32] = 127
+    xq[32:64] = -127
+    d, packed = pack_weights(n, k, 64, 3, codes, meta, coef)
+    acc, y = run_gemm_i8(d, packed, xq, sx, cq, sc)
+    rows = si.sample_rows(n, 48, seed=3)
+    a1, a2, y_ref = O.linear_i32(codes, meta, cq, sc, xq, sx, 64, 3, rows=rows)
+    assert np.array_equal(acc[0][:, rows], a1) and np.array_equal(acc[1][:, rows], a2)
+    assert O.normwise_rel_err(y[:, rows], y_ref) <= TIGHT
+    b1, b2, _ = O.linear_i32(codes, meta, cq, sc, xq[:64], sx[:64], 64, 3)
+    assert np.array_equal(acc[0][:64], b1) and np.array_equal(acc[1][:64], b2)
+
+
+# ------------------------------------------------------------------------------------- boundary behaviour
+def test_argument_errors_return_status_without_launching(goq):
+    d = goq.desc(32, 256, 64, 3)
+    packed = torch.zeros(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
+    x = torch.zeros((1, 256), dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros((1, 32), dtype=torch.float32, device="cuda")
+
+    def status(fn, *a, **kw):
+        try:
+            fn(*a, **kw)
+        except goq.GoqError as e:
+            return e.status
+        return goq.OK
+
+    assert status(goq.gemv, d, packed, x, 0, y, goq.F32) == goq.ERR_INVALID_ARG
+    assert status(goq.gemv, d, packed, x, 17, y, goq.F32) == goq.ERR_INVALID_ARG
+    assert status(goq.gemv, d, packed, x, 1, y, 5) == goq.ERR_INVALID_ARG
+    assert status(goq.gemv, d, None, x, 1, y, goq.F32) == goq.ERR_INVALID_ARG
+    assert status(goq.gemv, goq.desc(32, 250, 64, 3), packed, x, 1, y, goq.F32) == goq.ERR_INVALID_ARG
+    xo = torch.zeros(2 * 256 + 8, dtype=torch.bfloat16, device="cuda")[1:]
+    assert status(goq.gemv, d, packed, xo, 1, y, goq.F32) == goq.ERR_ALIGNMENT
+    assert status(goq.gemv, d, packed[16:], x, 1, y, goq.F32) == goq.ERR_ALIGNMENT
+    small = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    z = torch.zeros(32 * 256, dtype=torch.uint8, device="cuda")
+    assert status(goq.pack, d, z, z, z, small) == goq.ERR_WORKSPACE
+    # integer path: static overflow bound and missing operands
+    big = goq.desc(16, 16768, 128, 3)
+    pb = torch.zeros(goq.packed_bytes(big), dtype=torch.uint8, device="cuda")
+    xi = torch.zeros((1, 16768), dtype=torch.int8, device="cuda")
+    cqz = torch.zeros((16, 131, 2), dtype=torch.int8, device="cuda")
+    acc = torch.zeros((2, 1, 16), dtype=torch.int32, device="cuda")
+    assert status(goq.gemm, big, pb, xi, 1, goq.I8, cq=cqz, acc=acc) == goq.ERR_OVERFLOW_BOUND
+    assert status(goq.gemm, d, packed, xi, 1, goq.I8, acc=acc) == goq.ERR_INVALID_ARG
+    assert status(goq.gemm, d, packed, x, 1, 9, y=y) == goq.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert float(y.abs().sum()) == 0.0
+
+
+def test_outputs_do_not_spill_past_their_buffers(goq):
+    from tests.gpu_util import pack_weights, dev
+    n, k, batch = 40, 192, 3
+    codes, meta, coef = _quantized(n, k, 64, 3, seed=51)
+    d, packed = pack_weights(n, k, 64, 3, codes, meta, coef)
+    x = dev(si.bf16_activations(batch, k, seed=52))
+    for variant in (1, 2):
+        buf = torch.full((batch * n + 64,), 7.5, dtype=torch.float32, device="cuda")
+        y = buf[32:32 + batch * n]
+        prev = goq.set_gemv_variant(variant)
+        goq.gemv(d, packed, x, batch, y, goq.F32)
+        goq.set_gemv_variant(prev)
+        torch.cuda.synchronize()
+        h = buf.cpu().numpy()
+        assert np.all(h[:32] == 7.5) and np.all(h[-32:] == 7.5) and not np.any(h[32:-32] == 7.5)
+
+
+def test_host_buffer_entry_point(goq):
+    from tests.gpu_util import pack_weights
+    n, k, batch = 64, 256, 4
+    codes, meta, coef = _quantized(n, k, 64, 3, seed=61)
+    d, packed = pack_weights(n, k, 64, 3, codes, meta, coef)
+    xb = si.bf16_activations(batch, k, seed=62)
+    xh = torch.from_numpy(xb.view(np.int16)).pin_memory()
+    yh = torch.zeros((batch, n), dtype=torch.float32).pin_memory()
+    xs = torch.empty((batch, k), dtype=torch.bfloat16, device="cuda")
+    ys = torch.empty((batch, n), dtype=torch.float32, device="cuda")
+    goq.gemv_host(d, packed, xh, batch, yh, goq.F32, xs, ys)
+    torch.cuda.synchronize()
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 64, 3)
+    assert O.normwise_rel_err(yh.numpy().astype(np.float64), y_ref) <= TIGHT
