@@ -1,0 +1,423 @@
+#!/usr/bin/env python
+"""Benchmark of the dual-basis PoT linear path on B200.
+
+Default arm: the CUDA path through the C ABI. A "step" is one batch-1 decode pass over every
+linear of a LLaMA-2-7B-shaped stack (32 layers x 7 linears = 224 W3/A16 GEMVs, group 128): about
+3.2 GB of packed weights per step, far larger than L2, so every step streams from HBM.
+`value` = algorithmic weight+activation bytes per step / device time (GB/s), summed over ranks.
+
+`--impl reference`: the CPU oracle timed as it stands on a bounded sample of the same workload.
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import synth_inputs as si  # noqa: E402
+
+GROUP = 128
+WBITS = 3
+METRIC = "w3a16_gemv_hbm_gbs"
+UNIT = "GB/s"
+WORKLOAD = "llama2-7b-shaped linear stack (32 layers x 7 linears), W3 dual-basis PoT, group 128, batch-1 decode GEMV"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), float(p.get("bf16_tflops", 1590.0)), "measured (MEASURED_PEAKS.json)"
+    return 6650.0, 1590.0, "fallback (earlier measurement on this pool)"
+
+
+def algorithmic_bytes(n, k, batch, y_bytes=4):
+    """Weights (codes + 0.75-bit records + fp16 coefficient pairs) + activations in + outputs."""
+    return n * k * (4 * WBITS + 3) // 32 + n * (k // GROUP) * 4 + batch * k * 2 + batch * n * y_bytes
+
+
+# ---------------------------------------------------------------------------------------------
+# clock sampling during the timed region (NVML, read-only)
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    def __init__(self, device_index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons", None)
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                if get_reasons:
+                    r = get_reasons(self.h)
+                    for k, bit in names.items():
+                        if r & bit:
+                            self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.004)
+
+    def __enter__(self):
+        if self.nv:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ---------------------------------------------------------------------------------------------
+def oracle_sample(rows_per_linear=2048, seed=0):
+    """One layer's seven linears restricted to `rows_per_linear` output rows each, batch 1."""
+    items = []
+    for i, (name, n, k) in enumerate(si.LLAMA2_7B_LINEARS):
+        r = min(rows_per_linear, n)
+        codes, meta, coef = si.random_quantized(r, k, GROUP, WBITS, seed=seed * 7 + i)
+        x = si.bf16_bits_to_f64(si.bf16_activations(1, k, seed=100 + i))
+        items.append((codes, meta, coef, x, algorithmic_bytes(r, k, 1)))
+    return items
+
+
+def time_oracle(items, repeats=1):
+    from oracle import goq_oracle as O
+    best = float("inf")
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        for codes, meta, coef, x, _ in items:
+            O.linear_f64(codes, meta, coef, x, GROUP, WBITS)
+        best = min(best, time.perf_counter() - t0)
+    nbytes = sum(it[4] for it in items)
+    return nbytes / best / 1e9, best
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    items = oracle_sample()
+    for _ in range(args.warmup):
+        time_oracle(items)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time_oracle(items)
+    dt = (time.perf_counter() - t0) / args.steps
+    nbytes = sum(it[4] for it in items)
+    val = nbytes / dt / 1e9
+    sample = "one layer's 7 linears x 2048 output rows each, batch 1, per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# CUDA arm
+# ---------------------------------------------------------------------------------------------
+def build_stack(goq, torch, layers, seed0, batch):
+    """Random W3 records generated on the device (seeded), packed by goq_pack."""
+    gen = torch.Generator(device="cuda")
+    stack = []
+    for layer in range(layers):
+        for idx, (name, n, k) in enumerate(si.LLAMA2_7B_LINEARS):
+            gen.manual_seed(seed0 + layer * 7 + idx)
+            d = goq.desc(n, k, GROUP, WBITS)
+            codes = torch.randint(0, 1 << WBITS, (n, k), dtype=torch.uint8, device="cuda", generator=gen)
+            meta = torch.randint(0, 64, (n, k // 8), dtype=torch.uint8, device="cuda", generator=gen)
+            coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * 0.03).to(torch.float16)
+            packed = torch.empty(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
+            goq.pack(d, codes, meta, coef, packed)
+            x = torch.randn((batch, k), device="cuda", generator=gen).to(torch.bfloat16)
+            y = torch.empty((batch, n), dtype=torch.float32, device="cuda")
+            stack.append({"d": d, "packed": packed, "x": x, "y": y, "n": n, "k": k})
+            del codes, meta, coef
+    torch.cuda.synchronize()
+    return stack
+
+
+def capture(torch, fn):
+    """Capture fn() (a sequence of library calls on the current stream) into a CUDA graph."""
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        fn()  # warm-up outside capture
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    return g
+
+
+def time_graph(torch, graph, steps, warmup):
+    for _ in range(warmup):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps  # ms per step
+
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2605_26092_b200 import build
+    build.build()
+    from paper_2605_26092_b200 import goq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    hbm_peak, tf_peak, peak_src = measured_peaks()
+
+    layers = args.layers
+    stack = build_stack(goq, torch, layers, seed0=1000 * rank, batch=1)
+    n_lin = len(stack)
+    step_bytes = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack)
+
+    def step():
+        for s in stack:
+            goq.gemv(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32)
+
+    graph = capture(torch, step)
+
+    # ---- timed region: warm-up, then exactly K steps between barriers ---------------------------
+    for _ in range(max(args.warmup, 3)):
+        graph.replay()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with sampler:
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    ms = e0.elapsed_time(e1) / args.steps
+    t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    value = world * step_bytes / (ms_max * 1e-3) / 1e9
+
+    # ---- end to end: host buffers in, host buffers out, through goq_gemv_host -------------------
+    host = []
+    for s in stack:
+        xh = s["x"].cpu().pin_memory()
+        yh = torch.empty((1, s["n"]), dtype=torch.float32).pin_memory()
+        host.append((xh, yh))
+
+    def step_e2e():
+        for s, (xh, yh) in zip(stack, host):
+            goq.gemv_host(s["d"], s["packed"], xh, 1, yh, goq.F32, s["x"], s["y"])
+
+    g2 = capture(torch, step_e2e)
+    e2e_steps = max(3, args.steps // 4)
+    ms_e2e = time_graph(torch, g2, e2e_steps, 3)
+    t2 = torch.tensor([ms_e2e], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+    e2e_val = world * step_bytes / (float(t2.item()) * 1e-3) / 1e9
+    h2d = sum(s["k"] * 2 for s in stack)
+    d2h = sum(s["n"] * 4 for s in stack)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- rank 0 only: extras (other batch sizes, per-shape times, GEMM, integer path) and CPU baseline
+    extras = {}
+    if not args.no_extras:
+        extras = run_extras(torch, goq, stack, layers, tf_peak)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        items = oracle_sample()
+        gbs, secs = time_oracle(items, repeats=3)
+        cpu = {"value": gbs, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+               "sample": "one layer's 7 linears x 2048 output rows each, batch 1 (%.2f s per pass, best of 3)" % secs}
+
+    launch_bytes = step_bytes / n_lin
+    launch_ms = ms / n_lin
+    achieved = launch_bytes / (launch_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "layers": layers, "linears_per_step": n_lin, "batch": 1,
+                   "bytes_per_step": step_bytes, "l2": "weights per step %.2f GB >> 126 MB L2, no flush needed" % (step_bytes / 1e9),
+                   "launch": "one CUDA graph of %d goq_gemv nodes per step" % n_lin,
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
+                     "traffic": args.traffic_bytes, "peak_source": peak_src, "frac_of_8000_nominal": achieved / 8000.0,
+                     "kernel": "linear_mma_kernel<3,1>", "bytes_per_launch_avg": launch_bytes, "us_per_launch_avg": launch_ms * 1e3},
+        "cpu_baseline": cpu,
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "launch": "one CUDA graph of goq_gemv_host calls (pinned H2D, kernel, D2H per linear)"},
+        "gpu_launches": args.steps * n_lin,
+        "clocks": sampler.summary(),
+        "extras": extras,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_extras(torch, goq, stack, layers, tf_peak):
+    out = {}
+    n_lin = len(stack)
+    # decode at batch 4 and 16 over the same stack
+    for batch in (4, 16):
+        xs = [torch.randn((batch, s["k"]), device="cuda").to(torch.bfloat16) for s in stack]
+        ys = [torch.empty((batch, s["n"]), dtype=torch.float32, device="cuda") for s in stack]
+
+        def step():
+            for s, x, y in zip(stack, xs, ys):
+                goq.gemv(s["d"], s["packed"], x, batch, y, goq.F32)
+
+        g = capture(torch, step)
+        ms = time_graph(torch, g, 20, 3)
+        nbytes = sum(algorithmic_bytes(s["n"], s["k"], batch) for s in stack)
+        out["gemv_batch%d_gbs" % batch] = nbytes / (ms * 1e-3) / 1e9
+        del g, xs, ys
+    # per-shape batch-1 time (rotating over the layers' copies of that shape, so each launch reads cold weights)
+    shapes = {}
+    for idx, (name, n, k) in enumerate(si.LLAMA2_7B_LINEARS):
+        if (n, k) in shapes:
+            continue
+        sel = [s for s in stack if (s["n"], s["k"]) == (n, k)]
+
+        def step():
+            for s in sel:
+                goq.gemv(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32)
+
+        g = capture(torch, step)
+        ms = time_graph(torch, g, 20, 3)
+        us = ms * 1e3 / len(sel)
+        shapes[(n, k)] = {"us": us, "gbs": algorithmic_bytes(n, k, 1) / (us * 1e-6) / 1e9}
+        del g
+    out["gemv_batch1_per_shape"] = {"%dx%d" % k: v for k, v in shapes.items()}
+    # prefill GEMM, M = 2048, one layer's seven linears
+    m = 2048
+    layer0 = stack[:7]
+    xs = [torch.randn((m, s["k"]), device="cuda").to(torch.bfloat16) for s in layer0]
+    ys = [torch.empty((m, s["n"]), dtype=torch.float32, device="cuda") for s in layer0]
+
+    def step_gemm():
+        for s, x, y in zip(layer0, xs, ys):
+            goq.gemm(s["d"], s["packed"], x, m, goq.BF16, y=y, y_dtype=goq.F32)
+
+    step_gemm()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(3):
+        step_gemm()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / 3
+    flops = sum(2.0 * m * s["n"] * s["k"] for s in layer0)
+    out["gemm_m2048_layer_tflops"] = flops / (ms * 1e-3) / 1e12
+    out["gemm_m2048_frac_of_bf16_peak"] = out["gemm_m2048_layer_tflops"] / tf_peak
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--layers", type=int, default=si.LLAMA2_7B_LAYERS)
+    ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic-bytes", type=float, default=None,
+                    help="dram bytes per launch of the dominant kernel from an ncu capture (reported as-is)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 200:
+            args.steps = 5
+        if args.warmup == 5:
+            args.warmup = 1
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()
