@@ -193,6 +193,7 @@ def build_stack(goq, torch, layers, seed0, batch):
             x = torch.randn((batch, k), device="cuda", generator=gen).to(torch.bfloat16)
             y = torch.empty((batch, n), dtype=torch.float32, device="cuda")
             stack.append({"d": d, "packed": packed, "x": x, "y": y, "n": n, "k": k})
+            build_stack.ws_bytes = max(getattr(build_stack, "ws_bytes", 256), goq.workspace_bytes(d, goq.OP_GEMV, 16))
             del codes, meta, coef
     torch.cuda.synchronize()
     return stack
@@ -244,10 +245,13 @@ def run_cuda(args):
     stack = build_stack(goq, torch, layers, seed0=1000 * rank, batch=1)
     n_lin = len(stack)
     step_bytes = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack)
+    # one scratch buffer shared by all calls: launches on one stream run in order
+    ws = torch.empty(build_stack.ws_bytes, dtype=torch.uint8, device="cuda")
+    goq.workspace_init(ws)
 
     def step():
         for s in stack:
-            goq.gemv(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32)
+            goq.gemv(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, ws=ws)
 
     graph = capture(torch, step)
 
@@ -284,7 +288,7 @@ def run_cuda(args):
 
     def step_e2e():
         for s, (xh, yh) in zip(stack, host):
-            goq.gemv_host(s["d"], s["packed"], xh, 1, yh, goq.F32, s["x"], s["y"])
+            goq.gemv_host(s["d"], s["packed"], xh, 1, yh, goq.F32, s["x"], s["y"], ws=ws)
 
     g2 = capture(torch, step_e2e)
     e2e_steps = max(3, args.steps // 4)
@@ -304,7 +308,7 @@ def run_cuda(args):
     # ---- rank 0 only: extras (other batch sizes, per-shape times, GEMM, integer path) and CPU baseline
     extras = {}
     if not args.no_extras:
-        extras = run_extras(torch, goq, stack, layers, tf_peak)
+        extras = run_extras(torch, goq, stack, layers, tf_peak, ws)
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         items = oracle_sample()
@@ -338,7 +342,7 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
-def run_extras(torch, goq, stack, layers, tf_peak):
+def run_extras(torch, goq, stack, layers, tf_peak, ws):
     out = {}
     n_lin = len(stack)
     # decode at batch 4 and 16 over the same stack
@@ -348,7 +352,7 @@ def run_extras(torch, goq, stack, layers, tf_peak):
 
         def step():
             for s, x, y in zip(stack, xs, ys):
-                goq.gemv(s["d"], s["packed"], x, batch, y, goq.F32)
+                goq.gemv(s["d"], s["packed"], x, batch, y, goq.F32, ws=ws)
 
         g = capture(torch, step)
         ms = time_graph(torch, g, 20, 3)
@@ -364,7 +368,7 @@ def run_extras(torch, goq, stack, layers, tf_peak):
 
         def step():
             for s in sel:
-                goq.gemv(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32)
+                goq.gemv(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, ws=ws)
 
         g = capture(torch, step)
         ms = time_graph(torch, g, 20, 3)

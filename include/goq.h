@@ -79,6 +79,15 @@ size_t goq_algorithmic_bytes(const goq_desc* desc);
 /* Scratch bytes goq_gemv / goq_gemm need for `m` activation rows (may be 0). */
 size_t goq_workspace_bytes(const goq_desc* desc, int op, int m);
 
+/* Zero-fill a scratch buffer (asynchronous on `stream`). A scratch buffer must be initialised once
+ * before its first use; every call leaves it ready for the next one. One buffer may serve any number
+ * of calls that run one after another on a stream; calls that may overlap need separate buffers. */
+goq_status goq_workspace_init(void* ws, size_t ws_bytes, void* stream);
+
+/* Read the device-side status word of a scratch buffer after synchronising `stream`:
+ * GOQ_OK, or GOQ_ERR_TIMEOUT if a kernel gave up on a bounded wait (its outputs are then undefined). */
+goq_status goq_workspace_status(const void* ws, void* stream, int* status_out);
+
 /* goq_pack - re-tile quantizer output into the layout the kernels stream (Sections 3.2-3.4 give
  * the fields; the layout is this library's own).
  *   codes     [n_out][k_in] uint8, one code per weight, value < 2^wbits
@@ -105,7 +114,8 @@ goq_status goq_unpack(const goq_desc* desc, const void* packed, uint8_t* codes_b
 /* goq_gemv - decode-time layer for a small batch (Eq. 4, float activations).
  *   x_bf16   [batch][k_in] bf16, 16-byte aligned, batch in 1..16
  *   y        out [batch][n_out], y_dtype GOQ_BF16 or GOQ_F32
- *   ws       scratch of goq_workspace_bytes(desc, GOQ_OP_GEMV, batch) bytes (may be NULL if that is 0)
+ *   ws       scratch of goq_workspace_bytes(desc, GOQ_OP_GEMV, batch) bytes, 256-byte aligned,
+ *            initialised once with goq_workspace_init (may be NULL if the size is 0)
  * Each PoT term is applied to the activation as an exponent shift; sums are fp32. */
 goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16, int batch, void* y,
                     int y_dtype, void* ws, size_t ws_bytes, void* stream);
@@ -133,7 +143,8 @@ goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x
                          size_t ws_bytes, void* stream);
 
 /* Force a kernel variant (benchmarks and tests only): 0 = automatic, 1 = scalar exponent-add
- * kernel, 2 = tensor-core fragment kernel. Process-wide. Returns the previous value. */
+ * kernel, 2 = tensor-core fragment kernel, 3 = streaming tensor-core kernel. Process-wide.
+ * Returns the previous value. */
 int goq_set_gemv_variant(int variant);
 
 #ifdef __cplusplus

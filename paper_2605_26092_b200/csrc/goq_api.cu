@@ -65,7 +65,7 @@ size_t goq_algorithmic_bytes(const goq_desc* desc) {
 size_t goq_workspace_bytes(const goq_desc* desc, int op, int m) {
     Geometry g;
     if (!goq::make_geometry(desc, &g) || m <= 0) return 0;
-    (void)op;
+    if (op == GOQ_OP_GEMV && m <= 16 && goq::gemv_stream_supported(g)) return goq::gemv_stream_workspace(g);
     return 0;
 }
 
@@ -97,10 +97,16 @@ goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16
     if (y_dtype != GOQ_BF16 && y_dtype != GOQ_F32) return GOQ_ERR_INVALID_ARG;
     if (!aligned(packed, 128) || !aligned(x_bf16, 16) || !aligned(y, y_dtype == GOQ_F32 ? 4 : 2))
         return GOQ_ERR_ALIGNMENT;
-    (void)ws;
-    (void)ws_bytes;
     if (goq_status s = check_arch()) return s;
     const int variant = g_gemv_variant.load(std::memory_order_relaxed);
+    bool use_stream = goq::gemv_stream_supported(g) && (variant == 0 || variant == 3);
+    if (variant == 3 && !use_stream) return GOQ_ERR_UNSUPPORTED;
+    if (use_stream) {
+        if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
+        if (ws_bytes < goq::gemv_stream_workspace(g)) return GOQ_ERR_WORKSPACE;
+        if (!goq::stream_hash_is_bijective()) return GOQ_ERR_UNSUPPORTED;
+        return from_cuda(goq::launch_gemv_stream(g, packed, x_bf16, batch, y, y_dtype, ws, (cudaStream_t)stream));
+    }
     bool use_mma = goq::linear_mma_supported(g);
     if (variant == 1) use_mma = false;
     if (variant == 2 && !use_mma) return GOQ_ERR_UNSUPPORTED;
@@ -151,6 +157,21 @@ goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x
     goq_status s = goq_gemv(desc, packed, x_stage, batch, y_stage, y_dtype, ws, ws_bytes, stream);
     if (s != GOQ_OK) return s;
     if (cudaMemcpyAsync(y_host, y_stage, yb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GOQ_ERR_CUDA;
+    return GOQ_OK;
+}
+
+goq_status goq_workspace_init(void* ws, size_t ws_bytes, void* stream) {
+    if (!ws || ws_bytes == 0) return GOQ_ERR_INVALID_ARG;
+    return from_cuda(cudaMemsetAsync(ws, 0, ws_bytes, (cudaStream_t)stream));
+}
+
+goq_status goq_workspace_status(const void* ws, void* stream, int* status_out) {
+    if (!ws || !status_out) return GOQ_ERR_INVALID_ARG;
+    int v = 0;
+    if (cudaMemcpyAsync(&v, ws, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+        return GOQ_ERR_CUDA;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return GOQ_ERR_CUDA;
+    *status_out = v;
     return GOQ_OK;
 }
 

@@ -1,17 +1,21 @@
 // Shared device/host helpers of libgoq: packed-layout index arithmetic and code decoding.
 //
 // Layout GOQ_LAYOUT_TILE16 ("tile16"). Rows are padded to a multiple of 16 (a row tile), k to a
-// multiple of 128 (a k-block). One 32-bit word holds one micro-block (8 weights, Section 3.3 of
-// the paper): nibble i, bits [4i+2:4i], is the code of weight i. For wbits <= 3 the six bits of
-// the exchange record sit in bit 3 of nibbles 0..5; for wbits = 4 the record is a byte in a side
-// plane with the same indexing. A (row tile, k-block) pair owns 256 consecutive words (1 KiB):
-//     word = v*128 + (g*4 + t)*4 + c
-// for row = 16*T + 8*v + g (v in 0..1, g in 0..7) and micro-block 4*c + t of the k-block
-// (c = 32-wide chunk 0..3, t = position 0..3 inside the chunk). A warp whose lane id is g*4+t
-// therefore reads 512 contiguous bytes with one 128-bit load per lane and every lane receives
-// whole micro-blocks of its two rows, which is what lets the exchange stay inside a thread.
-// Coefficient pairs (fp16 c1 in the low half, c2 in the high half of a 32-bit word) live in a
-// second plane: word (T*J + j)*16 + (row % 16) for group j of J = k_pad/group.
+// multiple of 128 (a k-block). The buffer is a sequence of unit records, one per (row tile T,
+// k-block bk), in the order T*k_blocks + bk, so a run of consecutive records is one contiguous
+// byte range (what a bulk copy wants). A unit record holds
+//   [0, 1024)            256 micro-block words. One 32-bit word = one micro-block (8 weights,
+//                        Section 3.3 of the paper): nibble i, bits [4i+2:4i], is the code of weight i;
+//                        for wbits <= 3 the six bits of the exchange record sit in bit 3 of nibbles 0..5.
+//                            word = v*128 + (g*4 + t)*4 + c
+//                        for row = 16*T + 8*v + g (v in 0..1, g in 0..7) and micro-block 4*c + t of the
+//                        k-block (c = 32-wide chunk 0..3, t = position 0..3 inside the chunk). A warp whose
+//                        lane id is g*4+t reads 512 contiguous bytes with one 128-bit load per lane and
+//                        every lane receives whole micro-blocks of its two rows, which keeps the exchange
+//                        inside a thread.
+//   [1024, 1024 + 64*G)  coefficient pairs of the unit's G = 128/group macro-blocks: word jj*16 + (row % 16),
+//                        fp16 c1 in the low half, c2 in the high half.
+//   then, wbits = 4 only: 256 record bytes, indexed like the words.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -22,13 +26,16 @@ namespace goq {
 constexpr int kTileRows = 16;
 constexpr int kBlockK = 128;
 constexpr int kWordsPerBlock = 256;
+constexpr int kCodeBytesPerUnit = kWordsPerBlock * 4;
 
 struct Geometry {
     int n_out, k_in, group, wbits;
     int n_pad, k_pad;
-    int n_tiles, k_blocks, n_groups;       // n_groups counts padded groups: k_pad / group
-    size_t code_words;                     // n_pad * k_pad / 8
-    size_t coef_off_bytes, meta_off_bytes; // plane offsets from the packed base (meta: wbits = 4 only)
+    int n_tiles, k_blocks, n_groups;  // n_groups counts padded groups: k_pad / group
+    int groups_per_block;             // 128 / group
+    int unit_bytes;                   // bytes of one unit record
+    int meta_off;                     // offset of the record-byte plane inside a unit (wbits = 4 only)
+    size_t n_units;
     size_t total_bytes;
 };
 
@@ -48,26 +55,21 @@ __host__ inline bool make_geometry(const goq_desc* d, Geometry* g) {
     g->n_tiles = g->n_pad / kTileRows;
     g->k_blocks = g->k_pad / kBlockK;
     g->n_groups = g->k_pad / gr;
-    g->code_words = (size_t)g->n_pad * (size_t)(g->k_pad / 8);
-    size_t off = g->code_words * 4;
-    off = align_up(off, 128);
-    g->coef_off_bytes = off;
-    off += (size_t)g->n_pad * (size_t)g->n_groups * 4;
-    off = align_up(off, 128);
-    g->meta_off_bytes = off;
-    if (d->wbits == 4) { off += g->code_words; off = align_up(off, 128); }
-    g->total_bytes = off;
+    g->groups_per_block = kBlockK / gr;
+    g->meta_off = kCodeBytesPerUnit + 64 * g->groups_per_block;
+    g->unit_bytes = g->meta_off + (d->wbits == 4 ? kWordsPerBlock : 0);
+    g->n_units = (size_t)g->n_tiles * g->k_blocks;
+    g->total_bytes = g->n_units * (size_t)g->unit_bytes;
     return true;
 }
 
-// index of the word of (row, micro-block mb = k/8) in the code plane
-__host__ __device__ inline size_t word_index(int row, int mb, int k_blocks) {
-    int T = row >> 4, rr = row & 15, v = rr >> 3, g = rr & 7;
-    int bk = mb >> 4, m = mb & 15, c = m >> 2, t = m & 3;
-    return ((size_t)T * k_blocks + bk) * kWordsPerBlock + v * 128 + (g * 4 + t) * 4 + c;
+// index of the word of (row, micro-block mb of the k-block) inside its unit record
+__host__ __device__ inline int word_in_unit(int row, int mb) {
+    int rr = row & 15, v = rr >> 3, g = rr & 7, c = (mb & 15) >> 2, t = mb & 3;
+    return v * 128 + (g * 4 + t) * 4 + c;
 }
-__host__ __device__ inline size_t coef_index(int row, int j, int n_groups) {
-    return ((size_t)(row >> 4) * n_groups + j) * 16 + (row & 15);
+__host__ __device__ inline size_t unit_offset(int tile, int bk, int k_blocks, int unit_bytes) {
+    return ((size_t)tile * k_blocks + bk) * (size_t)unit_bytes;
 }
 
 // ---- scalar decode helpers (used by pack/unpack and the scalar kernels) --------------------

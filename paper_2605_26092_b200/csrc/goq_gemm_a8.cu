@@ -26,7 +26,8 @@ constexpr int kA8Tokens = 128;
 
 template <int WB>
 __global__ void __launch_bounds__(kA8Tokens)
-gemm_a8_dp4a_kernel(const uint32_t* __restrict__ words, const int8_t* __restrict__ x, const float* __restrict__ sx,
+gemm_a8_dp4a_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int8_t* __restrict__ x,
+                    const float* __restrict__ sx,
                     const int8_t* __restrict__ cq, const float* __restrict__ sc, void* __restrict__ y, int y_dtype,
                     int32_t* __restrict__ acc_out, int n_out, int k_in, int k_blocks, int group, int m_total) {
     __shared__ __align__(16) int8_t b1s[16][kBlockK];
@@ -47,7 +48,8 @@ gemm_a8_dp4a_kernel(const uint32_t* __restrict__ words, const int8_t* __restrict
         __syncthreads();
         // expand this block's 256 micro-block words to int8 operands
         for (int wi = threadIdx.x; wi < kWordsPerBlock; wi += kA8Tokens) {
-            const uint32_t w = words[((size_t)T * k_blocks + bk) * kWordsPerBlock + wi];
+            const uint32_t w =
+                reinterpret_cast<const uint32_t*>(packed + unit_offset(T, bk, k_blocks, unit_bytes))[wi];
             const int v = wi >> 7, ln = (wi >> 2) & 31, c = wi & 3;
             const int row = v * 8 + (ln >> 2), kk = c * 32 + (ln & 3) * 8;
             const uint32_t meta = gather_meta(w);
@@ -126,13 +128,13 @@ gemm_a8_dp4a_kernel(const uint32_t* __restrict__ words, const int8_t* __restrict
 
 cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* x, int m, const float* sx,
                            const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, cudaStream_t st) {
-    auto* words = (const uint32_t*)packed;
+    auto* words = (const uint8_t*)packed;
     dim3 grid(g.n_tiles, (m + kA8Tokens - 1) / kA8Tokens), block(kA8Tokens);
     if (g.wbits == 3)
-        gemm_a8_dp4a_kernel<3><<<grid, block, 0, st>>>(words, x, sx, cq, sc, y, y_dtype, acc, g.n_out, g.k_in,
+        gemm_a8_dp4a_kernel<3><<<grid, block, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, g.n_out, g.k_in,
                                                        g.k_blocks, g.group, m);
     else
-        gemm_a8_dp4a_kernel<2><<<grid, block, 0, st>>>(words, x, sx, cq, sc, y, y_dtype, acc, g.n_out, g.k_in,
+        gemm_a8_dp4a_kernel<2><<<grid, block, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, g.n_out, g.k_in,
                                                        g.k_blocks, g.group, m);
     return cudaGetLastError();
 }

@@ -29,10 +29,9 @@ __device__ __forceinline__ float pot_apply(float x, uint32_t e, uint32_t sign) {
 
 template <int WB, int MB>
 __global__ void __launch_bounds__(128)
-gemv_scalar_kernel(const uint32_t* __restrict__ words, const uint32_t* __restrict__ coefp,
-                   const uint8_t* __restrict__ metap, const uint16_t* __restrict__ x, void* __restrict__ y,
-                   int y_dtype, int n_out, int k_in, int n_tiles, int k_blocks, int n_groups, int group,
-                   int batch) {
+gemv_scalar_kernel(const uint8_t* __restrict__ packed, int unit_bytes, int meta_off,
+                   const uint16_t* __restrict__ x, void* __restrict__ y,
+                   int y_dtype, int n_out, int k_in, int n_tiles, int k_blocks, int group, int batch) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int T = blockIdx.x * 4 + warp;
     if (T >= n_tiles) return;
@@ -47,13 +46,14 @@ gemv_scalar_kernel(const uint32_t* __restrict__ words, const uint32_t* __restric
         for (int m = 0; m < MB; ++m) acc[v][m] = s1[v][m] = s2[v][m] = 0.f;
 
     for (int bk = 0; bk < k_blocks; ++bk) {
-        const size_t wbase = ((size_t)T * k_blocks + bk) * kWordsPerBlock;
-        const uint4* blk = reinterpret_cast<const uint4*>(words + wbase);
+        const uint8_t* unit = packed + unit_offset(T, bk, k_blocks, unit_bytes);
+        const uint4* blk = reinterpret_cast<const uint4*>(unit);
+        const uint32_t* coefp = reinterpret_cast<const uint32_t*>(unit + kCodeBytesPerUnit);
         uint4 wv[2] = {blk[lane], blk[32 + lane]};
         uint32_t mv[2] = {0, 0};
         if (WB == 4) {
-            mv[0] = *reinterpret_cast<const uint32_t*>(metap + wbase + lane * 4);
-            mv[1] = *reinterpret_cast<const uint32_t*>(metap + wbase + 128 + lane * 4);
+            mv[0] = *reinterpret_cast<const uint32_t*>(unit + meta_off + lane * 4);
+            mv[1] = *reinterpret_cast<const uint32_t*>(unit + meta_off + 128 + lane * 4);
         }
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -89,10 +89,10 @@ gemv_scalar_kernel(const uint32_t* __restrict__ words, const uint32_t* __restric
                 }
             }
             if (group < 32 || ((c + 1) * 32) % group == 0) {
-                const int j = k0 / group;
+                const int jj = (c * 32 + t * 8) / group;  // macro-block inside this k-block
 #pragma unroll
                 for (int v = 0; v < 2; ++v) {
-                    uint32_t cf = coefp[((size_t)T * n_groups + j) * 16 + v * 8 + g];
+                    uint32_t cf = coefp[jj * 16 + v * 8 + g];
                     float c1 = __half2float(__ushort_as_half((unsigned short)(cf & 0xFFFFu)));
                     float c2 = __half2float(__ushort_as_half((unsigned short)(cf >> 16)));
 #pragma unroll
@@ -123,13 +123,10 @@ template <int WB>
 static cudaError_t launch_scalar_wb(const Geometry& g, const void* packed, const void* x, int batch, void* y,
                                     int y_dtype, cudaStream_t st) {
     auto* base = (const uint8_t*)packed;
-    auto* words = (const uint32_t*)base;
-    auto* coefp = (const uint32_t*)(base + g.coef_off_bytes);
-    auto* metap = base + g.meta_off_bytes;
     dim3 grid((g.n_tiles + 3) / 4), block(128);
 #define GOQ_LAUNCH_SC(MB)                                                                                      \
-    gemv_scalar_kernel<WB, MB><<<grid, block, 0, st>>>(words, coefp, metap, (const uint16_t*)x, y, y_dtype,    \
-                                                       g.n_out, g.k_in, g.n_tiles, g.k_blocks, g.n_groups,     \
+    gemv_scalar_kernel<WB, MB><<<grid, block, 0, st>>>(base, g.unit_bytes, g.meta_off, (const uint16_t*)x, y,  \
+                                                       y_dtype, g.n_out, g.k_in, g.n_tiles, g.k_blocks,        \
                                                        g.group, batch)
     if (batch <= 1) GOQ_LAUNCH_SC(1);
     else if (batch <= 2) GOQ_LAUNCH_SC(2);
@@ -231,9 +228,9 @@ constexpr int kMmaWarps = 8;
 
 template <int WB, int NT>
 __global__ void __launch_bounds__(kMmaWarps * 32)
-linear_mma_kernel(const uint32_t* __restrict__ words, const uint32_t* __restrict__ coefp,
-                  const uint8_t* __restrict__ metap, const uint16_t* __restrict__ x, void* __restrict__ y,
-                  int y_dtype, int n_out, int k_in, int k_blocks, int n_groups, int group, int m_total) {
+linear_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, int meta_off,
+                  const uint16_t* __restrict__ x, void* __restrict__ y,
+                  int y_dtype, int n_out, int k_in, int k_blocks, int group, int m_total) {
     __shared__ uint4 lut[64];
     extern __shared__ float red[];  // [kMmaWarps][32][NT*4]
     if (threadIdx.x < 64) lut[threadIdx.x] = make_exchange_entry(threadIdx.x);
@@ -252,14 +249,15 @@ linear_mma_kernel(const uint32_t* __restrict__ words, const uint32_t* __restrict
         for (int r = 0; r < 4; ++r) acc[nt][r] = d1[nt][r] = d2[nt][r] = 0.f;
 
     for (int bk = warp; bk < k_blocks; bk += kMmaWarps) {
-        const size_t wbase = ((size_t)T * k_blocks + bk) * kWordsPerBlock;
-        const uint4* blk = reinterpret_cast<const uint4*>(words + wbase);
+        const uint8_t* unit = packed + unit_offset(T, bk, k_blocks, unit_bytes);
+        const uint4* blk = reinterpret_cast<const uint4*>(unit);
+        const uint32_t* coefp = reinterpret_cast<const uint32_t*>(unit + kCodeBytesPerUnit);
         const uint4 wv0 = blk[lane], wv1 = blk[32 + lane];
         const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
         uint32_t mv0 = 0, mv1 = 0;
         if (WB == 4) {
-            mv0 = *reinterpret_cast<const uint32_t*>(metap + wbase + lane * 4);
-            mv1 = *reinterpret_cast<const uint32_t*>(metap + wbase + 128 + lane * 4);
+            mv0 = *reinterpret_cast<const uint32_t*>(unit + meta_off + lane * 4);
+            mv1 = *reinterpret_cast<const uint32_t*>(unit + meta_off + 128 + lane * 4);
         }
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -282,8 +280,7 @@ linear_mma_kernel(const uint32_t* __restrict__ words, const uint32_t* __restrict
                 mma_bf16_16816(d2[nt], Q0[2], Q1[2], Q0[3], Q1[3], xa[nt].z, xa[nt].w);
             }
             if (((c + 1) % cpg) == 0) {
-                const int j = (bk * kBlockK + c * 32) / group;
-                const uint32_t* cf = coefp + ((size_t)T * n_groups + j) * 16;
+                const uint32_t* cf = coefp + ((c * 32) / group) * 16;
                 const uint32_t cfa = cf[g], cfb = cf[8 + g];
                 const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
                 const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
@@ -328,13 +325,10 @@ template <int WB, int NT>
 static cudaError_t launch_mma_nt(const Geometry& g, const void* packed, const void* x, int m, void* y, int y_dtype,
                                  cudaStream_t st) {
     auto* base = (const uint8_t*)packed;
-    auto* words = (const uint32_t*)base;
-    auto* coefp = (const uint32_t*)(base + g.coef_off_bytes);
-    auto* metap = base + g.meta_off_bytes;
     dim3 grid(g.n_tiles, (m + 8 * NT - 1) / (8 * NT)), block(kMmaWarps * 32);
     size_t smem = (size_t)kMmaWarps * 32 * NT * 4 * sizeof(float);
-    linear_mma_kernel<WB, NT><<<grid, block, smem, st>>>(words, coefp, metap, (const uint16_t*)x, y, y_dtype,
-                                                         g.n_out, g.k_in, g.k_blocks, g.n_groups, g.group, m);
+    linear_mma_kernel<WB, NT><<<grid, block, smem, st>>>(base, g.unit_bytes, g.meta_off, (const uint16_t*)x, y,
+                                                         y_dtype, g.n_out, g.k_in, g.k_blocks, g.group, m);
     return cudaGetLastError();
 }
 

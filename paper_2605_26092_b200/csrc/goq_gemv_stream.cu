@@ -1,0 +1,494 @@
+// Decode GEMV (batch <= 16), streaming kernel.
+//
+// Eq. 4 of the paper read per macro-block:  y[m,n] = sum_j ( c1[n,j] S1 + c2[n,j] S2 ),
+// S1 = sum_{k in j} b1[n,k] x[m,k], S2 likewise with b2. b1 and b2 enter the bf16 tensor-core MMA as
+// exact PoT operands (a PoT factor only shifts the activation's exponent, so no product rounds), the
+// sums are fp32, and the coefficient multiply happens once per macro-block outside the MMA.
+//
+// Work decomposition. The packed buffer is one contiguous array of unit records (1 KiB of codes plus
+// the coefficients of 16 rows x 128 k). CTA i takes the contiguous range [U*i/G, U*(i+1)/G) of the U
+// records, so every SM streams the same number of bytes whatever the shape. A producer thread moves the
+// range through a ring of shared-memory stages with 1-D bulk async copies (mbarrier completion); eight
+// consumer warps each take one record per stage. Lane (g,t) of a consumer owns whole micro-blocks of
+// rows g and g+8, so the Strided Dual-Exchange of Section 3.3 never leaves the thread. A 16-row tile
+// that straddles CTAs is finished by whichever CTA arrives last, adding the parked partial sums in CTA
+// order: results do not depend on timing. The weight prefetch starts before the wait on the preceding
+// kernel in the stream (programmatic dependent launch); activations, outputs and the scratch buffer are
+// touched only after it.
+//
+// Every mbarrier wait is bounded. On expiry the CTA raises an abort flag, records GOQ_ERR_TIMEOUT in
+// the scratch status word and runs out its control flow (all barriers are still reached) without
+// touching data.
+#include <cuda_fp16.h>
+#include "goq_common.cuh"
+#include "goq_internal.h"
+
+namespace goq {
+
+// ------------------------------------------------------------------------------------------------
+// scratch layout: [status 256 B][tile counters][partials kMaxCtas x 2 x 256 floats]
+// ------------------------------------------------------------------------------------------------
+constexpr int kMaxCtas = 512;
+constexpr int kStatusBytes = 256;
+constexpr int kPartialFloats = 16 * 16;  // one 16-row tile x up to 16 tokens
+
+struct StreamWs {
+    size_t counters_off, partials_off, total;
+};
+__host__ inline StreamWs stream_ws_layout(const Geometry& g) {
+    StreamWs w;
+    w.counters_off = kStatusBytes;
+    w.partials_off = align_up(w.counters_off + (size_t)g.n_tiles * 4, 256);
+    w.total = w.partials_off + (size_t)kMaxCtas * 2 * kPartialFloats * sizeof(float);
+    return w;
+}
+
+// ------------------------------------------------------------------------------------------------
+// PTX helpers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t prmt_b32(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait. Returns false (and raises *abort_flag) if the phase does not complete in time or another
+// thread has already given up.
+constexpr int kSpinLimit = 1 << 22;
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    for (int it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (it > 32) __nanosleep(40);
+    }
+    *abort_flag = 1;
+    return false;
+}
+// 1-D bulk async copy global -> shared, completion counted in bytes on an mbarrier.
+// Source, destination and size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------------------------
+// weights: code word -> bf16x2 operand registers
+// ------------------------------------------------------------------------------------------------
+// bf16 bit pattern of a PoT code, high byte / low byte tables indexed by the code
+template <int WB> struct PotBytes;
+template <> struct PotBytes<3> {  // +1 +.5 +.25 0 -1 -.5 -.25 -.125
+    static constexpr uint32_t H0 = 0x003E3F3Fu, H1 = 0xBEBEBFBFu, L0 = 0x00800080u, L1 = 0x00800080u;
+};
+template <> struct PotBytes<2> {  // +1 0 -1 -.5
+    static constexpr uint32_t H0 = 0xBFBF003Fu, H1 = 0u, L0 = 0x00800080u, L1 = 0u;
+};
+
+// The six record bits sit in bit 3 of nibbles 0..5 of a word. (spare bits * kHashMul) >> 26 is a
+// bijection of the 64 records onto 0..63 (checked exhaustively on the host before the first launch),
+// which replaces gathering the bits one by one.
+constexpr uint32_t kHashMul = 0x01008420u;
+__host__ __device__ inline uint32_t record_slot(uint32_t meta) { return (scatter_meta(meta) * kHashMul) >> 26; }
+
+constexpr int kLutCopies = 8;  // one copy per lane of a quarter-warp: 128-bit lookups never share a bank
+constexpr int kLutBytes = 64 * kLutCopies * 16;
+
+// Lookup entry of one exchange record: byte selectors that route the eight high (or low) bytes of b1
+// to b2's positions 0..3 (x) and 4..7 (y), and the sign flips of those positions (z, w: bit 7 of each byte).
+__device__ inline uint4 make_exchange_entry(uint32_t meta) {
+    const int s = (int)(meta & 3u) + 1;
+    const uint32_t flips = flip_mask(meta);
+    uint32_t sel_a = 0, sel_b = 0, f_a = 0, f_b = 0;
+    for (int i = 0; i < 4; ++i) {
+        sel_a |= (uint32_t)(i ^ s) << (4 * i);
+        sel_b |= (uint32_t)((4 + i) ^ s) << (4 * i);
+        f_a |= ((flips >> i) & 1u) << (8 * i + 7);
+        f_b |= ((flips >> (4 + i)) & 1u) << (8 * i + 7);
+    }
+    return make_uint4(sel_a, sel_b, f_a, f_b);
+}
+
+// R[q] = bf16x2 (b1 element 2q, 2q+1); Q[q] the same for b2 (Section 3.3: partner i XOR s routed by a
+// byte permute, pair signs XOR-ed into the bf16 sign bit; a flipped zero is -0 and adds nothing).
+template <int WB>
+__device__ __forceinline__ void expand_word(uint32_t w, const unsigned char* __restrict__ lut_lane, uint32_t (&R)[4],
+                                            uint32_t (&Q)[4]) {
+    const uint32_t m = w & 0x77777777u, mh = m >> 16;
+    const uint32_t ha = prmt_b32(PotBytes<WB>::H0, PotBytes<WB>::H1, m), hb = prmt_b32(PotBytes<WB>::H0, PotBytes<WB>::H1, mh);
+    const uint32_t la = prmt_b32(PotBytes<WB>::L0, PotBytes<WB>::L1, m), lb = prmt_b32(PotBytes<WB>::L0, PotBytes<WB>::L1, mh);
+    R[0] = prmt_b32(la, ha, 0x5140u);
+    R[1] = prmt_b32(la, ha, 0x7362u);
+    R[2] = prmt_b32(lb, hb, 0x5140u);
+    R[3] = prmt_b32(lb, hb, 0x7362u);
+    const uint32_t h = (w - m) * kHashMul;
+    const uint4 e = *reinterpret_cast<const uint4*>(lut_lane + ((h >> 19) & 0x1F80u));
+    const uint32_t qha = prmt_b32(ha, hb, e.x) ^ e.z, qhb = prmt_b32(ha, hb, e.y) ^ e.w;
+    const uint32_t qla = prmt_b32(la, lb, e.x), qlb = prmt_b32(la, lb, e.y);
+    Q[0] = prmt_b32(qla, qha, 0x5140u);
+    Q[1] = prmt_b32(qla, qha, 0x7362u);
+    Q[2] = prmt_b32(qlb, qhb, 0x5140u);
+    Q[3] = prmt_b32(qlb, qhb, 0x7362u);
+}
+
+// ------------------------------------------------------------------------------------------------
+// streaming kernel
+// ------------------------------------------------------------------------------------------------
+constexpr int kConsumerWarps = 8;
+constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;
+constexpr int kStageUnits = kConsumerWarps;
+
+struct StreamParams {
+    const uint8_t* packed;
+    const uint16_t* x;
+    void* y;
+    int* status;
+    int* counters;
+    float* partials;
+    int n_units, unit_bytes, k_blocks, k_in, n_out, m_total, y_dtype, n_stages;
+};
+
+__device__ __forceinline__ int owner_of_unit(int u, int n_units, int n_ctas) {
+    return (int)((((long long)u + 1) * n_ctas - 1) / n_units);
+}
+__device__ __forceinline__ int range_begin(int i, int n_units, int n_ctas) {
+    return (int)((long long)n_units * i / n_ctas);
+}
+
+template <int NT>
+__device__ __forceinline__ void store_tile_output(const StreamParams& p, int T, int o, float v) {
+    const int ln = o / (NT * 4), qq = o % (NT * 4), nt = qq >> 2, r = qq & 3;
+    const int row = T * 16 + (ln >> 2) + ((r & 2) ? 8 : 0);
+    const int tok = nt * 8 + (ln & 3) * 2 + (r & 1);
+    if (row < p.n_out && tok < p.m_total) {
+        if (p.y_dtype == GOQ_F32) reinterpret_cast<float*>(p.y)[(size_t)tok * p.n_out + row] = v;
+        else reinterpret_cast<uint16_t*>(p.y)[(size_t)tok * p.n_out + row] = f32_to_bf16_rne(v);
+    }
+}
+
+// WB: weight bits (2, 3); NT: 8-token column tiles (1, 2); CPG: 32-wide chunks per macro-block (1, 2, 4)
+template <int WB, int NT, int CPG>
+__global__ void __launch_bounds__(kStreamThreads) gemv_stream_kernel(const StreamParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    // carve-up: [ring stages][lut][red: 2 x 8 warps x 32 lanes x NT*4 floats][barriers]
+    const int stage_bytes = kStageUnits * p.unit_bytes;
+    unsigned char* ring = smem;
+    unsigned char* lut = ring + (size_t)p.n_stages * stage_bytes;
+    float* red = reinterpret_cast<float*>(lut + kLutBytes);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(red + 2 * kConsumerWarps * 32 * NT * 4);
+    uint64_t* empty_bar = full_bar + p.n_stages;
+    __shared__ int abort_flag;
+    __shared__ int last_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_ctas = gridDim.x;
+    const int u_begin = range_begin(blockIdx.x, p.n_units, n_ctas), u_end = range_begin(blockIdx.x + 1, p.n_units, n_ctas);
+    const int my_units = u_end - u_begin;
+    const int my_stages = (my_units + kStageUnits - 1) / kStageUnits;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        last_flag = 0;
+        for (int s = 0; s < p.n_stages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], kConsumerWarps);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i < 64 * kLutCopies; i += kStreamThreads) {
+        const uint32_t meta = i / kLutCopies, copy = i % kLutCopies;
+        *reinterpret_cast<uint4*>(lut + record_slot(meta) * (kLutCopies * 16) + copy * 16) = make_exchange_entry(meta);
+    }
+    __syncthreads();
+    // the next kernel in the stream may begin its own prologue and weight prefetch
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    if (warp == kConsumerWarps) {
+        // ---------------- producer: one thread streams this CTA's records through the ring -------------
+        if (lane == 0) {
+            const uint8_t* src = p.packed + (size_t)u_begin * p.unit_bytes;
+            int slot = 0, round = 0;
+            for (int s = 0; s < my_stages; ++s) {
+                if (round > 0) {
+                    if (!mbar_wait_bounded(&empty_bar[slot], (round - 1) & 1, &abort_flag)) break;
+                }
+                const int units = min(kStageUnits, my_units - s * kStageUnits);
+                const uint32_t bytes = (uint32_t)units * p.unit_bytes;
+                mbar_arrive_expect_tx(&full_bar[slot], bytes);
+                bulk_copy_g2s(ring + (size_t)slot * stage_bytes, src + (size_t)s * stage_bytes, bytes, &full_bar[slot]);
+                if (++slot == p.n_stages) { slot = 0; ++round; }
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers ---------------------------------------------------------------------
+    const int g = lane >> 2, t = lane & 3;
+    const unsigned char* lut_lane = lut + (lane & (kLutCopies - 1)) * 16;
+    const int k_blocks = p.k_blocks;
+
+    // everything below reads activations or writes outputs / scratch: wait for the preceding kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // per-lane activation row pointers (token nt*8+g), advanced by k
+    const uint16_t* xrow[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) xrow[nt] = p.x + (size_t)min(nt * 8 + g, p.m_total - 1) * p.k_in + t * 8;
+    bool has_tok[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) has_tok[nt] = (nt * 8 + g) < p.m_total;
+
+    const int tile_first = u_begin / k_blocks, tile_last = (my_units > 0) ? (u_end - 1) / k_blocks : -1;
+    int s = 0, slot = 0, phase = 0;  // stage cursor of this warp (same sequence for every warp)
+    int buf = 0;
+    for (int T = tile_first; T <= tile_last; ++T) {
+        float acc[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) acc[nt][r] = 0.f;
+        const int tile_u0 = T * k_blocks, tile_u1 = tile_u0 + k_blocks;
+
+        for (;;) {
+            const int stage_first = u_begin + s * kStageUnits;
+            if (stage_first >= u_end || stage_first >= tile_u1) break;  // no record of tile T in this stage
+            const int u = stage_first + warp;
+            const bool mine = (u < u_end) && (u >= tile_u0) && (u < tile_u1);
+            // a stage that straddles two tiles is visited once per tile; it is released on the last visit
+            const int stage_last = min(stage_first + kStageUnits, u_end) - 1;
+            const bool final_visit = stage_last < tile_u1;
+            if (mine && mbar_wait_bounded(&full_bar[slot], phase, &abort_flag)) {
+                const unsigned char* unit = ring + (size_t)slot * stage_bytes + (size_t)warp * p.unit_bytes;
+                const int kb0 = (u - tile_u0) * kBlockK;
+                const uint4 wv0 = reinterpret_cast<const uint4*>(unit)[lane];
+                const uint4 wv1 = reinterpret_cast<const uint4*>(unit)[32 + lane];
+                const uint32_t* coefp = reinterpret_cast<const uint32_t*>(unit + kCodeBytesPerUnit);
+                const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
+                float d1[NT][4], d2[NT][4];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) d1[nt][r] = d2[nt][r] = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int k0 = kb0 + c * 32;
+                    uint4 xa[NT];
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        xa[nt] = make_uint4(0, 0, 0, 0);  // lanes without a token feed zeros; the MMA is warp-wide
+                        if (has_tok[nt] && (k0 + t * 8) < p.k_in) xa[nt] = *reinterpret_cast<const uint4*>(xrow[nt] + k0);
+                    }
+                    uint32_t R0[4], Q0[4], R1[4], Q1[4];
+                    expand_word<WB>(w0[c], lut_lane, R0, Q0);
+                    expand_word<WB>(w1[c], lut_lane, R1, Q1);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        mma_bf16(d1[nt], R0[0], R1[0], R0[1], R1[1], xa[nt].x, xa[nt].y);
+                        mma_bf16(d2[nt], Q0[0], Q1[0], Q0[1], Q1[1], xa[nt].x, xa[nt].y);
+                        mma_bf16(d1[nt], R0[2], R1[2], R0[3], R1[3], xa[nt].z, xa[nt].w);
+                        mma_bf16(d2[nt], Q0[2], Q1[2], Q0[3], Q1[3], xa[nt].z, xa[nt].w);
+                    }
+                    if (((c + 1) % CPG) == 0) {
+                        constexpr int kDummy = 0;
+                        (void)kDummy;
+                        const int jj = c / CPG;
+                        const uint32_t cfa = coefp[jj * 16 + g], cfb = coefp[jj * 16 + 8 + g];
+                        const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
+                        const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
+                        const float c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
+                        const float c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            acc[nt][0] += c1a * d1[nt][0] + c2a * d2[nt][0];
+                            acc[nt][1] += c1a * d1[nt][1] + c2a * d2[nt][1];
+                            acc[nt][2] += c1b * d1[nt][2] + c2b * d2[nt][2];
+                            acc[nt][3] += c1b * d1[nt][3] + c2b * d2[nt][3];
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) d1[nt][r] = d2[nt][r] = 0.f;
+                        }
+                    }
+                }
+            }
+            if (!final_visit) break;  // the stage continues into the next tile: finish this tile first
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[slot]);
+            ++s;
+            if (++slot == p.n_stages) { slot = 0; phase ^= 1; }
+        }
+
+        // ---- fixed-order sum of the eight warps' partial results for tile T ----
+        float* rb = red + (size_t)buf * kConsumerWarps * 32 * NT * 4;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) rb[(warp * 32 + lane) * (NT * 4) + nt * 4 + r] = acc[nt][r];
+        consumer_bar_sync();
+        const int seg0 = max(u_begin, tile_u0), seg1 = min(u_end, tile_u1);
+        const bool full_tile = (seg0 == tile_u0) && (seg1 == tile_u1);
+        constexpr int kOut = 32 * NT * 4;  // outputs of one tile: 16 rows x 8*NT tokens (<= 256)
+        float sum = 0.f;
+        if (tid < kOut) {
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) sum += rb[w * 32 * NT * 4 + tid];
+        }
+        const bool aborted = abort_flag != 0;
+        if (full_tile) {
+            if (!aborted && tid < kOut) store_tile_output<NT>(p, T, tid, sum);
+        } else {
+            // park the partial sums; the CTA that arrives last at this tile adds them in CTA order
+            const int slot_id = (T == tile_first) ? 0 : 1;
+            float* mine_p = p.partials + ((size_t)blockIdx.x * 2 + slot_id) * kPartialFloats;
+            if (tid < kOut) __stcg(mine_p + tid, sum);
+            __threadfence();
+            consumer_bar_sync();
+            const int i_lo = owner_of_unit(tile_u0, p.n_units, n_ctas), i_hi = owner_of_unit(tile_u1 - 1, p.n_units, n_ctas);
+            if (tid == 0) {
+                const int old = atomicAdd(&p.counters[T], 1);
+                const int last = (old == (i_hi - i_lo)) ? 1 : 0;
+                if (last) p.counters[T] = 0;  // leave the scratch clean for the next call
+                last_flag = last;
+            }
+            consumer_bar_sync();
+            if (last_flag && !aborted && tid < kOut) {
+                __threadfence();
+                float tot = 0.f;
+                for (int i = i_lo; i <= i_hi; ++i) {
+                    const int first_tile_i = range_begin(i, p.n_units, n_ctas) / k_blocks;
+                    const int sl = (T == first_tile_i) ? 0 : 1;
+                    tot += __ldcg(p.partials + ((size_t)i * 2 + sl) * kPartialFloats + tid);
+                }
+                store_tile_output<NT>(p, T, tid, tot);
+            }
+            consumer_bar_sync();  // last_flag is reused by the next split tile
+        }
+        buf ^= 1;
+    }
+    if (tid == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
+}
+
+bool gemv_stream_supported(const Geometry& g) { return g.group >= 32 && g.wbits <= 3; }
+
+size_t gemv_stream_workspace(const Geometry& g) { return stream_ws_layout(g).total; }
+
+bool stream_hash_is_bijective() {
+    bool seen[64] = {};
+    for (uint32_t meta = 0; meta < 64; ++meta) {
+        uint32_t s = record_slot(meta);
+        if (seen[s]) return false;
+        seen[s] = true;
+    }
+    return true;
+}
+
+static int sm_count() {
+    static int cached[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (cached[dev] == 0) {
+        int n = 0;
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        cached[dev] = n > 0 ? n : 148;
+    }
+    return cached[dev];
+}
+
+template <int WB, int NT, int CPG>
+static cudaError_t launch_stream(const Geometry& g, const StreamParams& p0, cudaStream_t st) {
+    StreamParams p = p0;
+    constexpr int kCtasPerSm = 2;
+    int grid = sm_count() * kCtasPerSm;
+    if (grid > kMaxCtas) grid = kMaxCtas;
+    if (grid > p.n_units) grid = p.n_units;
+    // ring depth: what fits in ~70 KB, at most what one CTA will ever use
+    const int stage_bytes = kStageUnits * g.unit_bytes;
+    int n_stages = (70 * 1024) / stage_bytes;
+    const int need = (p.n_units / grid + 1 + kStageUnits - 1) / kStageUnits + 1;
+    if (n_stages > need) n_stages = need;
+    if (n_stages < 2) n_stages = 2;
+    p.n_stages = n_stages;
+    const size_t smem = (size_t)n_stages * stage_bytes + kLutBytes +
+                        (size_t)2 * kConsumerWarps * 32 * NT * 4 * sizeof(float) + (size_t)2 * n_stages * sizeof(uint64_t);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<WB, NT, CPG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             160 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kStreamThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<WB, NT, CPG>, p);
+}
+
+template <int WB, int NT>
+static cudaError_t launch_stream_cpg(const Geometry& g, const StreamParams& p, cudaStream_t st) {
+    switch (g.group) {
+        case 32: return launch_stream<WB, NT, 1>(g, p, st);
+        case 64: return launch_stream<WB, NT, 2>(g, p, st);
+        default: return launch_stream<WB, NT, 4>(g, p, st);
+    }
+}
+
+cudaError_t launch_gemv_stream(const Geometry& g, const void* packed, const void* x, int m, void* y, int y_dtype,
+                               void* ws, cudaStream_t st) {
+    const StreamWs L = stream_ws_layout(g);
+    auto* wsb = (uint8_t*)ws;
+    StreamParams p;
+    p.packed = (const uint8_t*)packed;
+    p.x = (const uint16_t*)x;
+    p.y = y;
+    p.status = (int*)wsb;
+    p.counters = (int*)(wsb + L.counters_off);
+    p.partials = (float*)(wsb + L.partials_off);
+    p.n_units = (int)g.n_units;
+    p.unit_bytes = g.unit_bytes;
+    p.k_blocks = g.k_blocks;
+    p.k_in = g.k_in;
+    p.n_out = g.n_out;
+    p.m_total = m;
+    p.y_dtype = y_dtype;
+    p.n_stages = 0;
+    if (g.wbits == 3) return m <= 8 ? launch_stream_cpg<3, 1>(g, p, st) : launch_stream_cpg<3, 2>(g, p, st);
+    return m <= 8 ? launch_stream_cpg<2, 1>(g, p, st) : launch_stream_cpg<2, 2>(g, p, st);
+}
+
+}  // namespace goq

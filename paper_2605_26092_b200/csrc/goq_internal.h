@@ -18,6 +18,14 @@ cudaError_t launch_linear_mma(const Geometry& g, const void* packed, const void*
                               int y_dtype, cudaStream_t st);
 bool linear_mma_supported(const Geometry& g);
 
+// Decode GEMV, streaming kernel (group >= 32, wbits <= 3, m <= 16). `ws` holds gemv_stream_workspace(g)
+// bytes whose tile counters are zero on entry (goq_workspace_init) and are left zero on return.
+bool gemv_stream_supported(const Geometry& g);
+size_t gemv_stream_workspace(const Geometry& g);
+bool stream_hash_is_bijective();
+cudaError_t launch_gemv_stream(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y, int y_dtype,
+                               void* ws, cudaStream_t st);
+
 // Integer-activation layer.
 cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* x, int m, const float* sx,
                            const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, cudaStream_t st);

@@ -8,8 +8,8 @@
 namespace goq {
 
 __global__ void pack_words_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ meta,
-                                  uint32_t* __restrict__ words, uint8_t* __restrict__ meta_plane,
-                                  int n_out, int k_in, int n_pad, int k_pad, int wbits) {
+                                  uint8_t* __restrict__ packed, int n_out, int k_in, int n_pad, int k_pad,
+                                  int wbits, int unit_bytes, int meta_off) {
     const int mbs = k_pad / 8;
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)n_pad * mbs) return;
@@ -25,17 +25,18 @@ __global__ void pack_words_kernel(const uint8_t* __restrict__ codes, const uint8
 #pragma unroll
         for (int i = 0; i < 8; ++i) w |= zero_code << (4 * i);
     }
-    size_t wi = word_index(row, mb, k_pad / kBlockK);
+    uint8_t* unit = packed + unit_offset(row >> 4, mb >> 4, k_pad / kBlockK, unit_bytes);
+    const int wi = word_in_unit(row, mb);
     if (wbits <= 3) {
         w |= scatter_meta(m);
     } else {
-        meta_plane[wi] = (uint8_t)m;
+        unit[meta_off + wi] = (uint8_t)m;
     }
-    words[wi] = w;
+    reinterpret_cast<uint32_t*>(unit)[wi] = w;
 }
 
-__global__ void pack_coef_kernel(const uint16_t* __restrict__ coef, uint32_t* __restrict__ plane, int n_out,
-                                 int n_pad, int groups_in, int groups_pad) {
+__global__ void pack_coef_kernel(const uint16_t* __restrict__ coef, uint8_t* __restrict__ packed, int n_out,
+                                 int n_pad, int groups_in, int groups_pad, int gpb, int k_blocks, int unit_bytes) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)n_pad * groups_pad) return;
     int row = (int)(idx / groups_pad), j = (int)(idx % groups_pad);
@@ -44,19 +45,21 @@ __global__ void pack_coef_kernel(const uint16_t* __restrict__ coef, uint32_t* __
         const uint16_t* c = coef + ((size_t)row * groups_in + j) * 2;
         v = (uint32_t)c[0] | ((uint32_t)c[1] << 16);
     }
-    plane[coef_index(row, j, groups_pad)] = v;
+    uint8_t* unit = packed + unit_offset(row >> 4, j / gpb, k_blocks, unit_bytes);
+    reinterpret_cast<uint32_t*>(unit + kCodeBytesPerUnit)[(j % gpb) * 16 + (row & 15)] = v;
 }
 
-__global__ void unpack_kernel(const uint32_t* __restrict__ words, const uint8_t* __restrict__ meta_plane,
-                              uint8_t* __restrict__ codes_b1, uint8_t* __restrict__ codes_b2, int n_out, int k_in,
-                              int k_pad, int wbits) {
+__global__ void unpack_kernel(const uint8_t* __restrict__ packed, uint8_t* __restrict__ codes_b1,
+                              uint8_t* __restrict__ codes_b2, int n_out, int k_in, int k_pad, int wbits,
+                              int unit_bytes, int meta_off) {
     const int mbs = k_in / 8;
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)n_out * mbs) return;
     int row = (int)(idx / mbs), mb = (int)(idx % mbs);
-    size_t wi = word_index(row, mb, k_pad / kBlockK);
-    uint32_t w = words[wi];
-    uint32_t m = (wbits <= 3) ? gather_meta(w) : (uint32_t)meta_plane[wi];
+    const uint8_t* unit = packed + unit_offset(row >> 4, mb >> 4, k_pad / kBlockK, unit_bytes);
+    const int wi = word_in_unit(row, mb);
+    uint32_t w = reinterpret_cast<const uint32_t*>(unit)[wi];
+    uint32_t m = (wbits <= 3) ? gather_meta(w) : (uint32_t)unit[meta_off + wi];
     const uint32_t cmask = (wbits <= 3) ? 0x77777777u : 0xFFFFFFFFu;
     uint32_t cw = w & cmask;
     const uint32_t emax = (1u << (wbits - 1)) - 1u;
@@ -81,12 +84,13 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ words, const uint8_t*
     }
 }
 
-__global__ void unpack_coef_kernel(const uint32_t* __restrict__ plane, uint16_t* __restrict__ coef, int n_out,
-                                   int groups_in, int groups_pad) {
+__global__ void unpack_coef_kernel(const uint8_t* __restrict__ packed, uint16_t* __restrict__ coef, int n_out,
+                                   int groups_in, int gpb, int k_blocks, int unit_bytes) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)n_out * groups_in) return;
     int row = (int)(idx / groups_in), j = (int)(idx % groups_in);
-    uint32_t v = plane[coef_index(row, j, groups_pad)];
+    const uint8_t* unit = packed + unit_offset(row >> 4, j / gpb, k_blocks, unit_bytes);
+    uint32_t v = reinterpret_cast<const uint32_t*>(unit + kCodeBytesPerUnit)[(j % gpb) * 16 + (row & 15)];
     coef[idx * 2] = (uint16_t)(v & 0xFFFFu);
     coef[idx * 2 + 1] = (uint16_t)(v >> 16);
 }
@@ -94,33 +98,28 @@ __global__ void unpack_coef_kernel(const uint32_t* __restrict__ plane, uint16_t*
 cudaError_t launch_pack(const Geometry& g, const uint8_t* codes, const uint8_t* meta, const uint16_t* coef,
                         void* packed, cudaStream_t st) {
     auto* base = (uint8_t*)packed;
-    auto* words = (uint32_t*)base;
-    auto* coefp = (uint32_t*)(base + g.coef_off_bytes);
-    auto* metap = base + g.meta_off_bytes;
-    size_t nw = g.code_words;
-    pack_words_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(codes, meta, words, metap, g.n_out, g.k_in,
-                                                                   g.n_pad, g.k_pad, g.wbits);
+    size_t nw = (size_t)g.n_pad * (g.k_pad / 8);
+    pack_words_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(codes, meta, base, g.n_out, g.k_in, g.n_pad,
+                                                                   g.k_pad, g.wbits, g.unit_bytes, g.meta_off);
     size_t nc = (size_t)g.n_pad * g.n_groups;
-    pack_coef_kernel<<<(unsigned)((nc + 255) / 256), 256, 0, st>>>(coef, coefp, g.n_out, g.n_pad,
-                                                                  g.k_in / g.group, g.n_groups);
+    pack_coef_kernel<<<(unsigned)((nc + 255) / 256), 256, 0, st>>>(coef, base, g.n_out, g.n_pad, g.k_in / g.group,
+                                                                  g.n_groups, g.groups_per_block, g.k_blocks,
+                                                                  g.unit_bytes);
     return cudaGetLastError();
 }
 
 cudaError_t launch_unpack(const Geometry& g, const void* packed, uint8_t* b1, uint8_t* b2, uint16_t* coef,
                           cudaStream_t st) {
     auto* base = (const uint8_t*)packed;
-    auto* words = (const uint32_t*)base;
-    auto* coefp = (const uint32_t*)(base + g.coef_off_bytes);
-    auto* metap = base + g.meta_off_bytes;
     if (b1 || b2) {
         size_t n = (size_t)g.n_out * (g.k_in / 8);
-        unpack_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(words, metap, b1, b2, g.n_out, g.k_in, g.k_pad,
-                                                                  g.wbits);
+        unpack_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(base, b1, b2, g.n_out, g.k_in, g.k_pad, g.wbits,
+                                                                  g.unit_bytes, g.meta_off);
     }
     if (coef) {
         size_t n = (size_t)g.n_out * (g.k_in / g.group);
-        unpack_coef_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(coefp, coef, g.n_out, g.k_in / g.group,
-                                                                       g.n_groups);
+        unpack_coef_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(base, coef, g.n_out, g.k_in / g.group,
+                                                                       g.groups_per_block, g.k_blocks, g.unit_bytes);
     }
     return cudaGetLastError();
 }

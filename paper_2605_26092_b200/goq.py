@@ -21,7 +21,8 @@ LAYOUT_TILE16 = 1
 
 EXPORTS = (
     "goq_status_string", "goq_packed_bytes", "goq_algorithmic_bytes", "goq_workspace_bytes", "goq_pack",
-    "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant",
+    "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant", "goq_workspace_init",
+    "goq_workspace_status",
 )
 
 
@@ -64,6 +65,10 @@ def lib() -> ctypes.CDLL:
         L.goq_gemv_host.restype = c_int
         L.goq_gemv_host.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p,
                                     c_void_p, c_size_t, c_void_p]
+        L.goq_workspace_init.restype = c_int
+        L.goq_workspace_init.argtypes = [c_void_p, c_size_t, c_void_p]
+        L.goq_workspace_status.restype = c_int
+        L.goq_workspace_status.argtypes = [c_void_p, c_void_p, POINTER(c_int)]
         L.goq_set_gemv_variant.restype = c_int
         L.goq_set_gemv_variant.argtypes = [c_int]
         _lib = L
@@ -104,6 +109,27 @@ def algorithmic_bytes(d: Desc) -> int:
 
 def workspace_bytes(d: Desc, op: int, m: int) -> int:
     return lib().goq_workspace_bytes(ctypes.byref(d), op, m)
+
+
+def workspace_init(ws, stream=None):
+    _check(lib().goq_workspace_init(_ptr(ws), ws.numel() * ws.element_size(), _stream(stream)), "goq_workspace_init")
+
+
+def workspace_status(ws, stream=None) -> int:
+    out = c_int(0)
+    _check(lib().goq_workspace_status(_ptr(ws), _stream(stream), ctypes.byref(out)), "goq_workspace_status")
+    return out.value
+
+
+def new_workspace(d: Desc, op: int, m: int):
+    """Allocate (torch) and initialise a scratch buffer large enough for the call; None if none is needed."""
+    import torch
+    n = workspace_bytes(d, op, m)
+    if n == 0:
+        return None
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+    workspace_init(ws)
+    return ws
 
 
 def set_gemv_variant(variant: int) -> int:

@@ -28,9 +28,10 @@ def run_gemv(d, packed, x_bits: np.ndarray, y_dtype=goq.F32, variant=0):
     batch = x_bits.shape[0]
     x = dev(x_bits)
     y = torch.empty((batch, d.n_out), dtype=torch.float32 if y_dtype == goq.F32 else torch.bfloat16, device="cuda")
+    ws = goq.new_workspace(d, goq.OP_GEMV, batch)
     prev = goq.set_gemv_variant(variant)
     try:
-        goq.gemv(d, packed, x, batch, y, y_dtype)
+        goq.gemv(d, packed, x, batch, y, y_dtype, ws=ws)
     finally:
         goq.set_gemv_variant(prev)
     torch.cuda.synchronize()

@@ -76,7 +76,7 @@ def _quantized(n, k, g, b, seed, outliers=False):
     return O.quantize_geo(w, g, b)
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 @pytest.mark.parametrize("batch", [1, 8])
 def test_config1_single_layer_256(goq, variant, batch):
     """K = N = 256, W3, group 64, fp16 coefficients, bf16 activations, batch 1 and 8, seed 0."""
@@ -97,6 +97,8 @@ def test_config1_single_layer_256(goq, variant, batch):
     (40, 192, 64, 3, 3, 1), (40, 192, 64, 3, 3, 2), (17, 384, 128, 3, 16, 2), (17, 384, 128, 3, 16, 1),
     (33, 256, 32, 2, 5, 2), (33, 256, 32, 2, 5, 1), (24, 128, 16, 4, 2, 1), (16, 128, 8, 3, 1, 1),
     (48, 256, 64, 4, 9, 2), (48, 256, 64, 4, 9, 1), (16, 128, 128, 3, 1, 2), (300, 1152, 128, 3, 12, 2),
+    (40, 192, 64, 3, 3, 3), (17, 384, 128, 3, 16, 3), (33, 256, 32, 2, 5, 3), (16, 128, 128, 3, 1, 3),
+    (300, 1152, 128, 3, 12, 3), (64, 512, 32, 3, 7, 3),
 ])
 def test_gemv_ragged_shapes_bit_widths_and_groups(goq, n, k, g, b, batch, variant):
     from tests.gpu_util import pack_weights, run_gemv
@@ -117,7 +119,9 @@ def test_two_kernel_variants_agree_closely_and_runs_are_deterministic(goq):
     y1 = run_gemv(d, packed, xb, goq.F32, 1)
     y2 = run_gemv(d, packed, xb, goq.F32, 2)
     assert O.normwise_rel_err(y1, y2) < 1e-5
-    for v in (1, 2):
+    y3 = run_gemv(d, packed, xb, goq.F32, 3)
+    assert O.normwise_rel_err(y3, y2) < 1e-5
+    for v in (1, 2, 3):
         a = run_gemv(d, packed, xb, goq.F32, v)
         b = run_gemv(d, packed, xb, goq.F32, v)
         assert np.array_equal(a, b)
@@ -134,7 +138,7 @@ def test_extreme_activations_keep_exponent_arithmetic_right(goq):
     x[1, ::5] *= 2.0 ** 100
     xb = si.f32_to_bf16_bits(x.astype(np.float32))
     y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 64, 3)
-    for v in (1, 2):
+    for v in (1, 2, 3):
         assert O.normwise_rel_err(run_gemv(d, packed, xb, goq.F32, v), y_ref) <= TIGHT
 
 
@@ -240,6 +244,10 @@ def test_argument_errors_return_status_without_launching(goq):
     xo = torch.zeros(2 * 256 + 8, dtype=torch.bfloat16, device="cuda")[1:]
     assert status(goq.gemv, d, packed, xo, 1, y, goq.F32) == goq.ERR_ALIGNMENT
     assert status(goq.gemv, d, packed[16:], x, 1, y, goq.F32) == goq.ERR_ALIGNMENT
+    assert goq.workspace_bytes(d, goq.OP_GEMV, 1) > 0
+    assert status(goq.gemv, d, packed, x, 1, y, goq.F32) == goq.ERR_WORKSPACE          # scratch missing
+    tiny = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    assert status(goq.gemv, d, packed, x, 1, y, goq.F32, ws=tiny) == goq.ERR_WORKSPACE  # scratch too small
     small = torch.zeros(64, dtype=torch.uint8, device="cuda")
     z = torch.zeros(32 * 256, dtype=torch.uint8, device="cuda")
     assert status(goq.pack, d, z, z, z, small) == goq.ERR_WORKSPACE
@@ -262,11 +270,12 @@ def test_outputs_do_not_spill_past_their_buffers(goq):
     codes, meta, coef = _quantized(n, k, 64, 3, seed=51)
     d, packed = pack_weights(n, k, 64, 3, codes, meta, coef)
     x = dev(si.bf16_activations(batch, k, seed=52))
-    for variant in (1, 2):
+    ws = goq.new_workspace(d, goq.OP_GEMV, batch)
+    for variant in (1, 2, 3):
         buf = torch.full((batch * n + 64,), 7.5, dtype=torch.float32, device="cuda")
         y = buf[32:32 + batch * n]
         prev = goq.set_gemv_variant(variant)
-        goq.gemv(d, packed, x, batch, y, goq.F32)
+        goq.gemv(d, packed, x, batch, y, goq.F32, ws=ws)
         goq.set_gemv_variant(prev)
         torch.cuda.synchronize()
         h = buf.cpu().numpy()
@@ -283,7 +292,8 @@ def test_host_buffer_entry_point(goq):
     yh = torch.zeros((batch, n), dtype=torch.float32).pin_memory()
     xs = torch.empty((batch, k), dtype=torch.bfloat16, device="cuda")
     ys = torch.empty((batch, n), dtype=torch.float32, device="cuda")
-    goq.gemv_host(d, packed, xh, batch, yh, goq.F32, xs, ys)
+    ws = goq.new_workspace(d, goq.OP_GEMV, batch)
+    goq.gemv_host(d, packed, xh, batch, yh, goq.F32, xs, ys, ws=ws)
     torch.cuda.synchronize()
     y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 64, 3)
     assert O.normwise_rel_err(yh.numpy().astype(np.float64), y_ref) <= TIGHT
