@@ -142,6 +142,29 @@ goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x
                          void* y_host, int y_dtype, void* x_stage, void* y_stage, void* ws,
                          size_t ws_bytes, void* stream);
 
+/* goq_gemv_static - goq_gemv without a scratch argument, for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging convenience of this library, not part of the method.)
+ * Who needs it: code that runs inside a serving engine or plugin host which already owns all device memory
+ * through its own arena; latency-critical decode loops that must not risk the device-wide synchronisation
+ * cudaMalloc/cudaFree imply; plain C callers with no device allocator of their own. The scratch lives in a
+ * fixed array inside the library image (GOQ_STATIC_SCRATCH_BYTES per GPU that loads the library, held until
+ * the process exits); nothing is allocated or freed by this call, by any CUDA call it makes, or through torch.
+ *   Arguments and results exactly as goq_gemv (same kernel, same numerics).
+ *   Limits: the layer's scratch need, goq_workspace_bytes(desc, GOQ_OP_GEMV, batch), must not exceed
+ *   GOQ_STATIC_SCRATCH_BYTES (about 262 000 sixteen-row tiles, i.e. n_out up to ~4 million), otherwise
+ *   GOQ_ERR_WORKSPACE is returned and nothing is launched; configurations goq_gemv serves with its
+ *   scratch-free kernels (group < 32, wbits = 4) return GOQ_ERR_UNSUPPORTED here - use goq_gemv for them.
+ *   First call on each device: looks up the array's device address (once per device, with that device
+ *   current). Make that first call outside any stream capture.
+ *   Sharing: every call on a device uses the same array. The call clears the part that must start at zero
+ *   and the kernel leaves the rest in a state the next call can overwrite, so calls issued one after another
+ *   on one stream are fine. Calls that can overlap on the GPU (different streams, or different host threads
+ *   feeding different streams) race on the array and corrupt each other's results: serialise them or give
+ *   the others their own scratch through goq_gemv. */
+#define GOQ_STATIC_SCRATCH_BYTES (2u * 1024u * 1024u)
+goq_status goq_gemv_static(const goq_desc* desc, const void* packed, const void* x_bf16, int batch, void* y,
+                           int y_dtype, void* stream);
+
 /* Force a kernel variant (benchmarks and tests only): 0 = automatic, 1 = scalar exponent-add
  * kernel, 2 = tensor-core fragment kernel, 3 = streaming tensor-core kernel. Process-wide.
  * Returns the previous value. */

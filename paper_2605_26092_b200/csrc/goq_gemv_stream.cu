@@ -399,6 +399,7 @@ __global__ void __launch_bounds__(kStreamThreads) gemv_stream_kernel(const Strea
 bool gemv_stream_supported(const Geometry& g) { return g.group >= 32 && g.wbits <= 3; }
 
 size_t gemv_stream_workspace(const Geometry& g) { return stream_ws_layout(g).total; }
+size_t gemv_stream_zeroed_prefix(const Geometry& g) { return stream_ws_layout(g).partials_off; }
 
 bool stream_hash_is_bijective() {
     bool seen[64] = {};

@@ -22,6 +22,7 @@ bool linear_mma_supported(const Geometry& g);
 // bytes whose tile counters are zero on entry (goq_workspace_init) and are left zero on return.
 bool gemv_stream_supported(const Geometry& g);
 size_t gemv_stream_workspace(const Geometry& g);
+size_t gemv_stream_zeroed_prefix(const Geometry& g);  // leading bytes of the scratch that must be zero on entry
 bool stream_hash_is_bijective();
 cudaError_t launch_gemv_stream(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y, int y_dtype,
                                void* ws, cudaStream_t st);

@@ -22,7 +22,7 @@ LAYOUT_TILE16 = 1
 EXPORTS = (
     "goq_status_string", "goq_packed_bytes", "goq_algorithmic_bytes", "goq_workspace_bytes", "goq_pack",
     "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant", "goq_workspace_init",
-    "goq_workspace_status",
+    "goq_workspace_status", "goq_gemv_static",
 )
 
 
@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.goq_workspace_init.argtypes = [c_void_p, c_size_t, c_void_p]
         L.goq_workspace_status.restype = c_int
         L.goq_workspace_status.argtypes = [c_void_p, c_void_p, POINTER(c_int)]
+        L.goq_gemv_static.restype = c_int
+        L.goq_gemv_static.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p]
         L.goq_set_gemv_variant.restype = c_int
         L.goq_set_gemv_variant.argtypes = [c_int]
         _lib = L
@@ -150,6 +152,13 @@ def gemv(d: Desc, packed, x_bf16, batch: int, y, y_dtype: int, ws=None, stream=N
     wsb = 0 if ws is None else ws.numel() * ws.element_size()
     _check(lib().goq_gemv(ctypes.byref(d), _ptr(packed), _ptr(x_bf16), batch, _ptr(y), y_dtype, _ptr(ws), wsb,
                           _stream(stream)), "goq_gemv")
+
+
+def gemv_static(d: Desc, packed, x_bf16, batch: int, y, y_dtype: int, stream=None):
+    """goq_gemv_static: the decode GEMV with the library's built-in scratch array (no scratch argument).
+    For callers that cannot allocate device memory; calls that may overlap on the GPU must not share it."""
+    _check(lib().goq_gemv_static(ctypes.byref(d), _ptr(packed), _ptr(x_bf16), batch, _ptr(y), y_dtype,
+                                 _stream(stream)), "goq_gemv_static")
 
 
 def gemm(d: Desc, packed, x, m: int, x_dtype: int, y=None, y_dtype: int = F32, sx=None, cq=None, sc=None,
