@@ -101,7 +101,6 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
                  "l"(src), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
-__device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------------------------
 // weights: code word -> bf16x2 operand registers
@@ -126,18 +125,50 @@ constexpr int kLutBytes = 64 * kLutCopies * 16;
 
 // Lookup entry of one exchange record: byte selectors that route the eight high (or low) bytes of b1
 // to b2's positions 0..3 (x) and 4..7 (y), and the sign flips of those positions (z, w: bit 7 of each byte).
-__device__ inline uint4 make_exchange_entry(uint32_t meta) {
-    const int s = (int)(meta & 3u) + 1;
-    const uint32_t flips = flip_mask(meta);
-    uint32_t sel_a = 0, sel_b = 0, f_a = 0, f_b = 0;
-    for (int i = 0; i < 4; ++i) {
-        sel_a |= (uint32_t)(i ^ s) << (4 * i);
-        sel_b |= (uint32_t)((4 + i) ^ s) << (4 * i);
-        f_a |= ((flips >> i) & 1u) << (8 * i + 7);
-        f_b |= ((flips >> (4 + i)) & 1u) << (8 * i + 7);
-    }
-    return make_uint4(sel_a, sel_b, f_a, f_b);
+// The table is built at compile time, indexed by record_slot(record).
+struct ExchangeLut {
+    uint32_t v[64][4];
+};
+constexpr uint32_t cx_scatter(uint32_t meta) {
+    uint32_t r = 0;
+    for (int i = 0; i < 6; ++i) r |= ((meta >> i) & 1u) << (4 * i + 3);
+    return r;
 }
+constexpr uint32_t cx_flips(uint32_t meta) {
+    // bit i = 1 iff b2 element i has the opposite sign of the b1 element routed to it:
+    // pair (i, j = i^s), i < j, flag f (1 iff eta = -1): y_i = -eta x_j -> f^1 ; y_j = eta x_i -> f
+    const int s = (int)(meta & 3u) + 1;
+    uint32_t flips = 0;
+    int p = 0;
+    for (int i = 0; i < 8; ++i) {
+        const int j = i ^ s;
+        if (i < j) {
+            const uint32_t f = (meta >> (2 + p)) & 1u;
+            flips |= (f ^ 1u) << i;
+            flips |= f << j;
+            ++p;
+        }
+    }
+    return flips;
+}
+constexpr ExchangeLut make_exchange_lut() {
+    ExchangeLut t{};
+    for (uint32_t meta = 0; meta < 64; ++meta) {
+        const int s = (int)(meta & 3u) + 1;
+        const uint32_t flips = cx_flips(meta);
+        uint32_t sel_a = 0, sel_b = 0, f_a = 0, f_b = 0;
+        for (int i = 0; i < 4; ++i) {
+            sel_a |= (uint32_t)(i ^ s) << (4 * i);
+            sel_b |= (uint32_t)((4 + i) ^ s) << (4 * i);
+            f_a |= ((flips >> i) & 1u) << (8 * i + 7);
+            f_b |= ((flips >> (4 + i)) & 1u) << (8 * i + 7);
+        }
+        const uint32_t slot = (uint32_t)(cx_scatter(meta) * kHashMul) >> 26;
+        t.v[slot][0] = sel_a; t.v[slot][1] = sel_b; t.v[slot][2] = f_a; t.v[slot][3] = f_b;
+    }
+    return t;
+}
+__constant__ ExchangeLut c_exchange_lut = make_exchange_lut();
 
 // R[q] = bf16x2 (b1 element 2q, 2q+1); Q[q] the same for b2 (Section 3.3: partner i XOR s routed by a
 // byte permute, pair signs XOR-ed into the bf16 sign bit; a flipped zero is -0 and adds nothing).
@@ -164,9 +195,10 @@ __device__ __forceinline__ void expand_word(uint32_t w, const unsigned char* __r
 // ------------------------------------------------------------------------------------------------
 // streaming kernel
 // ------------------------------------------------------------------------------------------------
-constexpr int kConsumerWarps = 8;
+constexpr int kConsumerWarps = 16;
 constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;
 constexpr int kStageUnits = kConsumerWarps;
+__device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory"); }
 
 struct StreamParams {
     const uint8_t* packed;
@@ -185,30 +217,22 @@ __device__ __forceinline__ int range_begin(int i, int n_units, int n_ctas) {
     return (int)((long long)n_units * i / n_ctas);
 }
 
-template <int NT>
-__device__ __forceinline__ void store_tile_output(const StreamParams& p, int T, int o, float v) {
-    const int ln = o / (NT * 4), qq = o % (NT * 4), nt = qq >> 2, r = qq & 3;
-    const int row = T * 16 + (ln >> 2) + ((r & 2) ? 8 : 0);
-    const int tok = nt * 8 + (ln & 3) * 2 + (r & 1);
-    if (row < p.n_out && tok < p.m_total) {
-        if (p.y_dtype == GOQ_F32) reinterpret_cast<float*>(p.y)[(size_t)tok * p.n_out + row] = v;
-        else reinterpret_cast<uint16_t*>(p.y)[(size_t)tok * p.n_out + row] = f32_to_bf16_rne(v);
-    }
-}
+constexpr int kRedSlots = 4;  // ring of per-tile reduction buffers inside a CTA
 
 // WB: weight bits (2, 3); NT: 8-token column tiles (1, 2); CPG: 32-wide chunks per macro-block (1, 2, 4)
 template <int WB, int NT, int CPG>
-__global__ void __launch_bounds__(kStreamThreads) gemv_stream_kernel(const StreamParams p) {
+__global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream_kernel(const StreamParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    // carve-up: [ring stages][lut][red: 2 x 8 warps x 32 lanes x NT*4 floats][barriers]
+    // carve-up: [ring stages][lut][red: kRedSlots x 8 warps x 32 lanes x NT*4 floats][barriers]
     const int stage_bytes = kStageUnits * p.unit_bytes;
     unsigned char* ring = smem;
     unsigned char* lut = ring + (size_t)p.n_stages * stage_bytes;
     float* red = reinterpret_cast<float*>(lut + kLutBytes);
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(red + 2 * kConsumerWarps * 32 * NT * 4);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(red + kRedSlots * kConsumerWarps * 32 * NT * 4);
     uint64_t* empty_bar = full_bar + p.n_stages;
-    __shared__ int abort_flag;
-    __shared__ int last_flag;
+    __shared__ volatile int abort_flag;
+    __shared__ int arrive_cnt[kRedSlots];  // warps that have parked their sums for the tile using the slot
+    __shared__ int done_gen[kRedSlots];    // 1 + local index of the last tile fully reduced out of the slot
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_ctas = gridDim.x;
@@ -218,16 +242,12 @@ __global__ void __launch_bounds__(kStreamThreads) gemv_stream_kernel(const Strea
 
     if (tid == 0) {
         abort_flag = 0;
-        last_flag = 0;
+        for (int i = 0; i < kRedSlots; ++i) { arrive_cnt[i] = 0; done_gen[i] = 0; }
         for (int s = 0; s < p.n_stages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kConsumerWarps);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    for (int i = tid; i < 64 * kLutCopies; i += kStreamThreads) {
-        const uint32_t meta = i / kLutCopies, copy = i % kLutCopies;
-        *reinterpret_cast<uint4*>(lut + record_slot(meta) * (kLutCopies * 16) + copy * 16) = make_exchange_entry(meta);
     }
     __syncthreads();
     // the next kernel in the stream may begin its own prologue and weight prefetch
@@ -253,6 +273,13 @@ __global__ void __launch_bounds__(kStreamThreads) gemv_stream_kernel(const Strea
     }
 
     // ---------------- consumers ---------------------------------------------------------------------
+    // replicate the record table (8 bank-disjoint copies), while the first stages are in flight
+    for (int i = tid; i < 64 * kLutCopies; i += kConsumerWarps * 32) {
+        const uint32_t* e = c_exchange_lut.v[i / kLutCopies];
+        *reinterpret_cast<uint4*>(lut + (size_t)i * 16) = make_uint4(e[0], e[1], e[2], e[3]);
+    }
+    consumer_bar_sync();
+
     const int g = lane >> 2, t = lane & 3;
     const unsigned char* lut_lane = lut + (lane & (kLutCopies - 1)) * 16;
     const int k_blocks = p.k_blocks;
@@ -260,140 +287,185 @@ __global__ void __launch_bounds__(kStreamThreads) gemv_stream_kernel(const Strea
     // everything below reads activations or writes outputs / scratch: wait for the preceding kernel
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // per-lane activation row pointers (token nt*8+g), advanced by k
+    // per-lane activation row pointers (token nt*8+g)
     const uint16_t* xrow[NT];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) xrow[nt] = p.x + (size_t)min(nt * 8 + g, p.m_total - 1) * p.k_in + t * 8;
     bool has_tok[NT];
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) has_tok[nt] = (nt * 8 + g) < p.m_total;
+    for (int nt = 0; nt < NT; ++nt) {
+        xrow[nt] = p.x + (size_t)min(nt * 8 + g, p.m_total - 1) * p.k_in + t * 8;
+        has_tok[nt] = (nt * 8 + g) < p.m_total;
+    }
 
-    const int tile_first = u_begin / k_blocks, tile_last = (my_units > 0) ? (u_end - 1) / k_blocks : -1;
-    int s = 0, slot = 0, phase = 0;  // stage cursor of this warp (same sequence for every warp)
-    int buf = 0;
-    for (int T = tile_first; T <= tile_last; ++T) {
-        float acc[NT][4];
+    // This warp takes records u_begin + warp, + 8, ... (record i of the range sits in stage i / 8).
+    const int tile_first = (my_units > 0) ? u_begin / k_blocks : 0;
+    int slot = 0, phase = 0;
+    int T = -1, tile_u0 = 0, tile_u1 = 0;  // tile of the sums currently held in acc
+    float acc[NT][4];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+    for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int r = 0; r < 4; ++r) acc[nt][r] = 0.f;
-        const int tile_u0 = T * k_blocks, tile_u1 = tile_u0 + k_blocks;
+        for (int r = 0; r < 4; ++r) acc[nt][r] = 0.f;
 
-        for (;;) {
-            const int stage_first = u_begin + s * kStageUnits;
-            if (stage_first >= u_end || stage_first >= tile_u1) break;  // no record of tile T in this stage
-            const int u = stage_first + warp;
-            const bool mine = (u < u_end) && (u >= tile_u0) && (u < tile_u1);
-            // a stage that straddles two tiles is visited once per tile; it is released on the last visit
-            const int stage_last = min(stage_first + kStageUnits, u_end) - 1;
-            const bool final_visit = stage_last < tile_u1;
-            if (mine && mbar_wait_bounded(&full_bar[slot], phase, &abort_flag)) {
-                const unsigned char* unit = ring + (size_t)slot * stage_bytes + (size_t)warp * p.unit_bytes;
-                const int kb0 = (u - tile_u0) * kBlockK;
-                const uint4 wv0 = reinterpret_cast<const uint4*>(unit)[lane];
-                const uint4 wv1 = reinterpret_cast<const uint4*>(unit)[32 + lane];
-                const uint32_t* coefp = reinterpret_cast<const uint32_t*>(unit + kCodeBytesPerUnit);
-                const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
-                float d1[NT][4], d2[NT][4];
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) d1[nt][r] = d2[nt][r] = 0.f;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int k0 = kb0 + c * 32;
-                    uint4 xa[NT];
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        xa[nt] = make_uint4(0, 0, 0, 0);  // lanes without a token feed zeros; the MMA is warp-wide
-                        if (has_tok[nt] && (k0 + t * 8) < p.k_in) xa[nt] = *reinterpret_cast<const uint4*>(xrow[nt] + k0);
+    for (int i = warp;; i += kStageUnits) {
+        const int u = u_begin + i;
+        const bool more = (i < my_units) && (abort_flag == 0);
+        const int Tn = more ? u / k_blocks : -1;
+        if (Tn != T && T >= 0) {
+            {
+                // ---- park this warp's sums for tile T; the last warp to do so finishes the tile ----
+                const int lt = T - tile_first, rs = lt % kRedSlots;
+                const int a = max(u_begin, tile_u0) - u_begin, b = min(u_end, tile_u1) - u_begin;  // range-relative segment
+                const int contributors = min(kConsumerWarps, b - a);
+                bool ok = true;
+                if (lt >= kRedSlots) {  // the slot's previous tile must be fully reduced
+                    volatile int* dg = &done_gen[rs];
+                    int it = 0;
+                    while (*dg != lt - kRedSlots + 1) {
+                        if (abort_flag || ++it > kSpinLimit) { abort_flag = 1; ok = false; break; }
+                        __nanosleep(40);
                     }
-                    uint32_t R0[4], Q0[4], R1[4], Q1[4];
-                    expand_word<WB>(w0[c], lut_lane, R0, Q0);
-                    expand_word<WB>(w1[c], lut_lane, R1, Q1);
+                }
+                if (ok) {
+                    float* rb = red + (size_t)rs * kConsumerWarps * 32 * NT * 4;
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        mma_bf16(d1[nt], R0[0], R1[0], R0[1], R1[1], xa[nt].x, xa[nt].y);
-                        mma_bf16(d2[nt], Q0[0], Q1[0], Q0[1], Q1[1], xa[nt].x, xa[nt].y);
-                        mma_bf16(d1[nt], R0[2], R1[2], R0[3], R1[3], xa[nt].z, xa[nt].w);
-                        mma_bf16(d2[nt], Q0[2], Q1[2], Q0[3], Q1[3], xa[nt].z, xa[nt].w);
-                    }
-                    if (((c + 1) % CPG) == 0) {
-                        constexpr int kDummy = 0;
-                        (void)kDummy;
-                        const int jj = c / CPG;
-                        const uint32_t cfa = coefp[jj * 16 + g], cfb = coefp[jj * 16 + 8 + g];
-                        const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
-                        const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
-                        const float c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
-                        const float c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
+                    for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) {
-                            acc[nt][0] += c1a * d1[nt][0] + c2a * d2[nt][0];
-                            acc[nt][1] += c1a * d1[nt][1] + c2a * d2[nt][1];
-                            acc[nt][2] += c1b * d1[nt][2] + c2b * d2[nt][2];
-                            acc[nt][3] += c1b * d1[nt][3] + c2b * d2[nt][3];
+                        for (int r = 0; r < 4; ++r) rb[(warp * 32 + lane) * (NT * 4) + nt * 4 + r] = acc[nt][r];
+                    __threadfence_block();
+                    __syncwarp();
+                    int old = 0;
+                    if (lane == 0) old = atomicAdd(&arrive_cnt[rs], 1);
+                    old = __shfl_sync(0xFFFFFFFFu, old, 0);
+                    if (old == contributors - 1) {
+                        __threadfence_block();
+                        float out[NT * 4];
 #pragma unroll
-                            for (int r = 0; r < 4; ++r) d1[nt][r] = d2[nt][r] = 0.f;
+                        for (int q = 0; q < NT * 4; ++q) out[q] = 0.f;
+                        for (int w = 0; w < kConsumerWarps; ++w) {
+                            // warp w holds a record of the segment iff some i in [a, b) has i % 8 == w
+                            const int first = a + ((w - a) & (kStageUnits - 1));
+                            if (first < b) {
+#pragma unroll
+                                for (int q = 0; q < NT * 4; ++q) out[q] += rb[(w * 32 + lane) * (NT * 4) + q];
+                            }
+                        }
+                        const bool full_tile = (a + u_begin == tile_u0) && (b + u_begin == tile_u1);
+                        if (!full_tile) {
+                            // park the CTA's sums; the CTA that arrives last at this tile adds them in CTA order
+                            const int slot_id = (T == tile_first) ? 0 : 1;
+                            float* mine_p = p.partials + ((size_t)blockIdx.x * 2 + slot_id) * kPartialFloats;
+#pragma unroll
+                            for (int q = 0; q < NT * 4; ++q) __stcg(mine_p + lane * (NT * 4) + q, out[q]);
+                            __threadfence();
+                            __syncwarp();
+                            const int i_lo = owner_of_unit(tile_u0, p.n_units, n_ctas);
+                            const int i_hi = owner_of_unit(tile_u1 - 1, p.n_units, n_ctas);
+                            int prev = 0;
+                            if (lane == 0) prev = atomicAdd(&p.counters[T], 1);
+                            prev = __shfl_sync(0xFFFFFFFFu, prev, 0);
+                            if (prev == i_hi - i_lo) {
+                                __threadfence();
+#pragma unroll
+                                for (int q = 0; q < NT * 4; ++q) out[q] = 0.f;
+                                for (int c = i_lo; c <= i_hi; ++c) {
+                                    const int first_tile_c = range_begin(c, p.n_units, n_ctas) / k_blocks;
+                                    const float* pp = p.partials + ((size_t)c * 2 + ((T == first_tile_c) ? 0 : 1)) * kPartialFloats;
+#pragma unroll
+                                    for (int q = 0; q < NT * 4; ++q) out[q] += __ldcg(pp + lane * (NT * 4) + q);
+                                }
+                                if (lane == 0) p.counters[T] = 0;  // leave the scratch clean for the next call
+                            } else {
+                                T = -2;  // not the last CTA: nothing to store
+                            }
+                        }
+                        if (T >= 0 && abort_flag == 0) {
+#pragma unroll
+                            for (int q = 0; q < NT * 4; ++q) {
+                                const int nt = q >> 2, r = q & 3;
+                                const int row = T * 16 + g + ((r & 2) ? 8 : 0);
+                                const int tok = nt * 8 + t * 2 + (r & 1);
+                                if (row < p.n_out && tok < p.m_total) {
+                                    if (p.y_dtype == GOQ_F32) reinterpret_cast<float*>(p.y)[(size_t)tok * p.n_out + row] = out[q];
+                                    else reinterpret_cast<uint16_t*>(p.y)[(size_t)tok * p.n_out + row] = f32_to_bf16_rne(out[q]);
+                                }
+                            }
+                        }
+                        __syncwarp();
+                        if (lane == 0) {
+                            arrive_cnt[rs] = 0;
+                            __threadfence_block();
+                            done_gen[rs] = lt + 1;
                         }
                     }
                 }
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) acc[nt][r] = 0.f;
             }
-            if (!final_visit) break;  // the stage continues into the next tile: finish this tile first
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[slot]);
-            ++s;
-            if (++slot == p.n_stages) { slot = 0; phase ^= 1; }
+        }
+        if (!more) break;  // every path out of the loop: i only grows, so this is reached
+        if (Tn != T) {
+            T = Tn;
+            tile_u0 = T * k_blocks;
+            tile_u1 = tile_u0 + k_blocks;
         }
 
-        // ---- fixed-order sum of the eight warps' partial results for tile T ----
-        float* rb = red + (size_t)buf * kConsumerWarps * 32 * NT * 4;
+        if (mbar_wait_bounded(&full_bar[slot], phase, &abort_flag)) {
+            const unsigned char* unit = ring + (size_t)slot * stage_bytes + (size_t)warp * p.unit_bytes;
+            const int kb0 = (u - tile_u0) * kBlockK;
+            const uint4 wv0 = reinterpret_cast<const uint4*>(unit)[lane];
+            const uint4 wv1 = reinterpret_cast<const uint4*>(unit)[32 + lane];
+            const uint32_t* coefp = reinterpret_cast<const uint32_t*>(unit + kCodeBytesPerUnit);
+            const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
+            float d1[NT][4], d2[NT][4];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int r = 0; r < 4; ++r) rb[(warp * 32 + lane) * (NT * 4) + nt * 4 + r] = acc[nt][r];
-        consumer_bar_sync();
-        const int seg0 = max(u_begin, tile_u0), seg1 = min(u_end, tile_u1);
-        const bool full_tile = (seg0 == tile_u0) && (seg1 == tile_u1);
-        constexpr int kOut = 32 * NT * 4;  // outputs of one tile: 16 rows x 8*NT tokens (<= 256)
-        float sum = 0.f;
-        if (tid < kOut) {
+                for (int r = 0; r < 4; ++r) d1[nt][r] = d2[nt][r] = 0.f;
 #pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) sum += rb[w * 32 * NT * 4 + tid];
-        }
-        const bool aborted = abort_flag != 0;
-        if (full_tile) {
-            if (!aborted && tid < kOut) store_tile_output<NT>(p, T, tid, sum);
-        } else {
-            // park the partial sums; the CTA that arrives last at this tile adds them in CTA order
-            const int slot_id = (T == tile_first) ? 0 : 1;
-            float* mine_p = p.partials + ((size_t)blockIdx.x * 2 + slot_id) * kPartialFloats;
-            if (tid < kOut) __stcg(mine_p + tid, sum);
-            __threadfence();
-            consumer_bar_sync();
-            const int i_lo = owner_of_unit(tile_u0, p.n_units, n_ctas), i_hi = owner_of_unit(tile_u1 - 1, p.n_units, n_ctas);
-            if (tid == 0) {
-                const int old = atomicAdd(&p.counters[T], 1);
-                const int last = (old == (i_hi - i_lo)) ? 1 : 0;
-                if (last) p.counters[T] = 0;  // leave the scratch clean for the next call
-                last_flag = last;
-            }
-            consumer_bar_sync();
-            if (last_flag && !aborted && tid < kOut) {
-                __threadfence();
-                float tot = 0.f;
-                for (int i = i_lo; i <= i_hi; ++i) {
-                    const int first_tile_i = range_begin(i, p.n_units, n_ctas) / k_blocks;
-                    const int sl = (T == first_tile_i) ? 0 : 1;
-                    tot += __ldcg(p.partials + ((size_t)i * 2 + sl) * kPartialFloats + tid);
+            for (int c = 0; c < 4; ++c) {
+                const int k0 = kb0 + c * 32;
+                uint4 xa[NT];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    xa[nt] = make_uint4(0, 0, 0, 0);  // lanes without a token feed zeros; the MMA is warp-wide
+                    if (has_tok[nt] && (k0 + t * 8) < p.k_in) xa[nt] = *reinterpret_cast<const uint4*>(xrow[nt] + k0);
                 }
-                store_tile_output<NT>(p, T, tid, tot);
+                uint32_t R0[4], Q0[4], R1[4], Q1[4];
+                expand_word<WB>(w0[c], lut_lane, R0, Q0);
+                expand_word<WB>(w1[c], lut_lane, R1, Q1);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    mma_bf16(d1[nt], R0[0], R1[0], R0[1], R1[1], xa[nt].x, xa[nt].y);
+                    mma_bf16(d2[nt], Q0[0], Q1[0], Q0[1], Q1[1], xa[nt].x, xa[nt].y);
+                    mma_bf16(d1[nt], R0[2], R1[2], R0[3], R1[3], xa[nt].z, xa[nt].w);
+                    mma_bf16(d2[nt], Q0[2], Q1[2], Q0[3], Q1[3], xa[nt].z, xa[nt].w);
+                }
+                if (((c + 1) % CPG) == 0) {
+                    const int jj = c / CPG;
+                    const uint32_t cfa = coefp[jj * 16 + g], cfb = coefp[jj * 16 + 8 + g];
+                    const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
+                    const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
+                    const float c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
+                    const float c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        acc[nt][0] += c1a * d1[nt][0] + c2a * d2[nt][0];
+                        acc[nt][1] += c1a * d1[nt][1] + c2a * d2[nt][1];
+                        acc[nt][2] += c1b * d1[nt][2] + c2b * d2[nt][2];
+                        acc[nt][3] += c1b * d1[nt][3] + c2b * d2[nt][3];
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) d1[nt][r] = d2[nt][r] = 0.f;
+                    }
+                }
             }
-            consumer_bar_sync();  // last_flag is reused by the next split tile
         }
-        buf ^= 1;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[slot]);
+        if (++slot == p.n_stages) { slot = 0; phase ^= 1; }
     }
-    if (tid == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
+    if (lane == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
 }
 
 bool gemv_stream_supported(const Geometry& g) { return g.group >= 32 && g.wbits <= 3; }
@@ -427,7 +499,7 @@ static int sm_count() {
 template <int WB, int NT, int CPG>
 static cudaError_t launch_stream(const Geometry& g, const StreamParams& p0, cudaStream_t st) {
     StreamParams p = p0;
-    constexpr int kCtasPerSm = 2;
+    constexpr int kCtasPerSm = (NT == 1) ? 2 : 1;
     int grid = sm_count() * kCtasPerSm;
     if (grid > kMaxCtas) grid = kMaxCtas;
     if (grid > p.n_units) grid = p.n_units;
@@ -439,7 +511,7 @@ static cudaError_t launch_stream(const Geometry& g, const StreamParams& p0, cuda
     if (n_stages < 2) n_stages = 2;
     p.n_stages = n_stages;
     const size_t smem = (size_t)n_stages * stage_bytes + kLutBytes +
-                        (size_t)2 * kConsumerWarps * 32 * NT * 4 * sizeof(float) + (size_t)2 * n_stages * sizeof(uint64_t);
+                        (size_t)kRedSlots * kConsumerWarps * 32 * NT * 4 * sizeof(float) + (size_t)2 * n_stages * sizeof(uint64_t);
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<WB, NT, CPG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
