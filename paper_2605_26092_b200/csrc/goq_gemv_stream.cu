@@ -93,6 +93,13 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     *abort_flag = 1;
     return false;
 }
+// Device-scope fetch-add that releases this warp's earlier writes (ordered before it by __syncwarp) and
+// acquires the writes of the CTAs that incremented before.
+__device__ __forceinline__ int atomic_add_acq_rel_gpu(int* addr, int v) {
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
+    return old;
+}
 // 1-D bulk async copy global -> shared, completion counted in bytes on an mbarrier.
 // Source, destination and size are multiples of 16 bytes.
 __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -170,11 +177,31 @@ constexpr ExchangeLut make_exchange_lut() {
 }
 __constant__ ExchangeLut c_exchange_lut = make_exchange_lut();
 
+// Shared-memory loads by 32-bit shared-window address. They carry no memory clobber so the compiler may
+// schedule them freely; ordering after a barrier wait comes from the address, which is passed through
+// order_after_wait() once the wait has returned.
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t order_after_wait(uint32_t addr) {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %1;" : "=r"(r) : "r"(addr) : "memory");
+    return r;
+}
+
 // R[q] = bf16x2 (b1 element 2q, 2q+1); Q[q] the same for b2 (Section 3.3: partner i XOR s routed by a
 // byte permute, pair signs XOR-ed into the bf16 sign bit; a flipped zero is -0 and adds nothing).
+// lut_lane: shared address of this lane's copy of the record table; the table is 8 KiB aligned, so the
+// slot offset (bits 7..12) is OR-ed in.
 template <int WB>
-__device__ __forceinline__ void expand_word(uint32_t w, const unsigned char* __restrict__ lut_lane, uint32_t (&R)[4],
-                                            uint32_t (&Q)[4]) {
+__device__ __forceinline__ void expand_word(uint32_t w, uint32_t lut_lane, uint32_t (&R)[4], uint32_t (&Q)[4]) {
     const uint32_t m = w & 0x77777777u, mh = m >> 16;
     const uint32_t ha = prmt_b32(PotBytes<WB>::H0, PotBytes<WB>::H1, m), hb = prmt_b32(PotBytes<WB>::H0, PotBytes<WB>::H1, mh);
     const uint32_t la = prmt_b32(PotBytes<WB>::L0, PotBytes<WB>::L1, m), lb = prmt_b32(PotBytes<WB>::L0, PotBytes<WB>::L1, mh);
@@ -183,7 +210,7 @@ __device__ __forceinline__ void expand_word(uint32_t w, const unsigned char* __r
     R[2] = prmt_b32(lb, hb, 0x5140u);
     R[3] = prmt_b32(lb, hb, 0x7362u);
     const uint32_t h = (w - m) * kHashMul;
-    const uint4 e = *reinterpret_cast<const uint4*>(lut_lane + ((h >> 19) & 0x1F80u));
+    const uint4 e = lds128(((h >> 19) & 0x1F80u) | lut_lane);
     const uint32_t qha = prmt_b32(ha, hb, e.x) ^ e.z, qhb = prmt_b32(ha, hb, e.y) ^ e.w;
     const uint32_t qla = prmt_b32(la, lb, e.x), qlb = prmt_b32(la, lb, e.y);
     Q[0] = prmt_b32(qla, qha, 0x5140u);
@@ -208,6 +235,7 @@ struct StreamParams {
     int* counters;
     float* partials;
     int n_units, unit_bytes, k_blocks, k_in, n_out, m_total, y_dtype, n_stages;
+    int x_smem_bytes;  // > 0: the activations (m_total x k_in bf16) are staged in shared memory once per CTA
 };
 
 __device__ __forceinline__ int owner_of_unit(int u, int n_units, int n_ctas) {
@@ -217,23 +245,35 @@ __device__ __forceinline__ int range_begin(int i, int n_units, int n_ctas) {
     return (int)((long long)n_units * i / n_ctas);
 }
 
-constexpr int kRedSlots = 4;  // ring of per-tile reduction buffers inside a CTA
+#ifdef GOQ_TRACE
+__device__ unsigned long long g_trace[512][17][12];
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define GOQ_TR(slot) do { if ((threadIdx.x & 31) == 0) g_trace[blockIdx.x][threadIdx.x >> 5][slot] = gtime(); } while (0)
+#else
+#define GOQ_TR(slot) do { } while (0)
+#endif
+constexpr int kRedSlots = 2;  // ring of per-tile reduction buffers inside a CTA
 
 // WB: weight bits (2, 3); NT: 8-token column tiles (1, 2); CPG: 32-wide chunks per macro-block (1, 2, 4)
 template <int WB, int NT, int CPG>
 __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream_kernel(const StreamParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    // carve-up: [ring stages][lut][red: kRedSlots x 8 warps x 32 lanes x NT*4 floats][barriers]
+    // carve-up: [ring stages][red: kRedSlots x warps x 32 lanes x NT*4 floats][barriers][activations]
+    // The record table (8 bank-disjoint copies, 8 KiB) sits at the first 8 KiB boundary of the dynamic
+    // shared memory so that a slot offset can be OR-ed into its address; the launch reserves the slack.
+    unsigned char* lut = smem + ((8192u - (smem_u32(smem) & 8191u)) & 8191u);
     const int stage_bytes = kStageUnits * p.unit_bytes;
-    unsigned char* ring = smem;
-    unsigned char* lut = ring + (size_t)p.n_stages * stage_bytes;
-    float* red = reinterpret_cast<float*>(lut + kLutBytes);
+    unsigned char* ring = lut + kLutBytes;
+    float* red = reinterpret_cast<float*>(ring + (size_t)p.n_stages * stage_bytes);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(red + kRedSlots * kConsumerWarps * 32 * NT * 4);
     uint64_t* empty_bar = full_bar + p.n_stages;
+    uint64_t* x_bar = empty_bar + p.n_stages;
+    const uint16_t* xs = reinterpret_cast<const uint16_t*>(x_bar + 2);  // 16-byte aligned: barriers come in pairs
     __shared__ volatile int abort_flag;
     __shared__ int arrive_cnt[kRedSlots];  // warps that have parked their sums for the tile using the slot
     __shared__ int done_gen[kRedSlots];    // 1 + local index of the last tile fully reduced out of the slot
 
+    GOQ_TR(0);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_ctas = gridDim.x;
     const int u_begin = range_begin(blockIdx.x, p.n_units, n_ctas), u_end = range_begin(blockIdx.x + 1, p.n_units, n_ctas);
@@ -247,9 +287,11 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kConsumerWarps);
         }
+        mbar_init(x_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    GOQ_TR(1);
     // the next kernel in the stream may begin its own prologue and weight prefetch
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
@@ -258,7 +300,9 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
         if (lane == 0) {
             const uint8_t* src = p.packed + (size_t)u_begin * p.unit_bytes;
             int slot = 0, round = 0;
+            bool x_issued = (p.x_smem_bytes == 0);
             for (int s = 0; s < my_stages; ++s) {
+
                 if (round > 0) {
                     if (!mbar_wait_bounded(&empty_bar[slot], (round - 1) & 1, &abort_flag)) break;
                 }
@@ -267,7 +311,19 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
                 mbar_arrive_expect_tx(&full_bar[slot], bytes);
                 bulk_copy_g2s(ring + (size_t)slot * stage_bytes, src + (size_t)s * stage_bytes, bytes, &full_bar[slot]);
                 if (++slot == p.n_stages) { slot = 0; ++round; }
+                if (s == 0) GOQ_TR(2);
+                if (!x_issued && (s + 1 == my_stages || s + 1 == p.n_stages)) {
+                    // the ring is primed: now the activations, which the preceding kernel may have produced
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    const uint32_t row_bytes = (uint32_t)p.k_in * 2;
+                    mbar_arrive_expect_tx(x_bar, row_bytes * p.m_total);
+                    for (int r = 0; r < p.m_total; ++r)
+                        bulk_copy_g2s(const_cast<uint16_t*>(xs) + (size_t)r * p.k_blocks * kBlockK, p.x + (size_t)r * p.k_in,
+                                      row_bytes, x_bar);
+                    x_issued = true;
+                }
             }
+            GOQ_TR(3);
         }
         return;
     }
@@ -278,24 +334,42 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
         const uint32_t* e = c_exchange_lut.v[i / kLutCopies];
         *reinterpret_cast<uint4*>(lut + (size_t)i * 16) = make_uint4(e[0], e[1], e[2], e[3]);
     }
+    if (p.x_smem_bytes) {  // zero the padding [k_in, k_pad) of every staged activation row
+        const int kp = p.k_blocks * kBlockK, tail = kp - p.k_in;
+        uint16_t* xw = const_cast<uint16_t*>(xs);
+        for (int i = tid; i < tail * p.m_total; i += kConsumerWarps * 32) xw[(size_t)(i / tail) * kp + p.k_in + (i % tail)] = 0;
+    }
     consumer_bar_sync();
+    GOQ_TR(2);
 
     const int g = lane >> 2, t = lane & 3;
-    const unsigned char* lut_lane = lut + (lane & (kLutCopies - 1)) * 16;
+    const uint32_t lut_lane = smem_u32(lut) + (lane & (kLutCopies - 1)) * 16;
     const int k_blocks = p.k_blocks;
+    const int k_pad = k_blocks * kBlockK;
 
     // everything below reads activations or writes outputs / scratch: wait for the preceding kernel
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    GOQ_TR(3);
+    int tr_n = 0;
 
-    // per-lane activation row pointers (token nt*8+g)
+    // per-lane activation row (token nt*8+g). Lanes whose token does not exist read the last token's
+    // row instead of zeros: an MMA output column depends only on its own B column, and columns of
+    // missing tokens are never stored.
     const uint16_t* xrow[NT];
-    bool has_tok[NT];
+    uint32_t xrow_s[NT];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-        xrow[nt] = p.x + (size_t)min(nt * 8 + g, p.m_total - 1) * p.k_in + t * 8;
-        has_tok[nt] = (nt * 8 + g) < p.m_total;
+        const int row = min(nt * 8 + g, p.m_total - 1);
+        xrow[nt] = p.x + (size_t)row * p.k_in + t * 8;
+        xrow_s[nt] = smem_u32(xs) + (uint32_t)(row * k_pad + t * 8) * 2;
     }
-
+    const bool x_staged = p.x_smem_bytes != 0;
+    const bool k_ragged = (p.k_in & (kBlockK - 1)) != 0;  // the last k-block is partly padding
+    if (x_staged) {
+        mbar_wait_bounded(x_bar, 0, &abort_flag);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) xrow_s[nt] = order_after_wait(xrow_s[nt]);
+    }
     // This warp takes records u_begin + warp, + 8, ... (record i of the range sits in stage i / 8).
     const int tile_first = (my_units > 0) ? u_begin / k_blocks : 0;
     int slot = 0, phase = 0;
@@ -356,15 +430,13 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
                             float* mine_p = p.partials + ((size_t)blockIdx.x * 2 + slot_id) * kPartialFloats;
 #pragma unroll
                             for (int q = 0; q < NT * 4; ++q) __stcg(mine_p + lane * (NT * 4) + q, out[q]);
-                            __threadfence();
                             __syncwarp();
                             const int i_lo = owner_of_unit(tile_u0, p.n_units, n_ctas);
                             const int i_hi = owner_of_unit(tile_u1 - 1, p.n_units, n_ctas);
                             int prev = 0;
-                            if (lane == 0) prev = atomicAdd(&p.counters[T], 1);
+                            if (lane == 0) prev = atomic_add_acq_rel_gpu(&p.counters[T], 1);
                             prev = __shfl_sync(0xFFFFFFFFu, prev, 0);
                             if (prev == i_hi - i_lo) {
-                                __threadfence();
 #pragma unroll
                                 for (int q = 0; q < NT * 4; ++q) out[q] = 0.f;
                                 for (int c = i_lo; c <= i_hi; ++c) {
@@ -412,11 +484,11 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
         }
 
         if (mbar_wait_bounded(&full_bar[slot], phase, &abort_flag)) {
-            const unsigned char* unit = ring + (size_t)slot * stage_bytes + (size_t)warp * p.unit_bytes;
+            if (tr_n < 3) GOQ_TR(4 + 2 * tr_n);
+            const uint32_t unit = order_after_wait(smem_u32(ring) + slot * stage_bytes + warp * p.unit_bytes + lane * 16);
             const int kb0 = (u - tile_u0) * kBlockK;
-            const uint4 wv0 = reinterpret_cast<const uint4*>(unit)[lane];
-            const uint4 wv1 = reinterpret_cast<const uint4*>(unit)[32 + lane];
-            const uint32_t* coefp = reinterpret_cast<const uint32_t*>(unit + kCodeBytesPerUnit);
+            const uint4 wv0 = lds128(unit), wv1 = lds128(unit + 512);
+            const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
             const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
             float d1[NT][4], d2[NT][4];
 #pragma unroll
@@ -429,8 +501,13 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
                 uint4 xa[NT];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                    xa[nt] = make_uint4(0, 0, 0, 0);  // lanes without a token feed zeros; the MMA is warp-wide
-                    if (has_tok[nt] && (k0 + t * 8) < p.k_in) xa[nt] = *reinterpret_cast<const uint4*>(xrow[nt] + k0);
+                    if (x_staged) {
+                        xa[nt] = lds128(xrow_s[nt] + k0 * 2);  // rows are padded with zeros up to k_pad
+                    } else {
+                        // beyond k_in the weights are zero-valued padding: feed zeros
+                        xa[nt] = make_uint4(0, 0, 0, 0);
+                        if (!k_ragged || (k0 + t * 8) < p.k_in) xa[nt] = *reinterpret_cast<const uint4*>(xrow[nt] + k0);
+                    }
                 }
                 uint32_t R0[4], Q0[4], R1[4], Q1[4];
                 expand_word<WB>(w0[c], lut_lane, R0, Q0);
@@ -444,7 +521,7 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
                 }
                 if (((c + 1) % CPG) == 0) {
                     const int jj = c / CPG;
-                    const uint32_t cfa = coefp[jj * 16 + g], cfb = coefp[jj * 16 + 8 + g];
+                    const uint32_t cfa = lds32(coef_addr + jj * 64), cfb = lds32(coef_addr + jj * 64 + 32);
                     const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
                     const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
                     const float c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
@@ -462,9 +539,12 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
             }
         }
         __syncwarp();
+        if (tr_n < 3) GOQ_TR(5 + 2 * tr_n);
+        ++tr_n;
         if (lane == 0) mbar_arrive(&empty_bar[slot]);
         if (++slot == p.n_stages) { slot = 0; phase ^= 1; }
     }
+    GOQ_TR(10);
     if (lane == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
 }
 
@@ -496,6 +576,8 @@ static int sm_count() {
     return cached[dev];
 }
 
+bool g_stream_pdl = true;  // programmatic dependent launch on the streaming kernel
+
 template <int WB, int NT, int CPG>
 static cudaError_t launch_stream(const Geometry& g, const StreamParams& p0, cudaStream_t st) {
     StreamParams p = p0;
@@ -505,13 +587,16 @@ static cudaError_t launch_stream(const Geometry& g, const StreamParams& p0, cuda
     if (grid > p.n_units) grid = p.n_units;
     // ring depth: what fits in ~70 KB, at most what one CTA will ever use
     const int stage_bytes = kStageUnits * g.unit_bytes;
-    int n_stages = (70 * 1024) / stage_bytes;
+    const int x_bytes = p.m_total * g.k_pad * 2;
+    p.x_smem_bytes = (x_bytes <= 40 * 1024) ? x_bytes : 0;
+    int n_stages = ((kCtasPerSm == 2 ? 56 : 100) * 1024) / stage_bytes;
     const int need = (p.n_units / grid + 1 + kStageUnits - 1) / kStageUnits + 1;
     if (n_stages > need) n_stages = need;
     if (n_stages < 2) n_stages = 2;
     p.n_stages = n_stages;
-    const size_t smem = (size_t)n_stages * stage_bytes + kLutBytes +
-                        (size_t)kRedSlots * kConsumerWarps * 32 * NT * 4 * sizeof(float) + (size_t)2 * n_stages * sizeof(uint64_t);
+    const size_t smem = (size_t)2 * kLutBytes + (size_t)n_stages * stage_bytes +
+                        (size_t)kRedSlots * kConsumerWarps * 32 * NT * 4 * sizeof(float) +
+                        (size_t)(2 * n_stages + 2) * sizeof(uint64_t) + (size_t)p.x_smem_bytes;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<WB, NT, CPG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -528,7 +613,7 @@ static cudaError_t launch_stream(const Geometry& g, const StreamParams& p0, cuda
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = g_stream_pdl ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<WB, NT, CPG>, p);
 }
 
@@ -560,6 +645,7 @@ cudaError_t launch_gemv_stream(const Geometry& g, const void* packed, const void
     p.m_total = m;
     p.y_dtype = y_dtype;
     p.n_stages = 0;
+    p.x_smem_bytes = 0;
     if (g.wbits == 3) return m <= 8 ? launch_stream_cpg<3, 1>(g, p, st) : launch_stream_cpg<3, 2>(g, p, st);
     return m <= 8 ? launch_stream_cpg<2, 1>(g, p, st) : launch_stream_cpg<2, 2>(g, p, st);
 }
