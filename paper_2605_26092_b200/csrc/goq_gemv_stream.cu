@@ -84,11 +84,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // thread has already given up.
 constexpr int kSpinLimit = 1 << 22;
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
+    // try_wait itself suspends the thread for a hardware-defined interval before it reports failure
     for (int it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (it > 32) __nanosleep(40);
+        if ((it & 63) == 63 && *abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
@@ -255,7 +254,8 @@ __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; as
 constexpr int kRedSlots = 2;  // ring of per-tile reduction buffers inside a CTA
 
 // WB: weight bits (2, 3); NT: 8-token column tiles (1, 2); CPG: 32-wide chunks per macro-block (1, 2, 4)
-template <int WB, int NT, int CPG>
+// XS: activations staged in shared memory (small batches) or read from global memory
+template <int WB, int NT, int CPG, bool XS>
 __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream_kernel(const StreamParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     // carve-up: [ring stages][red: kRedSlots x warps x 32 lanes x NT*4 floats][barriers][activations]
@@ -363,7 +363,7 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
         xrow[nt] = p.x + (size_t)row * p.k_in + t * 8;
         xrow_s[nt] = smem_u32(xs) + (uint32_t)(row * k_pad + t * 8) * 2;
     }
-    const bool x_staged = p.x_smem_bytes != 0;
+    constexpr bool x_staged = XS;
     const bool k_ragged = (p.k_in & (kBlockK - 1)) != 0;  // the last k-block is partly padding
     if (x_staged) {
         mbar_wait_bounded(x_bar, 0, &abort_flag);
@@ -501,7 +501,7 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
                 uint4 xa[NT];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                    if (x_staged) {
+                    if constexpr (XS) {
                         xa[nt] = lds128(xrow_s[nt] + k0 * 2);  // rows are padded with zeros up to k_pad
                     } else {
                         // beyond k_in the weights are zero-valued padding: feed zeros
@@ -597,12 +597,12 @@ static cudaError_t launch_stream(const Geometry& g, const StreamParams& p0, cuda
     const size_t smem = (size_t)2 * kLutBytes + (size_t)n_stages * stage_bytes +
                         (size_t)kRedSlots * kConsumerWarps * 32 * NT * 4 * sizeof(float) +
                         (size_t)(2 * n_stages + 2) * sizeof(uint64_t) + (size_t)p.x_smem_bytes;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_stream_kernel<WB, NT, CPG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             160 * 1024);
+    auto kernel = p.x_smem_bytes ? gemv_stream_kernel<WB, NT, CPG, true> : gemv_stream_kernel<WB, NT, CPG, false>;
+    static bool attr_set[2] = {false, false};
+    if (!attr_set[p.x_smem_bytes ? 1 : 0]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[p.x_smem_bytes ? 1 : 0] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -614,7 +614,7 @@ static cudaError_t launch_stream(const Geometry& g, const StreamParams& p0, cuda
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g_stream_pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, gemv_stream_kernel<WB, NT, CPG>, p);
+    return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
 template <int WB, int NT>
