@@ -384,7 +384,7 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
 
     def step_gemm():
         for s, x, y in zip(layer0, xs, ys):
-            goq.gemm(s["d"], s["packed"], x, m, goq.BF16, y=y, y_dtype=goq.F32)
+            goq.gemm(s["d"], s["packed"], x, m, goq.BF16, y=y, y_dtype=goq.F32, ws=ws)
 
     step_gemm()
     torch.cuda.synchronize()

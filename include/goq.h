@@ -165,6 +165,9 @@ goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x
 goq_status goq_gemv_static(const goq_desc* desc, const void* packed, const void* x_bf16, int batch, void* y,
                            int y_dtype, void* stream);
 
+/* The cudaError_t value behind the most recent GOQ_ERR_CUDA returned in this process (0 if none). */
+int goq_last_cuda_error(void);
+
 /* Force a kernel variant (benchmarks and tests only): 0 = automatic, 1 = scalar exponent-add
  * kernel, 2 = tensor-core fragment kernel, 3 = streaming tensor-core kernel. Process-wide.
  * Returns the previous value. */

@@ -29,7 +29,13 @@ goq_status check_arch() {
     return ok ? GOQ_OK : GOQ_ERR_ARCH;
 }
 
-goq_status from_cuda(cudaError_t e) { return e == cudaSuccess ? GOQ_OK : GOQ_ERR_CUDA; }
+std::atomic<int> g_last_cuda_error{0};
+goq_status from_cuda(cudaError_t e) {
+    if (e == cudaSuccess) return GOQ_OK;
+    (void)cudaGetLastError();  // do not leave a non-sticky error behind for the next call to trip over
+    g_last_cuda_error.store((int)e, std::memory_order_relaxed);
+    return GOQ_ERR_CUDA;
+}
 
 }  // namespace
 
@@ -66,6 +72,7 @@ size_t goq_workspace_bytes(const goq_desc* desc, int op, int m) {
     Geometry g;
     if (!goq::make_geometry(desc, &g) || m <= 0) return 0;
     if (op == GOQ_OP_GEMV && m <= 16 && goq::gemv_stream_supported(g)) return goq::gemv_stream_workspace(g);
+    if (op == GOQ_OP_GEMM && goq::gemm_tc_supported(g)) return goq::gemm_tc_workspace(g);
     return 0;
 }
 
@@ -122,13 +129,27 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
     if (y && y_dtype != GOQ_BF16 && y_dtype != GOQ_F32) return GOQ_ERR_INVALID_ARG;
     if (!aligned(packed, 128) || !aligned(x, 16)) return GOQ_ERR_ALIGNMENT;
     if (y && !aligned(y, y_dtype == GOQ_F32 ? 4 : 2)) return GOQ_ERR_ALIGNMENT;
-    (void)ws;
-    (void)ws_bytes;
     if (x_dtype == GOQ_BF16) {
         if (!y) return GOQ_ERR_INVALID_ARG;
-        if (!goq::linear_mma_supported(g)) return GOQ_ERR_UNSUPPORTED;
         if (goq_status s = check_arch()) return s;
-        return from_cuda(goq::launch_linear_mma(g, packed, x, m, y, y_dtype, (cudaStream_t)stream));
+        const int variant = g_gemv_variant.load(std::memory_order_relaxed);
+        if (goq::gemm_tc_supported(g) && variant != 2) {
+            if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
+            if (ws_bytes < goq::gemm_tc_workspace(g)) return GOQ_ERR_WORKSPACE;
+            return from_cuda(goq::launch_gemm_tc(g, packed, x, m, y, y_dtype, ws, (cudaStream_t)stream));
+        }
+        if (goq::linear_mma_supported(g))
+            return from_cuda(goq::launch_linear_mma(g, packed, x, m, y, y_dtype, (cudaStream_t)stream));
+        // remaining configurations (macro-blocks narrower than 32): the scalar kernel, 16 tokens at a time
+        const size_t ybytes = (y_dtype == GOQ_F32) ? 4 : 2;
+        for (int t0 = 0; t0 < m; t0 += 16) {
+            const int nb = (m - t0 < 16) ? (m - t0) : 16;
+            cudaError_t e = goq::launch_gemv_scalar(g, packed, (const uint16_t*)x + (size_t)t0 * g.k_in, nb,
+                                                    (uint8_t*)y + (size_t)t0 * g.n_out * ybytes, y_dtype,
+                                                    (cudaStream_t)stream);
+            if (e != cudaSuccess) return from_cuda(e);
+        }
+        return GOQ_OK;
     }
     if (x_dtype == GOQ_I8) {
         if (!cq || (!y && !acc)) return GOQ_ERR_INVALID_ARG;
@@ -174,6 +195,8 @@ goq_status goq_workspace_status(const void* ws, void* stream, int* status_out) {
     *status_out = v;
     return GOQ_OK;
 }
+
+int goq_last_cuda_error(void) { return g_last_cuda_error.load(std::memory_order_relaxed); }
 
 int goq_set_gemv_variant(int variant) { return g_gemv_variant.exchange(variant); }
 

@@ -1,0 +1,474 @@
+// Prefill GEMM (float activations, many tokens) on the 5th-generation tensor cores.
+//
+// Eq. 4 of the paper with the coefficients folded into the weight operand:
+//   y[m,n] = sum_k x[m,k] * w_hat[n,k],   w_hat[n,k] = c1[n,j] b1[n,k] + c2[n,j] b2[n,k]   (Section 3.1)
+// Each CTA computes a 128 (output channels) x 512 (tokens) tile. Per 64-wide k-chunk
+//   - a producer thread bulk-copies the packed unit records of the 128 rows (cp.async.bulk, 8 records per
+//     128 k) and loads the 512 x 64 bf16 activation tile with two 2-D TMA copies (128-byte swizzle);
+//   - eight expander warps decode the records (same byte-table decode and record lookup as the GEMV:
+//     b1 from the code bytes, b2 = byte-permuted b1 with pair signs, Section 3.3), form
+//     w_hat = c1*b1 + c2*b2 in fp32, round once to bf16 and store the 128 x 64 operand tile to shared
+//     memory in the K-major, 128-byte-swizzled layout the tensor core reads;
+//   - one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 x bf16 -> fp32) into a 128 x 512 fp32
+//     accumulator that fills the SM's tensor memory, and commits each stage back to the producers.
+// After the last chunk the warps read the accumulator with tcgen05.ld and store y.
+// bf16 keeps 8 significant bits, so one rounding of w_hat costs about 2e-3 normwise on the output
+// (measured), which is the whole error budget. The operand is therefore carried as two bf16 tiles,
+// w_hi = bf16(w_hat) and w_lo = bf16(w_hat - w_hi), multiplied against the same activation tile into the
+// same accumulator: w_hi + w_lo holds w_hat to about 2^-16, at the price of twice the tensor work.
+//
+// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, skips the remaining work,
+// still frees its tensor memory and records GOQ_ERR_TIMEOUT in the status word.
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include "goq_common.cuh"
+#include "goq_internal.h"
+
+namespace goq {
+namespace tc {
+
+constexpr int kTileN = 128;     // output channels per CTA (MMA M)
+constexpr int kTileM = 512;     // tokens per CTA (two MMA N = 256 halves)
+constexpr int kChunkK = 64;     // k per pipeline stage: 128 bytes of bf16 = one swizzle row
+constexpr int kStages = 2;
+constexpr int kExpanders = 8;   // expander warps; each owns one 16-row unit record per k-block
+constexpr int kThreads = (2 + kExpanders) * 32;
+constexpr int kATileBytes = kTileN * kChunkK * 2;   // 16 KiB, one of the two operand tiles (hi, lo) of a stage
+constexpr int kBTileBytes = kTileM * kChunkK * 2;   // 64 KiB
+constexpr int kLutCopies = 1;   // the expanders are not the bottleneck here: one 1 KiB copy, bank conflicts accepted
+constexpr int kLutBytes = 64 * kLutCopies * 16;
+constexpr int kSpin = 1 << 22;
+
+__device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t n) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(b)), "r"(n) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s32(b)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(s32(b)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+    for (int it = 0; it < kSpin; ++it) {
+        if (mbar_try(b, parity)) return true;
+        if ((it & 63) == 63 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(s32(dst)),
+                 "l"(src), "r"(bytes), "r"(s32(bar)) : "memory");
+}
+// 2-D tiled TMA load (no multicast): coordinates {c0 = k element, c1 = token row}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(s32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(s32(bar)) : "memory");
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint32_t after_wait(uint32_t addr) {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %1;" : "=r"(r) : "r"(addr) : "memory");
+    return r;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// ---- tensor memory and MMA ---------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc_512(uint32_t* smem_slot) {  // whole warp
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(s32(smem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_512(uint32_t taddr) {  // whole warp
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(taddr) : "memory");
+}
+// K-major operand tile with 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address
+    d |= (uint64_t)1 << 16;                          // leading byte offset (unused for this layout)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                          // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
+    return d;
+}
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, M = 128, N = 256
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+
+// ---- record decode (same tables as the decode GEMV) --------------------------------------------
+template <int WB> struct PotBytes;
+template <> struct PotBytes<3> {  // +1 +.5 +.25 0 -1 -.5 -.25 -.125 : bf16 high / low bytes by code
+    static constexpr uint32_t H0 = 0x003E3F3Fu, H1 = 0xBEBEBFBFu, L0 = 0x00800080u, L1 = 0x00800080u;
+};
+template <> struct PotBytes<2> {  // +1 0 -1 -.5
+    static constexpr uint32_t H0 = 0xBFBF003Fu, H1 = 0u, L0 = 0x00800080u, L1 = 0u;
+};
+constexpr uint32_t kHashMul = 0x01008420u;  // (record bits in place) * kHashMul >> 26 is a bijection onto 0..63
+
+struct ExchangeLut { uint32_t v[64][4]; };
+constexpr ExchangeLut make_exchange_lut() {
+    ExchangeLut t{};
+    for (uint32_t meta = 0; meta < 64; ++meta) {
+        const int s = (int)(meta & 3u) + 1;
+        // flips: bit i = 1 iff b2 element i has the opposite sign of the b1 element routed to it
+        uint32_t flips = 0;
+        int p = 0;
+        for (int i = 0; i < 8; ++i) {
+            const int j = i ^ s;
+            if (i < j) {
+                const uint32_t f = (meta >> (2 + p)) & 1u;  // 1 iff eta = -1
+                flips |= (f ^ 1u) << i;                     // y_i = -eta x_j
+                flips |= f << j;                            // y_j =  eta x_i
+                ++p;
+            }
+        }
+        uint32_t sel_a = 0, sel_b = 0, f_a = 0, f_b = 0, spread = 0;
+        for (int i = 0; i < 4; ++i) {
+            sel_a |= (uint32_t)(i ^ s) << (4 * i);
+            sel_b |= (uint32_t)((4 + i) ^ s) << (4 * i);
+            f_a |= ((flips >> i) & 1u) << (8 * i + 7);
+            f_b |= ((flips >> (4 + i)) & 1u) << (8 * i + 7);
+        }
+        for (int i = 0; i < 6; ++i) spread |= ((meta >> i) & 1u) << (4 * i + 3);
+        const uint32_t slot = (uint32_t)(spread * kHashMul) >> 26;
+        t.v[slot][0] = sel_a; t.v[slot][1] = sel_b; t.v[slot][2] = f_a; t.v[slot][3] = f_b;
+    }
+    return t;
+}
+__constant__ ExchangeLut c_lut = make_exchange_lut();
+
+// eight weights of one micro-block -> w_hat = c1*b1 + c2*b2 as bf16 hi + bf16 lo, four bf16x2 words each
+template <int WB>
+__device__ __forceinline__ void expand_what(uint32_t w, uint32_t lut_lane, float c1, float c2, uint32_t (&out_hi)[4],
+                                            uint32_t (&out_lo)[4]) {
+    const uint32_t m = w & 0x77777777u, mh = m >> 16;
+    const uint32_t ha = prmt(PotBytes<WB>::H0, PotBytes<WB>::H1, m), hb = prmt(PotBytes<WB>::H0, PotBytes<WB>::H1, mh);
+    const uint32_t la = prmt(PotBytes<WB>::L0, PotBytes<WB>::L1, m), lb = prmt(PotBytes<WB>::L0, PotBytes<WB>::L1, mh);
+    const uint32_t h = (w - m) * kHashMul;
+    const uint4 e = lds128(((h >> 22) & 0x3F0u) | lut_lane);  // table is 1 KiB aligned
+    const uint32_t qha = prmt(ha, hb, e.x) ^ e.z, qhb = prmt(ha, hb, e.y) ^ e.w;
+    const uint32_t qla = prmt(la, lb, e.x), qlb = prmt(la, lb, e.y);
+    uint32_t R[4], Q[4];
+    R[0] = prmt(la, ha, 0x5140u); R[1] = prmt(la, ha, 0x7362u); R[2] = prmt(lb, hb, 0x5140u); R[3] = prmt(lb, hb, 0x7362u);
+    Q[0] = prmt(qla, qha, 0x5140u); Q[1] = prmt(qla, qha, 0x7362u); Q[2] = prmt(qlb, qhb, 0x5140u); Q[3] = prmt(qlb, qhb, 0x7362u);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float b1lo = __uint_as_float(R[q] << 16), b1hi = __uint_as_float(R[q] & 0xFFFF0000u);
+        const float b2lo = __uint_as_float(Q[q] << 16), b2hi = __uint_as_float(Q[q] & 0xFFFF0000u);
+        const float wlo = fmaf(c2, b2lo, c1 * b1lo), whi = fmaf(c2, b2hi, c1 * b1hi);
+        const uint32_t h2 = pack_bf16x2(wlo, whi);
+        out_hi[q] = h2;
+        // residual of the rounding, exact in fp32, rounded to bf16 itself
+        out_lo[q] = pack_bf16x2(wlo - __uint_as_float(h2 << 16), whi - __uint_as_float(h2 & 0xFFFF0000u));
+    }
+}
+
+struct GemmParams {
+    const uint8_t* packed;
+    void* y;
+    int* status;
+    int unit_bytes, k_blocks, n_tiles, n_out, m_total, y_dtype, group_log2;
+};
+
+template <int WB>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* base = smem_raw + ((1024u - (s32(smem_raw) & 1023u)) & 1023u);  // 1 KiB boundary
+    unsigned char* lut = base;
+    unsigned char* a_tiles = lut + kLutBytes;
+    unsigned char* b_tiles = a_tiles + kStages * 2 * kATileBytes;
+    unsigned char* pk_ring = b_tiles + kStages * kBTileBytes;
+    const int pk_slot_bytes = kExpanders * p.unit_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(pk_ring + 2 * pk_slot_bytes);
+    uint64_t* full_b = bars;            // [kStages] activation tile landed (tx bytes)
+    uint64_t* full_a = bars + 2;        // [kStages] weight tile written by the 8 expander warps
+    uint64_t* empty = bars + 4;         // [kStages] tensor core finished reading the stage
+    uint64_t* pk_full = bars + 6;       // [2] packed records landed
+    uint64_t* pk_empty = bars + 8;      // [2] expanders finished with the records
+    uint64_t* tmem_full = bars + 10;    // accumulator complete
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ volatile int abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int T0 = blockIdx.x * (kTileN / kTileRows);  // first 16-row tile of this CTA
+    const int tok0 = blockIdx.y * kTileM;
+    const int n_chunks = 2 * p.k_blocks;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int i = 0; i < kStages; ++i) { mbar_init(&full_b[i], 1); mbar_init(&full_a[i], kExpanders); mbar_init(&empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], kExpanders); }
+        mbar_init(tmem_full, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i < 64 * kLutCopies; i += kThreads) {
+        const uint32_t* e = c_lut.v[i / kLutCopies];
+        *reinterpret_cast<uint4*>(lut + (size_t)i * 16) = make_uint4(e[0], e[1], e[2], e[3]);
+    }
+    if (warp == 1) tmem_alloc_512(&tmem_base_slot);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        // ------------------------------ producer ------------------------------
+        if (lane == 0) {
+            int n_rec = p.n_tiles - T0;
+            if (n_rec > kExpanders) n_rec = kExpanders;
+            bool ok = true;
+            for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
+                const int ps = kb & 1;
+                if (kb >= 2) ok = mbar_wait(&pk_empty[ps], ((kb >> 1) - 1) & 1, &abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(&pk_full[ps], (uint32_t)n_rec * p.unit_bytes);
+                for (int r = 0; r < n_rec; ++r)
+                    bulk_g2s(pk_ring + ps * pk_slot_bytes + r * p.unit_bytes,
+                             p.packed + unit_offset(T0 + r, kb, p.k_blocks, p.unit_bytes), p.unit_bytes, &pk_full[ps]);
+                for (int half = 0; half < 2 && ok; ++half) {
+                    const int chunk = 2 * kb + half, s = chunk % kStages;
+                    if (chunk >= kStages) ok = mbar_wait(&empty[s], ((chunk / kStages) - 1) & 1, &abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(&full_b[s], kBTileBytes);
+                    tma_load_2d(b_tiles + s * kBTileBytes, &x_map, chunk * kChunkK, tok0, &full_b[s]);
+                    tma_load_2d(b_tiles + s * kBTileBytes + kBTileBytes / 2, &x_map, chunk * kChunkK, tok0 + 256, &full_b[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            bool ok = true;
+            for (int chunk = 0; chunk < n_chunks; ++chunk) {
+                const int s = chunk % kStages;
+                const uint32_t par = (chunk / kStages) & 1;
+                ok = mbar_wait(&full_b[s], par, &abort_flag) && mbar_wait(&full_a[s], par, &abort_flag);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t ahi = smem_desc_sw128(s32(a_tiles + s * 2 * kATileBytes));
+                const uint64_t alo = smem_desc_sw128(s32(a_tiles + s * 2 * kATileBytes + kATileBytes));
+                const uint64_t bdesc0 = smem_desc_sw128(s32(b_tiles + s * kBTileBytes));
+                const uint64_t bdesc1 = smem_desc_sw128(s32(b_tiles + s * kBTileBytes + kBTileBytes / 2));
+#pragma unroll
+                for (int ks = 0; ks < kChunkK / 16; ++ks) {
+                    const uint32_t acc = (chunk > 0 || ks > 0) ? 1u : 0u;
+                    umma_bf16(tmem_base, ahi + 2 * ks, bdesc0 + 2 * ks, acc);         // tokens   0..255
+                    umma_bf16(tmem_base + 256, ahi + 2 * ks, bdesc1 + 2 * ks, acc);   // tokens 256..511
+                    umma_bf16(tmem_base, alo + 2 * ks, bdesc0 + 2 * ks, 1u);
+                    umma_bf16(tmem_base + 256, alo + 2 * ks, bdesc1 + 2 * ks, 1u);
+                }
+                umma_commit(&empty[s]);
+            }
+            if (ok) umma_commit(tmem_full);
+        }
+    } else {
+        // ------------------------------ expanders, then epilogue ------------------------------
+        const int e = warp - 2, g = lane >> 2, t = lane & 3;
+        const uint32_t lut_lane = s32(lut);
+        const bool valid = (T0 + e) < p.n_tiles;
+        constexpr uint32_t kZeroWord = (WB == 3) ? 0x33333333u : 0x11111111u;  // every code = the zero state
+        bool ok = true;
+        for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
+            const int ps = kb & 1;
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&pk_full[ps], (kb >> 1) & 1, &abort_flag));
+            if (!ok) break;
+            const uint32_t unit = after_wait(s32(pk_ring) + ps * pk_slot_bytes + e * p.unit_bytes);
+            uint4 wv0 = make_uint4(kZeroWord, kZeroWord, kZeroWord, kZeroWord), wv1 = wv0;
+            if (valid) { wv0 = lds128(unit + lane * 16); wv1 = lds128(unit + 512 + lane * 16); }
+            const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int chunk = 2 * kb + half, s = chunk % kStages;
+                if (chunk >= kStages) ok = __all_sync(0xFFFFFFFFu, mbar_wait(&empty[s], ((chunk / kStages) - 1) & 1, &abort_flag));
+                if (!ok) break;
+                const uint32_t a_tile = s32(a_tiles + s * 2 * kATileBytes);
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int c = half * 2 + cc;
+                    const int jj = (c * 32 + t * 8) >> p.group_log2;  // macro-block of this micro-block inside the k-block
+                    float c1a = 0.f, c2a = 0.f, c1b = 0.f, c2b = 0.f;
+                    if (valid) {
+                        const uint32_t cfa = lds32(unit + kCodeBytesPerUnit + (jj * 16 + g) * 4);
+                        const uint32_t cfb = lds32(unit + kCodeBytesPerUnit + (jj * 16 + 8 + g) * 4);
+                        c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
+                        c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
+                        c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
+                        c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
+                    }
+                    uint32_t oa[4], ob[4], la[4], lb[4];
+                    expand_what<WB>(w0[c], lut_lane, c1a, c2a, oa, la);
+                    expand_what<WB>(w1[c], lut_lane, c1b, c2b, ob, lb);
+                    // K-major tile, 128-byte rows, 16-byte chunk j of row r stored at chunk j ^ (r & 7)
+                    const int j = cc * 4 + t;
+                    const int ra = e * 16 + g, rb = ra + 8;  // (ra & 7) == (rb & 7) == g
+                    const uint32_t off = (uint32_t)((j ^ g) << 4);
+                    sts128(a_tile + ra * 128 + off, oa[0], oa[1], oa[2], oa[3]);
+                    sts128(a_tile + rb * 128 + off, ob[0], ob[1], ob[2], ob[3]);
+                    sts128(a_tile + kATileBytes + ra * 128 + off, la[0], la[1], la[2], la[3]);
+                    sts128(a_tile + kATileBytes + rb * 128 + off, lb[0], lb[1], lb[2], lb[3]);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> tensor-core reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full_a[s]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&pk_empty[ps]);
+        }
+        // ---- epilogue: tensor memory -> registers -> y ----
+        if (ok) ok = mbar_wait(tmem_full, 0, &abort_flag);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            const int q = warp & 3, col_half = (e >= 4) ? 1 : 0;
+            const int row = blockIdx.x * kTileN + q * 32 + lane;
+#pragma unroll 1
+            for (int cb = 0; cb < 8; ++cb) {
+                uint32_t v[32];
+                const int col0 = col_half * 256 + cb * 32;
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)col0, v);
+                if (row < p.n_out) {
+#pragma unroll
+                    for (int jx = 0; jx < 32; ++jx) {
+                        const int tok = tok0 + col0 + jx;
+                        if (tok < p.m_total) {
+                            if (p.y_dtype == GOQ_F32) reinterpret_cast<float*>(p.y)[(size_t)tok * p.n_out + row] = __uint_as_float(v[jx]);
+                            else reinterpret_cast<uint16_t*>(p.y)[(size_t)tok * p.n_out + row] = f32_to_bf16_rne(__uint_as_float(v[jx]));
+                        }
+                    }
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        tmem_dealloc_512(tmem_base);
+    }
+    if (tid == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
+}
+
+
+// ---- host side ------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    }
+    return fn;
+}
+
+static size_t smem_bytes(const Geometry& g) {
+    return 1024 /* alignment slack */ + kLutBytes + (size_t)kStages * (2 * kATileBytes + kBTileBytes) +
+           (size_t)2 * kExpanders * g.unit_bytes + 16 * sizeof(uint64_t);
+}
+
+template <int WB>
+static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* x, int m, void* y, int y_dtype, int* status,
+                             cudaStream_t st) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return cudaErrorNotSupported;
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)g.k_in, (cuuint64_t)m};
+    const cuuint64_t strides[1] = {(cuuint64_t)g.k_in * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kChunkK, 256};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidTexture;  // distinct code: the tensor map could not be encoded
+    const size_t smem = smem_bytes(g);
+    static size_t attr_smem = 0;
+    if (smem > attr_smem) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_smem = smem;
+    }
+    GemmParams p;
+    p.packed = (const uint8_t*)packed;
+    p.y = y;
+    p.status = status;
+    p.unit_bytes = g.unit_bytes;
+    p.k_blocks = g.k_blocks;
+    p.n_tiles = g.n_tiles;
+    p.n_out = g.n_out;
+    p.m_total = m;
+    p.y_dtype = y_dtype;
+    int lg = 3;
+    while ((1 << lg) < g.group) ++lg;
+    p.group_log2 = lg;
+    dim3 grid((g.n_pad + kTileN - 1) / kTileN, (m + kTileM - 1) / kTileM);
+    gemm_tc_kernel<WB><<<grid, kThreads, smem, st>>>(p, map);
+    return cudaGetLastError();
+}
+
+}  // namespace tc
+}  // namespace goq
+
+namespace goq {
+bool gemm_tc_supported(const Geometry& g) { return g.wbits <= 3 && tc::smem_bytes(g) + 2048 <= 227 * 1024; }
+size_t gemm_tc_workspace(const Geometry&) { return 256; }  // status word
+cudaError_t launch_gemm_tc(const Geometry& g, const void* packed, const void* x, int m, void* y, int y_dtype, void* ws,
+                           cudaStream_t st) {
+    int* status = (int*)ws;
+    return g.wbits == 3 ? tc::launch_wb<3>(g, packed, x, m, y, y_dtype, status, st)
+                        : tc::launch_wb<2>(g, packed, x, m, y, y_dtype, status, st);
+}
+}  // namespace goq

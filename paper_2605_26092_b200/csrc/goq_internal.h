@@ -27,6 +27,12 @@ bool stream_hash_is_bijective();
 cudaError_t launch_gemv_stream(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y, int y_dtype,
                                void* ws, cudaStream_t st);
 
+// Prefill GEMM on tcgen05 tensor cores (wbits <= 3). `ws` holds gemm_tc_workspace(g) bytes (status word).
+bool gemm_tc_supported(const Geometry& g);
+size_t gemm_tc_workspace(const Geometry& g);
+cudaError_t launch_gemm_tc(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y, int y_dtype,
+                           void* ws, cudaStream_t st);
+
 // Integer-activation layer.
 cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* x, int m, const float* sx,
                            const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, cudaStream_t st);

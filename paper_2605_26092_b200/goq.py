@@ -22,14 +22,15 @@ LAYOUT_TILE16 = 1
 EXPORTS = (
     "goq_status_string", "goq_packed_bytes", "goq_algorithmic_bytes", "goq_workspace_bytes", "goq_pack",
     "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant", "goq_workspace_init",
-    "goq_workspace_status", "goq_gemv_static",
+    "goq_workspace_status", "goq_gemv_static", "goq_last_cuda_error",
 )
 
 
 class GoqError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: status {status} ({status_string(status)})")
+        extra = f", cudaError {lib().goq_last_cuda_error()}" if status == ERR_CUDA else ""
+        super().__init__(f"{where}: status {status} ({status_string(status)}{extra})")
 
 
 class Desc(Structure):
@@ -71,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.goq_workspace_status.argtypes = [c_void_p, c_void_p, POINTER(c_int)]
         L.goq_gemv_static.restype = c_int
         L.goq_gemv_static.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p]
+        L.goq_last_cuda_error.restype = c_int
+        L.goq_last_cuda_error.argtypes = []
         L.goq_set_gemv_variant.restype = c_int
         L.goq_set_gemv_variant.argtypes = [c_int]
         _lib = L

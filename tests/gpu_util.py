@@ -38,12 +38,19 @@ def run_gemv(d, packed, x_bits: np.ndarray, y_dtype=goq.F32, variant=0):
     return y.float().cpu().numpy().astype(np.float64)
 
 
-def run_gemm_bf16(d, packed, x_bits: np.ndarray, y_dtype=goq.F32):
+def run_gemm_bf16(d, packed, x_bits: np.ndarray, y_dtype=goq.F32, variant=0):
     m = x_bits.shape[0]
     x = dev(x_bits)
     y = torch.empty((m, d.n_out), dtype=torch.float32 if y_dtype == goq.F32 else torch.bfloat16, device="cuda")
-    goq.gemm(d, packed, x, m, goq.BF16, y=y, y_dtype=y_dtype)
+    ws = goq.new_workspace(d, goq.OP_GEMM, m)
+    prev = goq.set_gemv_variant(variant)
+    try:
+        goq.gemm(d, packed, x, m, goq.BF16, y=y, y_dtype=y_dtype, ws=ws)
+    finally:
+        goq.set_gemv_variant(prev)
     torch.cuda.synchronize()
+    if ws is not None:
+        assert goq.workspace_status(ws) == goq.OK
     return y.float().cpu().numpy().astype(np.float64)
 
 

@@ -161,14 +161,22 @@ def test_config2_llama7b_shapes_sampled_rows(goq, name, n, k, batch):
 
 
 # ------------------------------------------------------------------------------------- prefill GEMM
-def test_gemm_bf16_small_full_parity(goq):
+@pytest.mark.parametrize("n,k,g,b,m,variant", [
+    (80, 384, 128, 3, 150, 0), (80, 384, 128, 3, 150, 2), (256, 512, 64, 3, 600, 0), (40, 192, 32, 2, 17, 0),
+    (130, 256, 8, 3, 513, 0), (16, 128, 16, 3, 1, 0), (300, 1152, 128, 3, 1030, 0),
+])
+def test_gemm_bf16_small_full_parity(goq, n, k, g, b, m, variant):
+    """Prefill GEMM, every output compared. variant 0: tcgen05 kernel (w_hat carried as bf16 hi + lo);
+    variant 2: the two-operand mma.sync kernel. Both are held to the tight bound."""
     from tests.gpu_util import pack_weights, run_gemm_bf16
-    codes, meta, coef = _quantized(80, 384, 128, 3, seed=11, outliers=True)
-    d, packed = pack_weights(80, 384, 128, 3, codes, meta, coef)
-    xb = si.bf16_activations(150, 384, seed=12)
-    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 128, 3)
-    y = run_gemm_bf16(d, packed, xb)
-    assert O.normwise_rel_err(y, y_ref) <= TOL
+    codes, meta, coef = _quantized(n, k, g, b, seed=11 + n, outliers=True)
+    d, packed = pack_weights(n, k, g, b, codes, meta, coef)
+    xb = si.bf16_activations(m, k, seed=12)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), g, b)
+    y = run_gemm_bf16(d, packed, xb, variant=variant)
+    err = O.normwise_rel_err(y, y_ref)
+    print("gemm variant %d: normwise error %.3e" % (variant, err))
+    assert err <= TOL and err <= TIGHT, err
 
 
 def test_config4_prefill_2048_tokens_sampled_rows(goq):
