@@ -398,6 +398,43 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
     flops = sum(2.0 * m * s["n"] * s["k"] for s in layer0)
     out["gemm_m2048_layer_tflops"] = flops / (ms * 1e-3) / 1e12
     out["gemm_m2048_frac_of_bf16_peak"] = out["gemm_m2048_layer_tflops"] / tf_peak
+    del xs, ys
+    # integer path: ViT-B/16-shaped linears, 197 x 64 tokens, W3 group 64, int8 activations and coefficients
+    mt = si.VIT_B16_TOKENS
+    vit = []
+    gen = torch.Generator(device="cuda")
+    for idx, (name, n, k) in enumerate(si.VIT_B16_LINEARS):
+        gen.manual_seed(5000 + idx)
+        d = goq.desc(n, k, 64, WBITS)
+        codes = torch.randint(0, 1 << WBITS, (n, k), dtype=torch.uint8, device="cuda", generator=gen)
+        meta = torch.randint(0, 64, (n, k // 8), dtype=torch.uint8, device="cuda", generator=gen)
+        coef = (torch.randn((n, k // 64, 2), device="cuda", generator=gen) * 0.03).to(torch.float16)
+        packed = torch.empty(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
+        goq.pack(d, codes, meta, coef, packed)
+        vit.append({
+            "d": d, "packed": packed, "n": n, "k": k,
+            "x": torch.randint(-127, 128, (mt, k), dtype=torch.int8, device="cuda", generator=gen),
+            "sx": torch.rand((mt,), device="cuda", generator=gen) * 0.01 + 0.001,
+            "cq": torch.randint(-127, 128, (n, k // 64, 2), dtype=torch.int8, device="cuda", generator=gen),
+            "sc": torch.rand((n, 2), device="cuda", generator=gen) * 1e-3 + 1e-4,
+            "acc": torch.empty((2, mt, n), dtype=torch.int32, device="cuda"),
+        })
+
+    def step_a8():
+        for v in vit:
+            goq.gemm(v["d"], v["packed"], v["x"], mt, goq.I8, sx=v["sx"], cq=v["cq"], sc=v["sc"], acc=v["acc"])
+
+    step_a8()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(3):
+        step_a8()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / 3
+    ops = sum(2.0 * 2.0 * mt * v["n"] * v["k"] for v in vit)  # two bases, multiply-add = 2 ops
+    out["w3a8_vit_b16_int_tops"] = ops / (ms * 1e-3) / 1e12
+    out["w3a8_vit_b16_ms"] = ms
     return out
 
 

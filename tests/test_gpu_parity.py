@@ -194,7 +194,8 @@ def test_config4_prefill_2048_tokens_sampled_rows(goq):
 
 
 # ------------------------------------------------------------------------------------- integer path
-@pytest.mark.parametrize("n,k,g,b,m", [(48, 256, 64, 3, 200), (20, 192, 32, 2, 130), (16, 128, 128, 3, 1)])
+@pytest.mark.parametrize("n,k,g,b,m", [(48, 256, 64, 3, 200), (20, 192, 32, 2, 130), (16, 128, 128, 3, 1),
+                                       (40, 128, 16, 3, 70), (200, 384, 128, 3, 333)])
 def test_int8_path_bit_exact_small(goq, n, k, g, b, m):
     from tests.gpu_util import pack_weights, run_gemm_i8
     codes, meta, coef = _quantized(n, k, g, b, seed=31)
