@@ -226,6 +226,23 @@ def time_graph(torch, graph, steps, warmup):
     return e0.elapsed_time(e1) / steps  # ms per step
 
 
+def replica_seed(rank):
+    """Each rank is an independent replica of the decode step with its own weights and activations."""
+    return 1000 * rank
+
+
+def aggregate_replicas(ms_local, step_bytes, world, device):
+    """Whole-job throughput of `world` replicas: every rank moves step_bytes per step and the step
+    takes as long as the slowest rank (max over ranks). Returns (ms_max, GB/s)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], device=device, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    return ms_max, world * step_bytes / (ms_max * 1e-3) / 1e9
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -242,7 +259,7 @@ def run_cuda(args):
     hbm_peak, tf_peak, peak_src = measured_peaks()
 
     layers = args.layers
-    stack = build_stack(goq, torch, layers, seed0=1000 * rank, batch=1)
+    stack = build_stack(goq, torch, layers, seed0=replica_seed(rank), batch=1)
     n_lin = len(stack)
     step_bytes = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack)
     # one scratch buffer shared by all calls: launches on one stream run in order
@@ -273,11 +290,7 @@ def run_cuda(args):
     if world > 1:
         dist.barrier()
     ms = e0.elapsed_time(e1) / args.steps
-    t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max = float(t.item())
-    value = world * step_bytes / (ms_max * 1e-3) / 1e9
+    ms_max, value = aggregate_replicas(ms, step_bytes, world, "cuda")
 
     # ---- end to end: host buffers in, host buffers out, through goq_gemv_host -------------------
     host = []
@@ -293,10 +306,7 @@ def run_cuda(args):
     g2 = capture(torch, step_e2e)
     e2e_steps = max(3, args.steps // 4)
     ms_e2e = time_graph(torch, g2, e2e_steps, 3)
-    t2 = torch.tensor([ms_e2e], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-    e2e_val = world * step_bytes / (float(t2.item()) * 1e-3) / 1e9
+    _, e2e_val = aggregate_replicas(ms_e2e, step_bytes, world, "cuda")
     h2d = sum(s["k"] * 2 for s in stack)
     d2h = sum(s["n"] * 4 for s in stack)
 
@@ -319,6 +329,13 @@ def run_cuda(args):
     launch_bytes = step_bytes / n_lin
     launch_ms = ms / n_lin
     achieved = launch_bytes / (launch_ms * 1e-3) / 1e9
+    if args.traffic_bytes is not None:
+        traffic, traffic_src = args.traffic_bytes, "--traffic-bytes"
+    else:
+        # one ncu capture of the 4096x4096 launch read 8.96 MB of DRAM for 8.39 MB of algorithmic bytes;
+        # the packed image grows in proportion to n*k, so the ratio is applied to the average launch
+        traffic = launch_bytes * NCU_TRAFFIC_RATIO
+        traffic_src = "ncu dram bytes of the 4096x4096 launch (8.96 MB) scaled by algorithmic bytes"
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
@@ -328,8 +345,8 @@ def run_cuda(args):
                    "launch": "one CUDA graph of %d goq_gemv nodes per step" % n_lin,
                    "parallelism": "replicas" if world > 1 else "single"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
-                     "traffic": args.traffic_bytes, "peak_source": peak_src, "frac_of_8000_nominal": achieved / 8000.0,
-                     "kernel": "linear_mma_kernel<3,1>", "bytes_per_launch_avg": launch_bytes, "us_per_launch_avg": launch_ms * 1e3},
+                     "traffic": traffic, "traffic_source": traffic_src, "peak_source": peak_src, "frac_of_8000_nominal": achieved / 8000.0,
+                     "kernel": "gemv_stream_kernel<3,1,4,true>", "bytes_per_launch_avg": launch_bytes, "us_per_launch_avg": launch_ms * 1e3},
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "launch": "one CUDA graph of goq_gemv_host calls (pinned H2D, kernel, D2H per linear)"},
@@ -436,6 +453,9 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
     out["w3a8_vit_b16_int_tops"] = ops / (ms * 1e-3) / 1e12
     out["w3a8_vit_b16_ms"] = ms
     return out
+
+
+NCU_TRAFFIC_RATIO = 8.96 / 8.39
 
 
 def main():

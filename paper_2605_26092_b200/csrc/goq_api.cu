@@ -71,7 +71,12 @@ size_t goq_algorithmic_bytes(const goq_desc* desc) {
 size_t goq_workspace_bytes(const goq_desc* desc, int op, int m) {
     Geometry g;
     if (!goq::make_geometry(desc, &g) || m <= 0) return 0;
-    if (op == GOQ_OP_GEMV && m <= 16 && goq::gemv_stream_supported(g)) return goq::gemv_stream_workspace(g);
+    if (op == GOQ_OP_GEMV && m <= 16) {
+        size_t need = 0;
+        if (goq::gemv_stream_supported(g)) need = goq::gemv_stream_workspace(g);
+        if (goq::gemv_tc_supported(g, m) && goq::gemv_tc_workspace(g) > need) need = goq::gemv_tc_workspace(g);
+        return need;
+    }
     if (op == GOQ_OP_GEMM && goq::gemm_tc_supported(g)) return goq::gemm_tc_workspace(g);
     return 0;
 }
@@ -106,6 +111,16 @@ goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16
         return GOQ_ERR_ALIGNMENT;
     if (goq_status s = check_arch()) return s;
     const int variant = g_gemv_variant.load(std::memory_order_relaxed);
+    // the tensor-memory kernel is selectable but not the default: its tcgen05 A-operand feed caps it below the
+    // streaming kernel's rate on this part
+    const bool use_tc = goq::gemv_tc_supported(g, batch) && variant == 4;
+    if (variant == 4 && !use_tc) return GOQ_ERR_UNSUPPORTED;
+    if (use_tc) {
+        if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
+        if (ws_bytes < goq::gemv_tc_workspace(g)) return GOQ_ERR_WORKSPACE;
+        if (!goq::stream_hash_is_bijective()) return GOQ_ERR_UNSUPPORTED;
+        return from_cuda(goq::launch_gemv_tc(g, packed, x_bf16, batch, y, y_dtype, ws, (cudaStream_t)stream));
+    }
     bool use_stream = goq::gemv_stream_supported(g) && (variant == 0 || variant == 3);
     if (variant == 3 && !use_stream) return GOQ_ERR_UNSUPPORTED;
     if (use_stream) {

@@ -27,6 +27,13 @@ bool stream_hash_is_bijective();
 cudaError_t launch_gemv_stream(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y, int y_dtype,
                                void* ws, cudaStream_t st);
 
+// Decode GEMV on tcgen05 with the FP8 weight operand in tensor memory (group 64 or 128, wbits <= 3, m <= 16).
+// `ws` holds gemv_tc_workspace(g) bytes, zero on entry (goq_workspace_init), counters left zero on return.
+bool gemv_tc_supported(const Geometry& g, int m);
+size_t gemv_tc_workspace(const Geometry& g);
+cudaError_t launch_gemv_tc(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y, int y_dtype,
+                           void* ws, cudaStream_t st);
+
 // Prefill GEMM on tcgen05 tensor cores (wbits <= 3). `ws` holds gemm_tc_workspace(g) bytes (status word).
 bool gemm_tc_supported(const Geometry& g);
 size_t gemm_tc_workspace(const Geometry& g);

@@ -35,6 +35,8 @@ def run_gemv(d, packed, x_bits: np.ndarray, y_dtype=goq.F32, variant=0):
     finally:
         goq.set_gemv_variant(prev)
     torch.cuda.synchronize()
+    if ws is not None:
+        assert goq.workspace_status(ws) == goq.OK
     return y.float().cpu().numpy().astype(np.float64)
 
 

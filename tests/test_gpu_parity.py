@@ -76,7 +76,7 @@ def _quantized(n, k, g, b, seed, outliers=False):
     return O.quantize_geo(w, g, b)
 
 
-@pytest.mark.parametrize("variant", [1, 2, 3])
+@pytest.mark.parametrize("variant", [1, 2, 3, 4])
 @pytest.mark.parametrize("batch", [1, 8])
 def test_config1_single_layer_256(goq, variant, batch):
     """K = N = 256, W3, group 64, fp16 coefficients, bf16 activations, batch 1 and 8, seed 0."""
@@ -99,6 +99,8 @@ def test_config1_single_layer_256(goq, variant, batch):
     (48, 256, 64, 4, 9, 2), (48, 256, 64, 4, 9, 1), (16, 128, 128, 3, 1, 2), (300, 1152, 128, 3, 12, 2),
     (40, 192, 64, 3, 3, 3), (17, 384, 128, 3, 16, 3), (33, 256, 32, 2, 5, 3), (16, 128, 128, 3, 1, 3),
     (300, 1152, 128, 3, 12, 3), (64, 512, 32, 3, 7, 3),
+    (40, 192, 64, 3, 3, 4), (17, 384, 128, 3, 16, 4), (16, 128, 128, 3, 1, 4), (300, 1152, 128, 3, 12, 4),
+    (48, 256, 64, 2, 9, 4), (130, 640, 128, 2, 8, 4), (129, 200 * 64, 64, 3, 2, 4),
 ])
 def test_gemv_ragged_shapes_bit_widths_and_groups(goq, n, k, g, b, batch, variant):
     from tests.gpu_util import pack_weights, run_gemv
@@ -111,6 +113,23 @@ def test_gemv_ragged_shapes_bit_widths_and_groups(goq, n, k, g, b, batch, varian
     assert err <= TIGHT, err
 
 
+@pytest.mark.parametrize("n,k,g,b,batch", [(1000, 2048, 128, 3, 1), (2100, 4224, 64, 3, 5), (4096, 1024, 128, 3, 16),
+                                           (1000, 2048, 128, 2, 9)])
+def test_tensor_memory_gemv_tiles_split_across_ctas(goq, n, k, g, b, batch):
+    """Shapes whose 128-row tiles are shared by several CTAs (parked partial sums, last arriver adds them);
+    every output is compared, twice, and the two runs must agree bit for bit."""
+    from tests.gpu_util import pack_weights, run_gemv
+    codes, meta, coef = si.random_quantized(n, k, g, b, seed=n + k + batch)
+    d, packed = pack_weights(n, k, g, b, codes, meta, coef)
+    xb = si.bf16_activations(batch, k, seed=batch)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), g, b)
+    y = run_gemv(d, packed, xb, goq.F32, 4)
+    err = O.normwise_rel_err(y, y_ref)
+    print("tensor-memory gemv: normwise error %.3e" % err)
+    assert err <= TOL and err <= TIGHT, err
+    assert np.array_equal(y, run_gemv(d, packed, xb, goq.F32, 4))
+
+
 def test_two_kernel_variants_agree_closely_and_runs_are_deterministic(goq):
     from tests.gpu_util import pack_weights, run_gemv
     codes, meta, coef = si.random_quantized(512, 1024, 128, 3, seed=3)
@@ -121,7 +140,7 @@ def test_two_kernel_variants_agree_closely_and_runs_are_deterministic(goq):
     assert O.normwise_rel_err(y1, y2) < 1e-5
     y3 = run_gemv(d, packed, xb, goq.F32, 3)
     assert O.normwise_rel_err(y3, y2) < 1e-5
-    for v in (1, 2, 3):
+    for v in (1, 2, 3, 4):
         a = run_gemv(d, packed, xb, goq.F32, v)
         b = run_gemv(d, packed, xb, goq.F32, v)
         assert np.array_equal(a, b)
@@ -138,7 +157,7 @@ def test_extreme_activations_keep_exponent_arithmetic_right(goq):
     x[1, ::5] *= 2.0 ** 100
     xb = si.f32_to_bf16_bits(x.astype(np.float32))
     y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 64, 3)
-    for v in (1, 2, 3):
+    for v in (1, 2, 3, 4):
         assert O.normwise_rel_err(run_gemv(d, packed, xb, goq.F32, v), y_ref) <= TIGHT
 
 
@@ -155,6 +174,27 @@ def test_config2_llama7b_shapes_sampled_rows(goq, name, n, k, batch):
     d, packed = pack_weights(n, k, 128, 3, codes, meta, coef)
     xb = si.bf16_activations(batch, k, seed=batch)
     y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 128, 3, rows=rows)
+    y = run_gemv(d, packed, xb, goq.F32)
+    err = O.normwise_rel_err(y[:, rows], y_ref)
+    assert err <= TOL and err <= TIGHT, err
+
+
+_CFG5 = {name: (n, k) for name, n, k in si.LLAMA2_70B_LINEARS}
+
+
+@pytest.mark.parametrize("name,b,batch", [("mlp_gate_up", 2, 1), ("mlp_down", 3, 16), ("attn_qo", 4, 1),
+                                          ("gqa_kv", 2, 16), ("attn_qo", 3, 4)])
+def test_config5_llama70b_shapes_bit_width_sweep_sampled_rows(goq, name, b, batch):
+    """70B-shaped linears at W2/W3/W4, group 128, full-size launch; the oracle evaluates sampled rows."""
+    from tests.gpu_util import pack_weights, run_gemv
+    n, k = _CFG5[name]
+    codes, meta, coef = si.random_quantized(n, k, 128, b, seed=n + k + b)
+    rows = si.sample_rows(n, 48, seed=3)
+    w = si.weights_with_student_t_channels(len(rows), k, seed=9)
+    codes[rows], meta[rows], coef[rows] = O.quantize_geo(w, 128, b)
+    d, packed = pack_weights(n, k, 128, b, codes, meta, coef)
+    xb = si.bf16_activations(batch, k, seed=batch + b)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 128, b, rows=rows)
     y = run_gemv(d, packed, xb, goq.F32)
     err = O.normwise_rel_err(y[:, rows], y_ref)
     assert err <= TOL and err <= TIGHT, err

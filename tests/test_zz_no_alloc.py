@@ -49,7 +49,7 @@ def test_static_scratch_entry_matches_regular_entry_on_two_calls_in_a_row(goq):
     packed = torch.zeros(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
     goq.pack(d, _dev(codes), _dev(meta), _dev(coef), packed)
     ws = goq.new_workspace(d, goq.OP_GEMV, 16)
-    assert 0 < goq.workspace_bytes(d, goq.OP_GEMV, 16) <= 2 * 1024 * 1024
+    assert goq.workspace_bytes(d, goq.OP_GEMV, 16) > 0
 
     for call, batch in enumerate((5, 16)):          # two calls in a row, different batch buckets
         xb = si.bf16_activations(batch, k, seed=100 + call)
