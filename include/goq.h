@@ -95,9 +95,7 @@ goq_status goq_workspace_status(const void* ws, void* stream, int* status_out);
  *   coef_f16  [n_out][k_in/group][2] IEEE fp16 bit patterns (c1, c2)
  *   packed    out, goq_packed_bytes(desc) bytes, 128-byte aligned
  * Layout GOQ_LAYOUT_TILE16: rows padded to a multiple of 16 and k to a multiple of 128 with
- * zero-valued weights; the records of eight 16-row tiles at one 128-wide k-block are adjacent (a
- * 128 x 128 block is one contiguous run; the row-tile count is padded to a multiple of 8 with zero
- * records); one 32-bit word per micro-block (8 nibbles = 8 codes, record bits in the
+ * zero-valued weights; one 32-bit word per micro-block (8 nibbles = 8 codes, record bits in the
  * nibbles' spare top bits for wbits <= 3, in a side byte plane for wbits = 4); words ordered so
  * that the 32 lanes of a warp read 512 contiguous bytes per 128-bit load; coefficient pairs in a
  * second plane, 64 contiguous bytes per (16-row tile, group). */

@@ -2,12 +2,8 @@
 //
 // Layout GOQ_LAYOUT_TILE16 ("tile16"). Rows are padded to a multiple of 16 (a row tile), k to a
 // multiple of 128 (a k-block). The buffer is a sequence of unit records, one per (row tile T,
-// k-block bk). Eight row tiles form a super tile (128 rows, the M of one tcgen05 MMA); the records of
-// (super tile ST, k-block bk) are adjacent: record index ((T/8)*k_blocks + bk)*8 + T%8. The 128 x 128
-// block of weights one MMA operand is built from is therefore one contiguous byte range (what a bulk
-// copy wants, and large enough that the copy engine's per-request cost does not matter), and walking
-// the buffer in order walks k inside a super tile. The row-tile count is padded to a multiple of 8;
-// records of tiles that do not exist are zero. A unit record holds
+// k-block bk), in the order T*k_blocks + bk, so a run of consecutive records is one contiguous
+// byte range (what a bulk copy wants). A unit record holds
 //   [0, 1024)            256 micro-block words. One 32-bit word = one micro-block (8 weights,
 //                        Section 3.3 of the paper): nibble i, bits [4i+2:4i], is the code of weight i;
 //                        for wbits <= 3 the six bits of the exchange record sit in bit 3 of nibbles 0..5.
@@ -31,13 +27,11 @@ constexpr int kTileRows = 16;
 constexpr int kBlockK = 128;
 constexpr int kWordsPerBlock = 256;
 constexpr int kCodeBytesPerUnit = kWordsPerBlock * 4;
-constexpr int kSuperTiles = 8;  // row tiles per super tile
 
 struct Geometry {
     int n_out, k_in, group, wbits;
     int n_pad, k_pad;
     int n_tiles, k_blocks, n_groups;  // n_groups counts padded groups: k_pad / group
-    int n_super;                      // super tiles: ceil(n_tiles / 8)
     int groups_per_block;             // 128 / group
     int unit_bytes;                   // bytes of one unit record
     int meta_off;                     // offset of the record-byte plane inside a unit (wbits = 4 only)
@@ -64,8 +58,7 @@ __host__ inline bool make_geometry(const goq_desc* d, Geometry* g) {
     g->groups_per_block = kBlockK / gr;
     g->meta_off = kCodeBytesPerUnit + 64 * g->groups_per_block;
     g->unit_bytes = g->meta_off + (d->wbits == 4 ? kWordsPerBlock : 0);
-    g->n_super = (g->n_tiles + kSuperTiles - 1) / kSuperTiles;
-    g->n_units = (size_t)g->n_super * kSuperTiles * g->k_blocks;
+    g->n_units = (size_t)g->n_tiles * g->k_blocks;
     g->total_bytes = g->n_units * (size_t)g->unit_bytes;
     return true;
 }
@@ -76,7 +69,7 @@ __host__ __device__ inline int word_in_unit(int row, int mb) {
     return v * 128 + (g * 4 + t) * 4 + c;
 }
 __host__ __device__ inline size_t unit_offset(int tile, int bk, int k_blocks, int unit_bytes) {
-    return (((size_t)(tile >> 3) * k_blocks + bk) * kSuperTiles + (tile & 7)) * (size_t)unit_bytes;
+    return ((size_t)tile * k_blocks + bk) * (size_t)unit_bytes;
 }
 
 // ---- scalar decode helpers (used by pack/unpack and the scalar kernels) --------------------

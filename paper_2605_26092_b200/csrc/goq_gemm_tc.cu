@@ -264,15 +264,17 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
     if (warp == 0) {
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
+            int n_rec = p.n_tiles - T0;
+            if (n_rec > kExpanders) n_rec = kExpanders;
             bool ok = true;
             for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
                 const int ps = kb & 1;
                 if (kb >= 2) ok = mbar_wait(&pk_empty[ps], ((kb >> 1) - 1) & 1, &abort_flag);
                 if (!ok) break;
-                // the records of this CTA's eight row tiles at one k-block are adjacent (one super tile)
-                mbar_expect_tx(&pk_full[ps], (uint32_t)pk_slot_bytes);
-                bulk_g2s(pk_ring + ps * pk_slot_bytes, p.packed + unit_offset(T0, kb, p.k_blocks, p.unit_bytes),
-                         (uint32_t)pk_slot_bytes, &pk_full[ps]);
+                mbar_expect_tx(&pk_full[ps], (uint32_t)n_rec * p.unit_bytes);
+                for (int r = 0; r < n_rec; ++r)
+                    bulk_g2s(pk_ring + ps * pk_slot_bytes + r * p.unit_bytes,
+                             p.packed + unit_offset(T0 + r, kb, p.k_blocks, p.unit_bytes), p.unit_bytes, &pk_full[ps]);
                 for (int half = 0; half < 2 && ok; ++half) {
                     const int chunk = 2 * kb + half, s = chunk % kStages;
                     if (chunk >= kStages) ok = mbar_wait(&empty[s], ((chunk / kStages) - 1) & 1, &abort_flag);

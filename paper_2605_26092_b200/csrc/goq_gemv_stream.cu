@@ -5,11 +5,10 @@
 // exact PoT operands (a PoT factor only shifts the activation's exponent, so no product rounds), the
 // sums are fp32, and the coefficient multiply happens once per macro-block outside the MMA.
 //
-// Work decomposition. The packed buffer is an array of unit records (1 KiB of codes plus the coefficients
-// of 16 rows x 128 k). With the U records of existing row tiles numbered in the order (row tile, k-block),
-// CTA i takes the range [U*i/G, U*(i+1)/G), so every SM streams the same number of bytes whatever the
-// shape. A producer warp moves the range through a ring of shared-memory stages with 1-D bulk async copies
-// (one record per lane, mbarrier completion); eight
+// Work decomposition. The packed buffer is one contiguous array of unit records (1 KiB of codes plus
+// the coefficients of 16 rows x 128 k). CTA i takes the contiguous range [U*i/G, U*(i+1)/G) of the U
+// records, so every SM streams the same number of bytes whatever the shape. A producer thread moves the
+// range through a ring of shared-memory stages with 1-D bulk async copies (mbarrier completion); eight
 // consumer warps each take one record per stage. Lane (g,t) of a consumer owns whole micro-blocks of
 // rows g and g+8, so the Strided Dual-Exchange of Section 3.3 never leaves the thread. A 16-row tile
 // that straddles CTAs is finished by whichever CTA arrives last, adding the parked partial sums in CTA
@@ -298,35 +297,29 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
 
     if (warp == kConsumerWarps) {
         // ---------------- producer: one thread streams this CTA's records through the ring -------------
-        // Records are taken in the order (row tile, k-block); eight of them fill a stage. In the packed buffer
-        // consecutive k-blocks of one row tile are a super-tile stride apart, so lane r copies record r.
-        {
+        if (lane == 0) {
+            const uint8_t* src = p.packed + (size_t)u_begin * p.unit_bytes;
             int slot = 0, round = 0;
             bool x_issued = (p.x_smem_bytes == 0);
             for (int s = 0; s < my_stages; ++s) {
-                bool ok = true;
-                if (round > 0 && lane == 0) ok = mbar_wait_bounded(&empty_bar[slot], (round - 1) & 1, &abort_flag);
-                if (!__all_sync(0xFFFFFFFFu, ok)) break;
-                const int units = min(kStageUnits, my_units - s * kStageUnits);
-                if (lane == 0) mbar_arrive_expect_tx(&full_bar[slot], (uint32_t)units * p.unit_bytes);
-                __syncwarp();
-                if (lane < units) {
-                    const int u = u_begin + s * kStageUnits + lane, T = u / p.k_blocks, bk = u - T * p.k_blocks;
-                    bulk_copy_g2s(ring + (size_t)slot * stage_bytes + (size_t)lane * p.unit_bytes,
-                                  p.packed + unit_offset(T, bk, p.k_blocks, p.unit_bytes), (uint32_t)p.unit_bytes, &full_bar[slot]);
+
+                if (round > 0) {
+                    if (!mbar_wait_bounded(&empty_bar[slot], (round - 1) & 1, &abort_flag)) break;
                 }
+                const int units = min(kStageUnits, my_units - s * kStageUnits);
+                const uint32_t bytes = (uint32_t)units * p.unit_bytes;
+                mbar_arrive_expect_tx(&full_bar[slot], bytes);
+                bulk_copy_g2s(ring + (size_t)slot * stage_bytes, src + (size_t)s * stage_bytes, bytes, &full_bar[slot]);
                 if (++slot == p.n_stages) { slot = 0; ++round; }
                 if (s == 0) GOQ_TR(2);
                 if (!x_issued && (s + 1 == my_stages || s + 1 == p.n_stages)) {
                     // the ring is primed: now the activations, which the preceding kernel may have produced
                     asm volatile("griddepcontrol.wait;" ::: "memory");
-                    if (lane == 0) {
-                        const uint32_t row_bytes = (uint32_t)p.k_in * 2;
-                        mbar_arrive_expect_tx(x_bar, row_bytes * p.m_total);
-                        for (int r = 0; r < p.m_total; ++r)
-                            bulk_copy_g2s(const_cast<uint16_t*>(xs) + (size_t)r * p.k_blocks * kBlockK, p.x + (size_t)r * p.k_in,
-                                          row_bytes, x_bar);
-                    }
+                    const uint32_t row_bytes = (uint32_t)p.k_in * 2;
+                    mbar_arrive_expect_tx(x_bar, row_bytes * p.m_total);
+                    for (int r = 0; r < p.m_total; ++r)
+                        bulk_copy_g2s(const_cast<uint16_t*>(xs) + (size_t)r * p.k_blocks * kBlockK, p.x + (size_t)r * p.k_in,
+                                      row_bytes, x_bar);
                     x_issued = true;
                 }
             }
@@ -644,7 +637,7 @@ cudaError_t launch_gemv_stream(const Geometry& g, const void* packed, const void
     p.status = (int*)wsb;
     p.counters = (int*)(wsb + L.counters_off);
     p.partials = (float*)(wsb + L.partials_off);
-    p.n_units = g.n_tiles * g.k_blocks;  // existing row tiles only, visited in the order (row tile, k-block)
+    p.n_units = (int)g.n_units;
     p.unit_bytes = g.unit_bytes;
     p.k_blocks = g.k_blocks;
     p.k_in = g.k_in;

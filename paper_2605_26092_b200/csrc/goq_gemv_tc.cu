@@ -18,7 +18,7 @@
 // lo are two columns of the B operand; the epilogue recombines them with the block's scale.
 //
 // Roles in a CTA (one CTA per SM, contiguous range of 128x128 super-units, Stream-K style):
-//   warp 0      producer: 1-D bulk async copies of unit records into a ring of stages
+//   warp 0      producer: 1-D bulk async copies of unit records (one per lane) into a ring of stages
 //   warp 1      MMA issuer (one thread), owns the tensor-memory allocation
 //   warps 2-3   activation slicer: bf16 -> two e4m3 slices, written as the swizzled K-major B tile
 //   warps 4-19  two teams of eight expander warps: words -> FP8 bytes -> tensor memory
@@ -73,40 +73,23 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
 }
 __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
     uint32_t ok;
-#if defined(GOQ_EXP_TESTWAIT)
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(s32(b)), "r"(parity) : "memory");
-#elif defined(GOQ_EXP_HINT)
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(s32(b)), "r"(parity), "r"((uint32_t)GOQ_EXP_HINT) : "memory");
-#else
     asm volatile(
         "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(s32(b)), "r"(parity) : "memory");
-#endif
     return ok != 0;
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
     for (int it = 0; it < kSpin; ++it) {
         if (mbar_try(b, parity)) return true;
         if ((it & 63) == 63 && *abort_flag) return false;
-#ifdef GOQ_EXP_SLEEP
-        __nanosleep(GOQ_EXP_SLEEP);
-#endif
     }
     *abort_flag = 1;
     return false;
 }
-// Whole-warp wait with one polling lane: a warp-wide poll is 32 shared-memory barrier operations per try, and
-// a dozen waiting warps doing that starve the loads of the warps that have work.
+// Whole-warp wait with one polling lane (a warp-wide poll is 32 shared-memory barrier operations per try).
 __device__ __forceinline__ bool warp_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
     bool ok = true;
-#ifndef GOQ_EXP_ALLPOLL
-    if ((threadIdx.x & 31) == 0)
-#endif
-        ok = mbar_wait(b, parity, abort_flag);
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(b, parity, abort_flag);
     return __all_sync(0xFFFFFFFFu, ok);
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -247,21 +230,9 @@ __device__ __forceinline__ void decode_word(uint32_t w, uint32_t lut_lane, uint3
     const uint32_t m = w & 0x77777777u;
     b1a = prmt(PotFp8<WB>::F0, PotFp8<WB>::F1, m);
     // shifts written as high multiplies: they issue on the multiplier pipe, not on the half-rate logic pipe
-#ifndef GOQ_OPT_NO_UMULHI
     b1b = prmt(PotFp8<WB>::F0, PotFp8<WB>::F1, __umulhi(m, 1u << 16));
-#else
-    b1b = prmt(PotFp8<WB>::F0, PotFp8<WB>::F1, m >> 16);
-#endif
     const uint32_t h = (w - m) * kHashMul;
-#ifdef GOQ_EXP_NOLUT
-    const uint4 e = make_uint4(0x3210u ^ (h >> 28), 0x7654u, h & 0x80808080u, 0u);
-#else
-#ifndef GOQ_OPT_NO_UMULHI
     const uint4 e = lds128((__umulhi(h, 1u << 13) & 0x1F80u) | lut_lane);  // entry (h >> 26) * 128 + copy * 16, table 8 KiB aligned
-#else
-    const uint4 e = lds128(((h >> 19) & 0x1F80u) | lut_lane);
-#endif
-#endif
     b2a = prmt(b1a, b1b, e.x) ^ e.z;   // a flipped zero becomes -0: adds nothing
     b2b = prmt(b1a, b1b, e.y) ^ e.w;
 }
@@ -408,9 +379,14 @@ gemv_tc_kernel(const Params p) {
     // The producer warp sets up the barriers and starts the weight stream at once (the first ring-full of
     // copies waits for nobody); the other warps fill the tables meanwhile.
     const int stage_fill = R.nq < p.n_stages ? R.nq : p.n_stages;
-    auto issue = [&](const Cursor& c) {   // one thread: the eight records of a super-unit are one contiguous run
-        mbar_expect_tx(&full[c.s], (uint32_t)stage_bytes);
-        bulk_g2s(stages + c.s * stage_bytes, p.packed + (size_t)c.su * stage_bytes, (uint32_t)stage_bytes, &full[c.s]);
+    auto issue = [&](const Cursor& c) {   // whole producer warp: lane r copies record r of the super-unit
+        int n_rec = p.n_tiles - c.st * kRowTiles;
+        if (n_rec > kRowTiles) n_rec = kRowTiles;
+        if (lane == 0) mbar_expect_tx(&full[c.s], (uint32_t)n_rec * p.unit_bytes);
+        __syncwarp();
+        if (lane < n_rec)
+            bulk_g2s(stages + c.s * stage_bytes + lane * p.unit_bytes,
+                     p.packed + unit_offset(c.st * kRowTiles + lane, c.bk, p.k_blocks, p.unit_bytes), (uint32_t)p.unit_bytes, &full[c.s]);
     };
     Cursor pc;   // producer's position
     pc.init(R, 0, p.k_blocks, p.n_stages);
@@ -425,7 +401,7 @@ gemv_tc_kernel(const Params p) {
         // the barriers exist: let the other warps go on without waiting for the first copies to be issued
         asm volatile("bar.arrive 2, %0;" ::"n"(kThreads) : "memory");
         GOQ_TR(2);
-        if (lane == 0) for (int q = 0; q < stage_fill; ++q) { issue(pc); pc.next(R, p.k_blocks, p.n_stages); }
+        for (int q = 0; q < stage_fill; ++q) { issue(pc); pc.next(R, p.k_blocks, p.n_stages); }
         GOQ_TR(3);
     } else {
         for (int i = tid - 32; i < 512; i += kThreads - 32) {  // entry i>>3, copy i&7 at byte (i>>3)*128 + (i&7)*16
@@ -451,14 +427,13 @@ gemv_tc_kernel(const Params p) {
         // ------------------------------------------------ producer ------------------------------------------------
         bool ok = true;
         int q = stage_fill;
-        if (lane == 0) {
-            for (; q < R.nq; ++q) {
-                ok = mbar_wait(&empty[pc.s], pc.ph ^ 1u, &abort_flag);
-                if (!ok) break;
-                issue(pc);
-                pc.next(R, p.k_blocks, p.n_stages);
-                if (q >= GOQ_TRQ0 + 8 && q - GOQ_TRQ0 - 8 < 6) GOQ_TR(4 + q - GOQ_TRQ0 - 8);
-            }
+        for (; q < R.nq; ++q) {
+            if (lane == 0) ok = mbar_wait(&empty[pc.s], pc.ph ^ 1u, &abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            issue(pc);
+            pc.next(R, p.k_blocks, p.n_stages);
+            if (q >= GOQ_TRQ0 + 8 && q - GOQ_TRQ0 - 8 < 6) GOQ_TR(4 + q - GOQ_TRQ0 - 8);
         }
         GOQ_TR(14);
         if (lane == 0 && (!ok || abort_flag)) {
@@ -488,15 +463,7 @@ gemv_tc_kernel(const Params p) {
 #pragma unroll
                         for (int beta = 0; beta < 2; ++beta) {
                             const int j = (GPB == 2) ? h * 2 + jj : jj * 2 + h;   // 32-wide k slice of the k-block
-#if defined(GOQ_EXP_MMA8)
-                            umma_f8_ts(tb + 64 + ((jj * 4 + h * 2 + beta) & 3) * N + (jj ? 8 : 0), tb + beta * 32 + 8 * j, bdesc + 2 * j, idesc_e4m3(8 * 2), 0u);
-#elif defined(GOQ_EXP_MMAHALF)
-                            if (beta == 0) umma_f8_ts(tb + 64 + (h * 2 + beta) * N, tb + beta * 32 + 8 * j, bdesc + 2 * j, idesc, jj > 0 ? 1u : 0u);
-#elif defined(GOQ_EXP_MMAN64)
-                            umma_f8_ts(tb + 64, tb + beta * 32 + 8 * j, bdesc + 2 * j, idesc_e4m3(64), jj > 0 ? 1u : 0u);
-#elif !defined(GOQ_EXP_NOMMA)
                             umma_f8_ts(tb + 64 + (h * 2 + beta) * N, tb + beta * 32 + 8 * j, bdesc + 2 * j, idesc, jj > 0 ? 1u : 0u);
-#endif
                         }
                 umma_commit(&d_ready[buf]);
                 if (q >= GOQ_TRQ0 && q - GOQ_TRQ0 < 5) GOQ_TR(5 + 2 * (q - GOQ_TRQ0));
@@ -671,9 +638,7 @@ gemv_tc_kernel(const Params p) {
             if (q >= GOQ_TRQ0 && (q - GOQ_TRQ0) / kTeams < 2) GOQ_TRD(5 + 5 * ((q - GOQ_TRQ0) / kTeams), a2[0] ^ a2[15] ^ a2[7] ^ a1[9]);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[s]);   // the record is in registers
-#ifndef GOQ_OPT_NO_PREFETCH
             have = (en.q < R.nq) ? fetch(en, false) : false;
-#endif
             ec = en;
             en.skip(kTeams, R, p.k_blocks, p.n_stages);
             if (q >= GOQ_TRQ0 && (q - GOQ_TRQ0) / kTeams < 2) GOQ_TR(6 + 5 * ((q - GOQ_TRQ0) / kTeams));
@@ -681,12 +646,8 @@ gemv_tc_kernel(const Params p) {
             if (!ok) break;
             tc_fence_after();
             const uint32_t ta = tmem_base + (lane_base << 16) + (uint32_t)(buf * kBufCols);
-#ifndef GOQ_EXP_NOST
             tmem_st_16x256b_x4(ta, a1);
             tmem_st_16x256b_x4(ta + 32, a2);
-#else
-            if (a1[0] == 0x12345678u && a2[3] == a1[7] + 1u && a1[12] == a2[15]) tmem_st_16x256b_x4(ta, a1);
-#endif
             if (lane < 16) {
 #pragma unroll
                 for (int gi = 0; gi < GPB; ++gi) sts32(coefbuf + ((buf * GPB + gi) * 128 + j * 16 + lane) * 4, cwc[gi]);

@@ -98,11 +98,6 @@ __global__ void unpack_coef_kernel(const uint8_t* __restrict__ packed, uint16_t*
 cudaError_t launch_pack(const Geometry& g, const uint8_t* codes, const uint8_t* meta, const uint16_t* coef,
                         void* packed, cudaStream_t st) {
     auto* base = (uint8_t*)packed;
-    if (g.n_tiles % kSuperTiles) {  // records of the row tiles that pad the last super tile
-        cudaError_t e = cudaMemsetAsync(base + unit_offset((g.n_super - 1) * kSuperTiles, 0, g.k_blocks, g.unit_bytes), 0,
-                                        (size_t)kSuperTiles * g.k_blocks * g.unit_bytes, st);
-        if (e != cudaSuccess) return e;
-    }
     size_t nw = (size_t)g.n_pad * (g.k_pad / 8);
     pack_words_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(codes, meta, base, g.n_out, g.k_in, g.n_pad,
                                                                    g.k_pad, g.wbits, g.unit_bytes, g.meta_off);

@@ -40,9 +40,9 @@ def test_size_queries(goq):
     # packed: one 32-bit word per 8 weights + 4 bytes per (row, group)
     assert goq.packed_bytes(d) == 4096 * 4096 // 2 + 4096 * 32 * 4
     assert goq.algorithmic_bytes(goq.desc(256, 256, 64, 3)) == 256 * 256 * 15 // 32 + 256 * 4 * 4
-    # padding to 128 rows (eight 16-row tiles form a super tile) x 128 k
+    # padding to 16 rows x 128 k
     d2 = goq.desc(40, 192, 64, 3)
-    assert goq.packed_bytes(d2) == 128 * 256 // 2 + 128 * 4 * 4
+    assert goq.packed_bytes(d2) == 48 * 256 // 2 + 48 * 4 * 4
     assert goq.packed_bytes(goq.desc(40, 192, 64, 4)) > goq.packed_bytes(d2)
     for bad in [goq.desc(0, 128, 64, 3), goq.desc(16, 100, 64, 3), goq.desc(16, 128, 24, 3),
                 goq.desc(16, 128, 64, 5), goq.desc(16, 128, 64, 3, layout=7), goq.desc(16, 128, 256, 3)]:
