@@ -266,9 +266,21 @@ def run_cuda(args):
     ws = torch.empty(build_stack.ws_bytes, dtype=torch.uint8, device="cuda")
     goq.workspace_init(ws)
 
-    def step():
-        for s in stack:
-            goq.gemv(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, ws=ws)
+    if args.launch == "sequence":
+        # the whole step is one persistent kernel; every linear waits for all earlier ones (stream-order semantics)
+        seq = goq.make_sequence([(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, True) for s in stack])
+        ws_seq = torch.empty(goq.sequence_workspace_bytes(n_lin), dtype=torch.uint8, device="cuda")
+        goq.workspace_init(ws_seq)
+        kernels_per_step = (n_lin + 255) // 256
+
+        def step():
+            goq.gemv_sequence(seq, ws_seq)
+    else:
+        kernels_per_step = n_lin
+
+        def step():
+            for s in stack:
+                goq.gemv(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, ws=ws)
 
     graph = capture(torch, step)
 
@@ -326,31 +338,40 @@ def run_cuda(args):
         cpu = {"value": gbs, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                "sample": "one layer's 7 linears x 2048 output rows each, batch 1 (%.2f s per pass, best of 3)" % secs}
 
-    launch_bytes = step_bytes / n_lin
-    launch_ms = ms / n_lin
+    launch_bytes = step_bytes / kernels_per_step
+    launch_ms = ms / kernels_per_step
     achieved = launch_bytes / (launch_ms * 1e-3) / 1e9
+    if args.launch == "sequence":
+        kernel_name = "gemv_seq_kernel<3,4>"
+        launch_desc = "one CUDA graph holding one goq_gemv_sequence call (%d linears, each waits for all earlier ones)" % n_lin
+        ratio, ratio_src = NCU_TRAFFIC_RATIO_SEQ, "ncu dram bytes of a 14-linear sequence launch scaled by algorithmic bytes"
+        if int(goq.workspace_status(ws_seq)) != 0:
+            raise RuntimeError("sequence kernel reported a device-side timeout")
+    else:
+        kernel_name = "gemv_stream_kernel<3,1,4,true>"
+        launch_desc = "one CUDA graph of %d goq_gemv nodes per step" % n_lin
+        # one ncu capture of the 4096x4096 launch read 8.96 MB of DRAM for 8.39 MB of algorithmic bytes;
+        # the packed image grows in proportion to n*k, so the ratio is applied to the average launch
+        ratio, ratio_src = NCU_TRAFFIC_RATIO, "ncu dram bytes of the 4096x4096 launch (8.96 MB) scaled by algorithmic bytes"
     if args.traffic_bytes is not None:
         traffic, traffic_src = args.traffic_bytes, "--traffic-bytes"
     else:
-        # one ncu capture of the 4096x4096 launch read 8.96 MB of DRAM for 8.39 MB of algorithmic bytes;
-        # the packed image grows in proportion to n*k, so the ratio is applied to the average launch
-        traffic = launch_bytes * NCU_TRAFFIC_RATIO
-        traffic_src = "ncu dram bytes of the 4096x4096 launch (8.96 MB) scaled by algorithmic bytes"
+        traffic, traffic_src = (launch_bytes * ratio, ratio_src) if ratio else (None, "not captured")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": WORKLOAD, "layers": layers, "linears_per_step": n_lin, "batch": 1,
                    "bytes_per_step": step_bytes, "l2": "weights per step %.2f GB >> 126 MB L2, no flush needed" % (step_bytes / 1e9),
-                   "launch": "one CUDA graph of %d goq_gemv nodes per step" % n_lin,
+                   "launch": launch_desc,
                    "parallelism": "replicas" if world > 1 else "single"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
                      "traffic": traffic, "traffic_source": traffic_src, "peak_source": peak_src, "frac_of_8000_nominal": achieved / 8000.0,
-                     "kernel": "gemv_stream_kernel<3,1,4,true>", "bytes_per_launch_avg": launch_bytes, "us_per_launch_avg": launch_ms * 1e3},
+                     "kernel": kernel_name, "bytes_per_launch_avg": launch_bytes, "us_per_launch_avg": launch_ms * 1e3},
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "launch": "one CUDA graph of goq_gemv_host calls (pinned H2D, kernel, D2H per linear)"},
-        "gpu_launches": args.steps * n_lin,
+        "gpu_launches": args.steps * kernels_per_step,
         "clocks": sampler.summary(),
         "extras": extras,
     }
@@ -376,6 +397,25 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
         nbytes = sum(algorithmic_bytes(s["n"], s["k"], batch) for s in stack)
         out["gemv_batch%d_gbs" % batch] = nbytes / (ms * 1e-3) / 1e9
         del g, xs, ys
+    # the same decode step issued the other way (per-linear launches in a CUDA graph)
+    def step_graph():
+        for s in stack:
+            goq.gemv(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, ws=ws)
+
+    g = capture(torch, step_graph)
+    ms = time_graph(torch, g, 20, 3)
+    out["gemv_graph_of_launches_gbs"] = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack) / (ms * 1e-3) / 1e9
+    del g
+    # ... and as a sequence whose dependencies follow a transformer layer (k, v and up need not wait)
+    names = [nm for nm, _, _ in si.LLAMA2_7B_LINEARS]
+    seq = goq.make_sequence([(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, names[j % 7] not in ("k_proj", "v_proj", "up_proj"))
+                             for j, s in enumerate(stack)])
+    ws_seq = torch.empty(goq.sequence_workspace_bytes(len(stack)), dtype=torch.uint8, device="cuda")
+    goq.workspace_init(ws_seq)
+    g = capture(torch, lambda: goq.gemv_sequence(seq, ws_seq))
+    ms = time_graph(torch, g, 20, 3)
+    out["gemv_sequence_layer_groups_gbs"] = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack) / (ms * 1e-3) / 1e9
+    del g
     # per-shape batch-1 time (rotating over the layers' copies of that shape, so each launch reads cold weights)
     shapes = {}
     for idx, (name, n, k) in enumerate(si.LLAMA2_7B_LINEARS):
@@ -456,6 +496,7 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
 
 
 NCU_TRAFFIC_RATIO = 8.96 / 8.39
+NCU_TRAFFIC_RATIO_SEQ = None   # dram bytes / algorithmic bytes of the sequence kernel, from its ncu capture
 
 
 def main():
@@ -467,6 +508,8 @@ def main():
     ap.add_argument("--layers", type=int, default=si.LLAMA2_7B_LAYERS)
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--launch", choices=("sequence", "graph"), default="sequence",
+                    help="how a step is issued: one goq_gemv_sequence call, or a CUDA graph of per-linear goq_gemv launches")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="dram bytes per launch of the dominant kernel from an ncu capture (reported as-is)")
     args = ap.parse_args()

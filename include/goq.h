@@ -165,6 +165,35 @@ goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x
 goq_status goq_gemv_static(const goq_desc* desc, const void* packed, const void* x_bf16, int batch, void* y,
                            int y_dtype, void* stream);
 
+/* goq_gemv_sequence: a chain of decode GEMVs (Eq. 4, one call of goq_gemv each) executed by ONE persistent
+ * cooperative kernel, in order. Results are those of calling goq_gemv item by item on one stream; what changes
+ * is the cost: no launch, prologue or first-byte latency per linear, and the weight stream never stops at a
+ * boundary between linears.
+ *   items    HOST array of n_items entries (read during the call, not kept):
+ *            desc, packed, x_bf16 [batch][k_in], y [batch][n_out], y_dtype as in goq_gemv, all device pointers;
+ *            depends != 0 : this item's x (or y) may alias outputs of EARLIER items of the sequence - the kernel
+ *                           then waits until every earlier item is complete before it reads x;
+ *            depends == 0 : x and y are independent of every earlier item (their buffers must not overlap the
+ *                           outputs of earlier items).
+ *   Constraints (else GOQ_ERR_UNSUPPORTED): every item has the same wbits (2 or 3) and group (32, 64, 128),
+ *   batch <= 8, and batch * round_up(k_in, 128) * 2 bytes <= 23040 (the activations are staged in shared memory).
+ *   ws       goq_sequence_workspace_bytes(n_items) bytes, 256-byte aligned, zeroed once with goq_workspace_init;
+ *            the call leaves it zero. One status word as for goq_gemv (goq_workspace_status).
+ * Sequences longer than GOQ_SEQUENCE_MAX_ITEMS are split into several launches. The device must support
+ * cooperative launches (every sm_100 device does); the grid is sized so that all CTAs are resident. */
+typedef struct {
+    goq_desc desc;
+    const void* packed;
+    const void* x_bf16;
+    void* y;
+    int32_t batch;
+    int32_t y_dtype;
+    int32_t depends;
+} goq_gemv_item;
+#define GOQ_SEQUENCE_MAX_ITEMS 256
+size_t goq_sequence_workspace_bytes(int n_items);
+goq_status goq_gemv_sequence(const goq_gemv_item* items, int n_items, void* ws, size_t ws_bytes, void* stream);
+
 /* The cudaError_t value behind the most recent GOQ_ERR_CUDA returned in this process (0 if none). */
 int goq_last_cuda_error(void);
 

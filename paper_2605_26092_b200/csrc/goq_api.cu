@@ -1,6 +1,7 @@
 // C ABI of libgoq: argument checks on the host, then one launcher per call.
 #include <atomic>
 #include <cstdlib>
+#include <vector>
 #include "goq_common.cuh"
 #include "goq_internal.h"
 
@@ -179,6 +180,38 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
                                              (cudaStream_t)stream));
     }
     return GOQ_ERR_INVALID_ARG;
+}
+
+size_t goq_sequence_workspace_bytes(int n_items) { return n_items > 0 ? goq::gemv_seq_workspace(n_items) : 0; }
+
+goq_status goq_gemv_sequence(const goq_gemv_item* items, int n_items, void* ws, size_t ws_bytes, void* stream) {
+    if (!items || n_items < 1) return GOQ_ERR_INVALID_ARG;
+    static thread_local std::vector<goq::SeqCall> calls;
+    calls.resize((size_t)n_items);
+    for (int i = 0; i < n_items; ++i) {
+        const goq_gemv_item& it = items[i];
+        goq::SeqCall& c = calls[(size_t)i];
+        if (!goq::make_geometry(&it.desc, &c.g) || !it.packed || !it.x_bf16 || !it.y) return GOQ_ERR_INVALID_ARG;
+        if (it.batch < 1 || it.batch > 16) return GOQ_ERR_INVALID_ARG;
+        if (it.y_dtype != GOQ_BF16 && it.y_dtype != GOQ_F32) return GOQ_ERR_INVALID_ARG;
+        if (!aligned(it.packed, 128) || !aligned(it.x_bf16, 16) || !aligned(it.y, it.y_dtype == GOQ_F32 ? 4 : 2))
+            return GOQ_ERR_ALIGNMENT;
+        if (!goq::gemv_seq_supported(c.g, it.batch)) return GOQ_ERR_UNSUPPORTED;
+        if (c.g.wbits != calls[0].g.wbits || c.g.group != calls[0].g.group) return GOQ_ERR_UNSUPPORTED;
+        c.packed = it.packed; c.x = it.x_bf16; c.y = it.y; c.m = it.batch; c.y_dtype = it.y_dtype; c.depends = it.depends ? 1 : 0;
+    }
+    if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
+    if (ws_bytes < goq::gemv_seq_workspace(n_items)) return GOQ_ERR_WORKSPACE;
+    if (goq_status s = check_arch()) return s;
+    if (!goq::stream_hash_is_bijective()) return GOQ_ERR_UNSUPPORTED;
+    for (int i0 = 0; i0 < n_items; i0 += goq::kSeqMaxItems) {
+        const int n = (n_items - i0 < goq::kSeqMaxItems) ? (n_items - i0) : goq::kSeqMaxItems;
+        // a chunk boundary is a kernel boundary on the stream: the first item of a chunk needs no counter wait
+        cudaError_t e = goq::launch_gemv_seq(&calls[(size_t)i0], n, calls[0].g.wbits, calls[0].g.group, calls[0].g.unit_bytes, ws,
+                                             (cudaStream_t)stream);
+        if (e != cudaSuccess) return from_cuda(e);
+    }
+    return GOQ_OK;
 }
 
 goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x_host, int batch, void* y_host,

@@ -1,0 +1,360 @@
+// A sequence of decode GEMVs (batch <= 8) in ONE persistent kernel.
+//
+// A decode step is a chain of small linears (Eq. 4 of the paper per layer): each streams a few MB of
+// packed weights, far too little to hide a kernel's launch, prologue, first-byte latency and tail. Here the
+// whole chain runs in one cooperative launch: every CTA stays resident, its producer thread keeps the
+// weight stream going across the boundary between two linears (weights never depend on an earlier result),
+// and a linear whose activations do depend on earlier outputs waits on a device-wide completion counter
+// before it reads them - only that wait and the activation fetch are serial.
+//
+// Work unit = one 16-row tile of one linear, all of K (no split across CTAs, hence no partial-sum hand-off):
+// tile number base_p + T goes to CTA (base_p + T) mod G. Inside the CTA the tile's unit records (16 rows x
+// 128 k each, contiguous in the packed buffer) are streamed 16 at a time into a ring of shared-memory
+// stages by 1-D bulk async copies; consumer warp w takes record w of each stage, so the warps split K. The
+// math per record is that of the streaming kernel: b1 and b2 as exact bf16 PoT operands of mma.sync
+// (the exchange of Section 3.3 stays inside a lane), fp32 sums, coefficient multiply once per macro-block.
+// The last warp to finish a tile adds the 16 partial sums in warp order and stores the outputs.
+//
+// Every wait is bounded (mbarriers, the completion counters); on expiry the CTA raises an abort flag, keeps
+// its control flow (all barriers are still reached), touches no more data and reports GOQ_ERR_TIMEOUT.
+#include "goq_stream_core.cuh"
+#include "goq_internal.h"
+
+namespace goq {
+namespace seq {
+
+constexpr int kConsumerWarps = 16;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kStageUnits = kConsumerWarps;
+constexpr int kRedSlots = 2;
+constexpr int kXBufBytes = 22 * 1024 + 512;   // staged activations of one linear: batch * k_pad * 2 bytes
+constexpr int kGlobalSpin = 1 << 20;          // polls (with a short sleep) of a completion counter
+
+struct Item {
+    const uint8_t* packed;
+    const uint16_t* x;
+    void* y;
+    int n_tiles, k_blocks, k_in, n_out, m_total, y_dtype, depends, tile_base;
+};
+struct Params {
+    Item item[kSeqMaxItems];
+    int n_items, unit_bytes, n_stages;
+    int* status;
+    int* done;   // [n_items] CTAs that have finished each linear; zero on entry, left zero
+};
+
+__device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory"); }
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// first tile of linear `it` that belongs to CTA `cta` (tiles cta-congruent modulo the grid, numbered across linears)
+__device__ __forceinline__ int first_tile(const Item& it, int cta, int n_ctas) {
+    int r = (cta - it.tile_base) % n_ctas;
+    return r < 0 ? r + n_ctas : r;
+}
+
+#ifdef GOQ_TRACE
+__device__ unsigned long long g_seq_trace[512][8][8];   // [cta][item][event], warp 0 lane 0, SM cycle counter
+#define GOQ_ST(item, ev) do { if (threadIdx.x == 0 && (item) >= GOQ_TRI0 && (item) < GOQ_TRI0 + 8) { unsigned long long t_; \
+    asm volatile("mov.u64 %0, %%clock64;" : "=l"(t_) :: "memory"); g_seq_trace[blockIdx.x][(item) - GOQ_TRI0][ev] = t_; } } while (0)
+#else
+#define GOQ_ST(item, ev) do { } while (0)
+#endif
+#ifndef GOQ_TRI0
+#define GOQ_TRI0 0
+#endif
+
+template <int WB, int CPG>
+__global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_constant__ Params p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* lut = smem + ((8192u - (smem_u32(smem) & 8191u)) & 8191u);   // 8 KiB boundary: slot offsets are OR-ed in
+    const int stage_bytes = kStageUnits * p.unit_bytes;
+    unsigned char* ring = lut + kLutBytes;
+    float* red = reinterpret_cast<float*>(ring + (size_t)p.n_stages * stage_bytes);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(red + kRedSlots * kConsumerWarps * 32 * 4);
+    uint64_t* empty_bar = full_bar + p.n_stages;
+    uint64_t* x_bar = empty_bar + p.n_stages;
+    uint16_t* xs = reinterpret_cast<uint16_t*>(x_bar + 2);
+    __shared__ volatile int abort_flag;
+    __shared__ int arrive_cnt[kRedSlots];
+    __shared__ int done_gen[kRedSlots];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_ctas = (int)gridDim.x, cta = (int)blockIdx.x;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int i = 0; i < kRedSlots; ++i) { arrive_cnt[i] = 0; done_gen[i] = 0; }
+        for (int s = 0; s < p.n_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kConsumerWarps); }
+        mbar_init(x_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kConsumerWarps) {
+        // ---------------- producer: the weight stream of every tile this CTA owns, linear after linear ----------------
+        if (lane == 0) {
+            int slot = 0, round = 0;
+            bool ok = true;
+            for (int i = 0; i < p.n_items && ok; ++i) {
+                const Item& it = p.item[i];
+                for (int T = first_tile(it, cta, n_ctas); T < it.n_tiles && ok; T += n_ctas) {
+                    const uint8_t* src = it.packed + unit_offset(T, 0, it.k_blocks, p.unit_bytes);
+                    for (int u0 = 0; u0 < it.k_blocks; u0 += kStageUnits) {
+                        if (round > 0 && !mbar_wait_bounded(&empty_bar[slot], (round - 1) & 1, &abort_flag)) { ok = false; break; }
+                        const int units = min(kStageUnits, it.k_blocks - u0);
+                        const uint32_t bytes = (uint32_t)units * p.unit_bytes;
+                        mbar_arrive_expect_tx(&full_bar[slot], bytes);
+                        bulk_copy_g2s(ring + (size_t)slot * stage_bytes, src + (size_t)u0 * p.unit_bytes, bytes, &full_bar[slot]);
+                        if (++slot == p.n_stages) { slot = 0; ++round; }
+                    }
+                }
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers ----------------
+    for (int i = tid; i < 64 * kLutCopies; i += kConsumerWarps * 32) {
+        const uint32_t* e = c_exchange_lut.v[i / kLutCopies];
+        *reinterpret_cast<uint4*>(lut + (size_t)i * 16) = make_uint4(e[0], e[1], e[2], e[3]);
+    }
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t lut_lane = smem_u32(lut) + (lane & (kLutCopies - 1)) * 16;
+    int slot = 0, phase = 0;   // position in the stage ring
+    int n_tile_local = 0;      // tiles this CTA has finished (indexes the reduction slots)
+    uint32_t x_phase = 0;
+
+    for (int i = 0; i <= p.n_items; ++i) {
+        // ---- boundary between linear i-1 and linear i ----
+        GOQ_ST(i, 0);
+        consumer_bar_sync();   // every warp has finished linear i-1: outputs stored, activation buffer free
+        GOQ_ST(i, 1);
+        if (i == p.n_items) {
+            if (tid == 0 && i > 0) {
+                // the CTA that completes the last linear last leaves the counters zero for the next call
+                const int prev = atomic_add_acq_rel_gpu(&p.done[i - 1], 1);
+                if (prev == n_ctas - 1) for (int j = 0; j < p.n_items; ++j) p.done[j] = 0;
+            }
+            break;
+        }
+        const Item& it = p.item[i];
+        const int k_pad = it.k_blocks * kBlockK;
+        const int T0 = first_tile(it, cta, n_ctas);
+        const bool have_work = T0 < it.n_tiles;
+        if (tid == 0) {
+            if (i > 0) atomic_add_acq_rel_gpu(&p.done[i - 1], 1);   // releases this CTA's outputs (ordered by the barrier above)
+            if (have_work && abort_flag == 0) {
+                bool ok = true;
+                if (it.depends && i > 0) {   // the activations may be outputs of earlier linears: all CTAs must be done with them
+                    int spins = 0;
+                    while (ld_acquire_gpu(&p.done[i - 1]) < n_ctas) {
+                        if (abort_flag || ++spins > kGlobalSpin) { abort_flag = 1; ok = false; break; }
+                        __nanosleep(64);
+                    }
+                }
+                GOQ_ST(i, 2);
+                if (ok) {
+                    const uint32_t row_bytes = (uint32_t)it.k_in * 2;
+                    mbar_arrive_expect_tx(x_bar, row_bytes * it.m_total);
+                    for (int r = 0; r < it.m_total; ++r) bulk_copy_g2s(xs + (size_t)r * k_pad, it.x + (size_t)r * it.k_in, row_bytes, x_bar);
+                }
+            }
+        }
+        if (!have_work) continue;
+        {   // zero the padding [k_in, k_pad) of every staged activation row (the copies do not touch it)
+            const int tail = k_pad - it.k_in;
+            for (int j = tid; j < tail * it.m_total; j += kConsumerWarps * 32) xs[(size_t)(j / tail) * k_pad + it.k_in + (j % tail)] = 0;
+        }
+        consumer_bar_sync();
+        const bool x_ok = mbar_wait_bounded(x_bar, x_phase, &abort_flag);
+        GOQ_ST(i, 3);
+        x_phase ^= 1u;
+        // lanes whose token does not exist read the last token's row: an MMA output column depends only on its own
+        // B column, and columns of missing tokens are never stored
+        const uint32_t xrow_s = order_after_wait(smem_u32(xs) + (uint32_t)(min(g, it.m_total - 1) * k_pad + t * 8) * 2);
+
+        for (int T = T0; T < it.n_tiles; T += n_ctas) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int u0 = 0; u0 < it.k_blocks; u0 += kStageUnits) {
+                const int units = min(kStageUnits, it.k_blocks - u0);
+                if (mbar_wait_bounded(&full_bar[slot], phase, &abort_flag) && x_ok && warp < units) {
+                    const uint32_t unit = order_after_wait(smem_u32(ring) + slot * stage_bytes + warp * p.unit_bytes + lane * 16);
+                    const int kb0 = (u0 + warp) * kBlockK;
+                    const uint4 wv0 = lds128(unit), wv1 = lds128(unit + 512);
+                    const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
+                    const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
+                    float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint4 xa = lds128(xrow_s + (kb0 + c * 32) * 2);
+                        uint32_t R0[4], Q0[4], R1[4], Q1[4];
+                        expand_word<WB>(w0[c], lut_lane, R0, Q0);
+                        expand_word<WB>(w1[c], lut_lane, R1, Q1);
+                        mma_bf16(d1, R0[0], R1[0], R0[1], R1[1], xa.x, xa.y);
+                        mma_bf16(d2, Q0[0], Q1[0], Q0[1], Q1[1], xa.x, xa.y);
+                        mma_bf16(d1, R0[2], R1[2], R0[3], R1[3], xa.z, xa.w);
+                        mma_bf16(d2, Q0[2], Q1[2], Q0[3], Q1[3], xa.z, xa.w);
+                        if (((c + 1) % CPG) == 0) {   // end of a macro-block: the coefficient multiply, outside the inner product
+                            const int jj = c / CPG;
+                            const uint32_t cfa = lds32(coef_addr + jj * 64), cfb = lds32(coef_addr + jj * 64 + 32);
+                            const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
+                            const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
+                            const float c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
+                            const float c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
+                            acc[0] += c1a * d1[0] + c2a * d2[0];
+                            acc[1] += c1a * d1[1] + c2a * d2[1];
+                            acc[2] += c1b * d1[2] + c2b * d2[2];
+                            acc[3] += c1b * d1[3] + c2b * d2[3];
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) d1[r] = d2[r] = 0.f;
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[slot]);
+                if (++slot == p.n_stages) { slot = 0; phase ^= 1; }
+            }
+            GOQ_ST(i, 4 + min(3, (T - T0) / n_ctas));
+            // ---- park this warp's sums; the last warp of the tile adds them in warp order and stores ----
+            const int rs = n_tile_local % kRedSlots;
+            const int contributors = min(kConsumerWarps, it.k_blocks);
+            if (warp < contributors) {
+                bool ok = abort_flag == 0;
+                if (ok && n_tile_local >= kRedSlots) {   // the slot's previous tile must be fully reduced
+                    volatile int* dg = &done_gen[rs];
+                    int spins = 0;
+                    while (*dg != n_tile_local - kRedSlots + 1) {
+                        if (abort_flag || ++spins > kSpinLimit) { abort_flag = 1; ok = false; break; }
+                        __nanosleep(40);
+                    }
+                }
+                if (ok) {
+                    float* rb = red + (size_t)rs * kConsumerWarps * 32 * 4;
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) rb[(warp * 32 + lane) * 4 + r] = acc[r];
+                    __threadfence_block();
+                    __syncwarp();
+                    int old = 0;
+                    if (lane == 0) old = atomicAdd(&arrive_cnt[rs], 1);
+                    old = __shfl_sync(0xFFFFFFFFu, old, 0);
+                    if (old == contributors - 1) {
+                        __threadfence_block();
+                        float out[4] = {0.f, 0.f, 0.f, 0.f};
+                        for (int w = 0; w < contributors; ++w) {
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) out[r] += rb[(w * 32 + lane) * 4 + r];
+                        }
+                        if (abort_flag == 0) {
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) {
+                                const int row = T * 16 + g + ((r & 2) ? 8 : 0);
+                                const int tok = t * 2 + (r & 1);
+                                if (row < it.n_out && tok < it.m_total) {
+                                    if (it.y_dtype == GOQ_F32) reinterpret_cast<float*>(it.y)[(size_t)tok * it.n_out + row] = out[r];
+                                    else reinterpret_cast<uint16_t*>(it.y)[(size_t)tok * it.n_out + row] = f32_to_bf16_rne(out[r]);
+                                }
+                            }
+                        }
+                        __syncwarp();
+                        if (lane == 0) {
+                            arrive_cnt[rs] = 0;
+                            __threadfence_block();
+                            done_gen[rs] = n_tile_local + 1;
+                        }
+                    }
+                }
+            }
+            ++n_tile_local;
+        }
+    }
+    if (tid == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
+}
+
+}  // namespace seq
+}  // namespace goq
+
+// ---- host side -------------------------------------------------------------------------------------
+namespace goq {
+
+static int seq_sm_count() {
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    return n > 0 ? n : 148;
+}
+
+bool gemv_seq_supported(const Geometry& g, int m) {
+    return g.group >= 32 && g.wbits <= 3 && m >= 1 && m <= 8 && (size_t)m * g.k_pad * 2 <= (size_t)seq::kXBufBytes;
+}
+size_t gemv_seq_workspace(int n_items) { return 256 + (size_t)(n_items > 0 ? n_items : 0) * sizeof(int); }
+
+template <int WB, int CPG>
+static cudaError_t launch_seq_cfg(seq::Params& p, cudaStream_t st) {
+    auto kernel = seq::gemv_seq_kernel<WB, CPG>;
+    const int stage_bytes = seq::kStageUnits * p.unit_bytes;
+    p.n_stages = 3;
+    const size_t smem = (size_t)2 * kLutBytes + (size_t)p.n_stages * stage_bytes + (size_t)seq::kRedSlots * seq::kConsumerWarps * 32 * 4 * sizeof(float) +
+                        (size_t)(2 * p.n_stages + 2) * sizeof(uint64_t) + (size_t)seq::kXBufBytes;
+    static size_t attr_smem = 0;
+    static int per_sm = 0;
+    if (smem > attr_smem) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, seq::kThreads, smem);
+        if (e != cudaSuccess) return e;
+        attr_smem = smem;
+    }
+    if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+    long long total_tiles = 0;
+    for (int i = 0; i < p.n_items; ++i) total_tiles += p.item[i].n_tiles;
+    int grid = seq_sm_count() * (per_sm > 2 ? 2 : per_sm);   // every CTA must be resident: the completion counters are waited on
+    if ((long long)grid > total_tiles) grid = (int)total_tiles;
+    int base = 0;
+    for (int i = 0; i < p.n_items; ++i) {   // tiles are numbered across linears; tile number mod grid = owning CTA
+        p.item[i].tile_base = base;
+        base = (base + p.item[i].n_tiles) % grid;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(seq::kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
+cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, int unit_bytes, void* ws, cudaStream_t st) {
+    static thread_local seq::Params p;   // ~14 KB: kept off the stack
+    auto* wsb = (uint8_t*)ws;
+    p.n_items = n;
+    p.unit_bytes = unit_bytes;
+    p.status = (int*)wsb;
+    p.done = (int*)(wsb + 256);
+    for (int i = 0; i < n; ++i) {
+        seq::Item& it = p.item[i];
+        it.packed = (const uint8_t*)calls[i].packed;
+        it.x = (const uint16_t*)calls[i].x;
+        it.y = calls[i].y;
+        it.n_tiles = calls[i].g.n_tiles;
+        it.k_blocks = calls[i].g.k_blocks;
+        it.k_in = calls[i].g.k_in;
+        it.n_out = calls[i].g.n_out;
+        it.m_total = calls[i].m;
+        it.y_dtype = calls[i].y_dtype;
+        it.depends = calls[i].depends;
+        it.tile_base = 0;
+    }
+    const int cpg = group / 32;
+    if (wbits == 3) return cpg == 1 ? launch_seq_cfg<3, 1>(p, st) : cpg == 2 ? launch_seq_cfg<3, 2>(p, st) : launch_seq_cfg<3, 4>(p, st);
+    return cpg == 1 ? launch_seq_cfg<2, 1>(p, st) : cpg == 2 ? launch_seq_cfg<2, 2>(p, st) : launch_seq_cfg<2, 4>(p, st);
+}
+
+}  // namespace goq

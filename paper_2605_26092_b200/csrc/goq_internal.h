@@ -34,6 +34,21 @@ size_t gemv_tc_workspace(const Geometry& g);
 cudaError_t launch_gemv_tc(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y, int y_dtype,
                            void* ws, cudaStream_t st);
 
+// A sequence of decode GEMVs in one persistent cooperative kernel (group >= 32, wbits <= 3, batch <= 8, the staged
+// activations of each linear fit in shared memory; every linear has the same wbits and group). `ws` holds
+// gemv_seq_workspace(n) bytes, zero on entry, left zero on return.
+constexpr int kSeqMaxItems = 256;
+struct SeqCall {
+    Geometry g;
+    const void* packed;
+    const void* x;
+    void* y;
+    int m, y_dtype, depends;
+};
+bool gemv_seq_supported(const Geometry& g, int m);
+size_t gemv_seq_workspace(int n_items);
+cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, int unit_bytes, void* ws, cudaStream_t st);
+
 // Prefill GEMM on tcgen05 tensor cores (wbits <= 3). `ws` holds gemm_tc_workspace(g) bytes (status word).
 bool gemm_tc_supported(const Geometry& g);
 size_t gemm_tc_workspace(const Geometry& g);

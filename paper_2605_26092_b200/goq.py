@@ -22,7 +22,8 @@ LAYOUT_TILE16 = 1
 EXPORTS = (
     "goq_status_string", "goq_packed_bytes", "goq_algorithmic_bytes", "goq_workspace_bytes", "goq_pack",
     "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant", "goq_workspace_init",
-    "goq_workspace_status", "goq_gemv_static", "goq_last_cuda_error",
+    "goq_workspace_status", "goq_gemv_static", "goq_last_cuda_error", "goq_sequence_workspace_bytes",
+    "goq_gemv_sequence",
 )
 
 
@@ -35,6 +36,11 @@ class GoqError(RuntimeError):
 
 class Desc(Structure):
     _fields_ = [("n_out", c_int32), ("k_in", c_int32), ("group", c_int32), ("wbits", c_int32), ("layout", c_int32)]
+
+
+class GemvItem(Structure):
+    _fields_ = [("desc", Desc), ("packed", c_void_p), ("x_bf16", c_void_p), ("y", c_void_p), ("batch", c_int32),
+                ("y_dtype", c_int32), ("depends", c_int32)]
 
 
 _lib = None
@@ -74,6 +80,10 @@ def lib() -> ctypes.CDLL:
         L.goq_gemv_static.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p]
         L.goq_last_cuda_error.restype = c_int
         L.goq_last_cuda_error.argtypes = []
+        L.goq_sequence_workspace_bytes.restype = ctypes.c_size_t
+        L.goq_sequence_workspace_bytes.argtypes = [c_int]
+        L.goq_gemv_sequence.restype = c_int
+        L.goq_gemv_sequence.argtypes = [POINTER(GemvItem), c_int, c_void_p, ctypes.c_size_t, c_void_p]
         L.goq_set_gemv_variant.restype = c_int
         L.goq_set_gemv_variant.argtypes = [c_int]
         _lib = L
@@ -162,6 +172,28 @@ def gemv_static(d: Desc, packed, x_bf16, batch: int, y, y_dtype: int, stream=Non
     For callers that cannot allocate device memory; calls that may overlap on the GPU must not share it."""
     _check(lib().goq_gemv_static(ctypes.byref(d), _ptr(packed), _ptr(x_bf16), batch, _ptr(y), y_dtype,
                                  _stream(stream)), "goq_gemv_static")
+
+
+def sequence_workspace_bytes(n_items: int) -> int:
+    return lib().goq_sequence_workspace_bytes(n_items)
+
+
+def make_sequence(items):
+    """items: iterable of (desc, packed, x_bf16, batch, y, y_dtype, depends). Returns the ctypes array
+    goq_gemv_sequence takes (it holds raw device pointers: keep the tensors alive)."""
+    items = list(items)
+    arr = (GemvItem * len(items))()
+    for a, (d, packed, x, batch, y, y_dtype, depends) in zip(arr, items):
+        a.desc = d
+        a.packed, a.x_bf16, a.y = _ptr(packed), _ptr(x), _ptr(y)
+        a.batch, a.y_dtype, a.depends = batch, y_dtype, 1 if depends else 0
+    return arr
+
+
+def gemv_sequence(seq, ws, stream=None):
+    """goq_gemv_sequence: a chain of decode GEMVs in one persistent kernel. `seq` comes from make_sequence."""
+    _check(lib().goq_gemv_sequence(seq, len(seq), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
+           "goq_gemv_sequence")
 
 
 def gemm(d: Desc, packed, x, m: int, x_dtype: int, y=None, y_dtype: int = F32, sx=None, cq=None, sc=None,

@@ -1,0 +1,138 @@
+"""goq_gemv_sequence: a chain of decode GEMVs in one persistent kernel, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import synth_inputs as si
+from oracle import goq_oracle as O
+
+pytestmark = pytest.mark.gpu
+TIGHT = 2e-5
+
+
+@pytest.fixture(scope="module")
+def goq():
+    from paper_2605_26092_b200 import build
+    build.build()
+    from paper_2605_26092_b200 import goq as g
+    g.lib()
+    assert torch.cuda.is_available()
+    return g
+
+
+def _layer(goq, n, k, g, b, seed):
+    from tests.gpu_util import pack_weights
+    codes, meta, coef = si.random_quantized(n, k, g, b, seed=seed)
+    d, packed = pack_weights(n, k, g, b, codes, meta, coef)
+    return dict(n=n, k=k, g=g, b=b, codes=codes, meta=meta, coef=coef, d=d, packed=packed)
+
+
+def _ws(goq, n_items):
+    ws = torch.empty(goq.sequence_workspace_bytes(n_items), dtype=torch.uint8, device="cuda")
+    goq.workspace_init(ws)
+    return ws
+
+
+def test_chain_with_real_dependencies_matches_oracle_stage_by_stage(goq):
+    """y0 = W0 x0 (bf16 out) feeds W1, whose bf16 output feeds W2: every stage is checked against the oracle
+    evaluated on the bits the previous stage actually produced."""
+    from tests.gpu_util import dev
+    batch = 3
+    shapes = [(256, 384), (512, 256), (130, 512)]   # (n_out, k_in): n_out of one = k_in of the next
+    layers = [_layer(goq, n, k, 64, 3, seed=40 + i) for i, (n, k) in enumerate(shapes)]
+    x0 = si.bf16_activations(batch, shapes[0][1], seed=5)
+    bufs = [dev(x0)] + [torch.zeros((batch, n), dtype=torch.bfloat16, device="cuda") for n, _ in shapes[:-1]]
+    y_last = torch.zeros((batch, shapes[-1][0]), dtype=torch.float32, device="cuda")
+    outs = bufs[1:] + [y_last]
+    items = [(L["d"], L["packed"], bufs[i], batch, outs[i], goq.BF16 if i < 2 else goq.F32, i > 0)
+             for i, L in enumerate(layers)]
+    seq = goq.make_sequence(items)
+    ws = _ws(goq, len(items))
+    for _ in range(2):   # the scratch is left clean: a second call needs no re-initialisation
+        goq.gemv_sequence(seq, ws)
+        torch.cuda.synchronize()
+        assert goq.workspace_status(ws) == goq.OK
+        x_bits = x0
+        for i, L in enumerate(layers):
+            y_ref = O.linear_f64(L["codes"], L["meta"], L["coef"], si.bf16_bits_to_f64(x_bits), L["g"], L["b"])
+            got = outs[i].float().cpu().numpy().astype(np.float64)
+            tol = TIGHT if i == 2 else 4e-3   # bf16 outputs carry one extra rounding
+            assert O.normwise_rel_err(got, y_ref) <= tol, (i, O.normwise_rel_err(got, y_ref))
+            if i < 2:
+                x_bits = outs[i].view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("g,b", [(128, 3), (32, 2)])
+def test_independent_items_of_mixed_shapes(goq, g, b):
+    """Ragged rows and k, fewer and more than 16 k-blocks per tile, batch 1..8, both output types."""
+    from tests.gpu_util import dev
+    shapes = [(40, 256, 1), (300, 4224, 2), (16, 128, 8), (1000, 1152, 5), (257, 2048 + 128, 3)]
+    layers, xs, ys, items = [], [], [], []
+    for i, (n, k, m) in enumerate(shapes):
+        L = _layer(goq, n, k, g, b, seed=90 + i)
+        xb = si.bf16_activations(m, k, seed=60 + i)
+        y = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda")
+        layers.append(L); xs.append(xb); ys.append(y)
+        items.append((L["d"], L["packed"], dev(xb), m, y, goq.F32, False))
+    keep = [it[2] for it in items]
+    seq = goq.make_sequence(items)
+    ws = _ws(goq, len(items))
+    goq.gemv_sequence(seq, ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    first = [y.clone() for y in ys]
+    for L, xb, y in zip(layers, xs, ys):
+        y_ref = O.linear_f64(L["codes"], L["meta"], L["coef"], si.bf16_bits_to_f64(xb), g, b)
+        err = O.normwise_rel_err(y.cpu().numpy().astype(np.float64), y_ref)
+        assert err <= TIGHT, err
+    goq.gemv_sequence(seq, ws)
+    torch.cuda.synchronize()
+    for a, y in zip(first, ys):
+        assert torch.equal(a, y)   # same sums in the same order: bit-identical
+    del keep
+
+
+def test_one_7b_shaped_layer_sampled_rows(goq):
+    from tests.gpu_util import dev
+    items, checks = [], []
+    for i, (name, n, k) in enumerate(si.LLAMA2_7B_LINEARS):
+        codes, meta, coef = si.random_quantized(n, k, 128, 3, seed=300 + i)
+        rows = si.sample_rows(n, 32, seed=i)
+        w = si.weights_with_outlier_channels(len(rows), k, seed=i)
+        codes[rows], meta[rows], coef[rows] = O.quantize_geo(w, 128, 3)
+        from tests.gpu_util import pack_weights
+        d, packed = pack_weights(n, k, 128, 3, codes, meta, coef)
+        xb = si.bf16_activations(1, k, seed=200 + i)
+        y = torch.zeros((1, n), dtype=torch.float32, device="cuda")
+        items.append((d, packed, dev(xb), 1, y, goq.F32, True))
+        checks.append((codes, meta, coef, xb, rows, y))
+    seq = goq.make_sequence(items)
+    ws = _ws(goq, len(items))
+    goq.gemv_sequence(seq, ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    for codes, meta, coef, xb, rows, y in checks:
+        y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 128, 3, rows=rows)
+        assert O.normwise_rel_err(y.cpu().numpy().astype(np.float64)[:, rows], y_ref) <= TIGHT
+
+
+def test_unsupported_and_invalid_sequences_return_a_status(goq):
+    from tests.gpu_util import dev
+    L = _layer(goq, 64, 256, 64, 3, seed=1)
+    L2 = _layer(goq, 64, 256, 128, 3, seed=2)
+    ws = _ws(goq, 2)
+    x9 = dev(si.bf16_activations(9, 256, seed=1))
+    y9 = torch.zeros((9, 64), dtype=torch.float32, device="cuda")
+    with pytest.raises(goq.GoqError) as e:
+        goq.gemv_sequence(goq.make_sequence([(L["d"], L["packed"], x9, 9, y9, goq.F32, False)]), ws)
+    assert e.value.status == goq.ERR_UNSUPPORTED
+    x1 = dev(si.bf16_activations(1, 256, seed=1))
+    y1 = torch.zeros((1, 64), dtype=torch.float32, device="cuda")
+    mixed = [(L["d"], L["packed"], x1, 1, y1, goq.F32, False), (L2["d"], L2["packed"], x1, 1, y1, goq.F32, True)]
+    with pytest.raises(goq.GoqError) as e:
+        goq.gemv_sequence(goq.make_sequence(mixed), ws)
+    assert e.value.status == goq.ERR_UNSUPPORTED
+    small = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(goq.GoqError) as e:
+        goq.gemv_sequence(goq.make_sequence(mixed[:1] * 2), small)
+    assert e.value.status == goq.ERR_WORKSPACE
