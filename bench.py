@@ -496,7 +496,7 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
 
 
 NCU_TRAFFIC_RATIO = 8.96 / 8.39
-NCU_TRAFFIC_RATIO_SEQ = None   # dram bytes / algorithmic bytes of the sequence kernel, from its ncu capture
+NCU_TRAFFIC_RATIO_SEQ = 215.3 / 202.9   # ncu: 215.3 MB of DRAM reads for the 202.9 MB (algorithmic) of a 14-linear launch
 
 
 def main():
