@@ -10,6 +10,7 @@ using goq::Geometry;
 namespace {
 
 std::atomic<int> g_gemv_variant{0};
+constexpr int kGemmViaGemvMaxTokens = 64;
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -78,7 +79,12 @@ size_t goq_workspace_bytes(const goq_desc* desc, int op, int m) {
         if (goq::gemv_tc_supported(g, m) && goq::gemv_tc_workspace(g) > need) need = goq::gemv_tc_workspace(g);
         return need;
     }
-    if (op == GOQ_OP_GEMM && goq::gemm_tc_supported(g)) return goq::gemm_tc_workspace(g);
+    if (op == GOQ_OP_GEMM) {
+        size_t need = goq::gemm_tc_supported(g) ? goq::gemm_tc_workspace(g) : 0;
+        if (m <= kGemmViaGemvMaxTokens && goq::gemv_stream_supported(g) && goq::gemv_stream_workspace(g) > need)
+            need = goq::gemv_stream_workspace(g);
+        return need;
+    }
     return 0;
 }
 
@@ -149,6 +155,22 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
         if (!y) return GOQ_ERR_INVALID_ARG;
         if (goq_status s = check_arch()) return s;
         const int variant = g_gemv_variant.load(std::memory_order_relaxed);
+        // Few tokens (17..64): the streaming GEMV kernel, 16 tokens per launch, is several times faster than a
+        // 128 x 512 tensor-core tile that would be mostly padding (measured crossover on 8192 x 8192: ~80 tokens).
+        if (m <= kGemmViaGemvMaxTokens && variant == 0 && goq::gemv_stream_supported(g)) {
+            if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
+            if (ws_bytes < goq::gemv_stream_workspace(g)) return GOQ_ERR_WORKSPACE;
+            if (!goq::stream_hash_is_bijective()) return GOQ_ERR_UNSUPPORTED;
+            const size_t ybytes = (y_dtype == GOQ_F32) ? 4 : 2;
+            for (int t0 = 0; t0 < m; t0 += 16) {
+                const int nb = (m - t0 < 16) ? (m - t0) : 16;
+                cudaError_t e = goq::launch_gemv_stream(g, packed, (const uint16_t*)x + (size_t)t0 * g.k_in, nb,
+                                                        (uint8_t*)y + (size_t)t0 * g.n_out * ybytes, y_dtype, ws,
+                                                        (cudaStream_t)stream);
+                if (e != cudaSuccess) return from_cuda(e);
+            }
+            return GOQ_OK;
+        }
         if (goq::gemm_tc_supported(g) && variant != 2) {
             if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
             if (ws_bytes < goq::gemm_tc_workspace(g)) return GOQ_ERR_WORKSPACE;
