@@ -168,7 +168,10 @@ goq_status goq_gemv_static(const goq_desc* desc, const void* packed, const void*
 /* goq_gemv_sequence: a chain of decode GEMVs (Eq. 4, one call of goq_gemv each) executed by ONE persistent
  * cooperative kernel, in order. Results are those of calling goq_gemv item by item on one stream; what changes
  * is the cost: no launch, prologue or first-byte latency per linear, and the weight stream never stops at a
- * boundary between linears.
+ * boundary between linears. When every item has batch <= 4 the kernel computes with integer operands: the
+ * activations of each token and 128-wide k-block become 16-bit fixed point (exact for every element within 2^-7 of
+ * the block's largest magnitude, rounded at 2^-15 of it below; measured normwise error ~1e-5 or less), and
+ * non-finite activations are not propagated (they saturate). Otherwise bf16 operands, exact products.
  *   items    HOST array of n_items entries (read during the call, not kept):
  *            desc, packed, x_bf16 [batch][k_in], y [batch][n_out], y_dtype as in goq_gemv, all device pointers;
  *            depends != 0 : this item's x (or y) may alias outputs of EARLIER items of the sequence - the kernel
@@ -199,7 +202,8 @@ int goq_last_cuda_error(void);
 
 /* Force a kernel variant (benchmarks and tests only): 0 = automatic, 1 = scalar exponent-add
  * kernel, 2 = tensor-core fragment kernel, 3 = streaming tensor-core kernel, 4 = tcgen05 kernel with
- * the FP8 weight operand in tensor memory. Process-wide.
+ * the FP8 weight operand in tensor memory, 5 = goq_gemv_sequence always with bf16 operands (it uses integer
+ * operands when every item has batch <= 4). Process-wide.
  * Returns the previous value. */
 int goq_set_gemv_variant(int variant);
 

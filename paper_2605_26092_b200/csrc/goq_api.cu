@@ -226,6 +226,7 @@ goq_status goq_gemv_sequence(const goq_gemv_item* items, int n_items, void* ws, 
     if (ws_bytes < goq::gemv_seq_workspace(n_items)) return GOQ_ERR_WORKSPACE;
     if (goq_status s = check_arch()) return s;
     if (!goq::stream_hash_is_bijective()) return GOQ_ERR_UNSUPPORTED;
+    goq::g_seq_int8 = g_gemv_variant.load(std::memory_order_relaxed) != 5;
     for (int i0 = 0; i0 < n_items; i0 += goq::kSeqMaxItems) {
         const int n = (n_items - i0 < goq::kSeqMaxItems) ? (n_items - i0) : goq::kSeqMaxItems;
         // a chunk boundary is a kernel boundary on the stream: the first item of a chunk needs no counter wait

@@ -28,6 +28,7 @@ constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kStageUnits = kConsumerWarps;
 constexpr int kRedSlots = 2;
 constexpr int kXBufBytes = 22 * 1024 + 512;   // staged activations of one linear: batch * k_pad * 2 bytes
+constexpr int kScaleFloats = 96 * 4;           // (integer form) one 2^-s per k-block and token: k_blocks <= 90, batch <= 4
 constexpr int kGlobalSpin = 1 << 20;          // polls (with a short sleep) of a completion counter
 
 struct Item {
@@ -50,6 +51,45 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
     return v;
 }
 
+// ---- integer operands (batch <= 4) -------------------------------------------------------------------
+// Every PoT state times 2^emax is a small integer, so b1 and b2 can feed the int8 tensor-core MMA as bytes
+// straight out of the byte-table lookup: no 16-bit operand registers to assemble (the largest share of the
+// logic-pipe work of the bf16 form), and half as many MMAs (k = 32). The activations are made integers too:
+// per token and 128-wide k-block, Q = rne(x * 2^s) with s chosen so that the block's largest magnitude lands in
+// [2^14, 2^15), split as Q = 256 q0 + q1 into two int8 rows of the B operand (columns 2t and 2t+1 of token t).
+// bf16 has 8 significant bits, so Q is exact for every element within 2^-7 of the block's largest; smaller ones
+// are rounded at 2^-15 of it. Integer sums are exact; 256 S0 + S1 is formed in int32 and converted once.
+template <int WB> struct IntTables;
+template <> struct IntTables<3> {  // codes 0..7 -> 8 4 2 0 -8 -4 -2 -1 and the negated table
+    static constexpr uint32_t P0 = 0x00020408u, P1 = 0xFFFEFCF8u, N0 = 0x00FEFCF8u, N1 = 0x01020408u;
+};
+template <> struct IntTables<2> {  // codes 0..3 -> 2 0 -2 -1
+    static constexpr uint32_t P0 = 0xFFFE0002u, P1 = 0u, N0 = 0x010200FEu, N1 = 0u;
+};
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// The record table holds sign-bit masks (bit 7 of each flipped byte); (mask >> 7) * 255 makes them byte masks.
+__device__ __forceinline__ uint32_t byte_mask(uint32_t sign_bits) { return (sign_bits >> 7) * 255u; }
+// one micro-block word -> b1 bytes (pa: weights 0..3, pb: 4..7) and b2 bytes, as int8 = value * 2^emax
+template <int WB>
+__device__ __forceinline__ void decode_i8(uint32_t w, uint32_t lut_lane, uint32_t& pa, uint32_t& pb, uint32_t& qa, uint32_t& qb) {
+    const uint32_t m = w & 0x77777777u, mh = m >> 16;
+    pa = prmt_b32(IntTables<WB>::P0, IntTables<WB>::P1, m);
+    pb = prmt_b32(IntTables<WB>::P0, IntTables<WB>::P1, mh);
+    const uint32_t na = prmt_b32(IntTables<WB>::N0, IntTables<WB>::N1, m), nb = prmt_b32(IntTables<WB>::N0, IntTables<WB>::N1, mh);
+    const uint32_t h = (w - m) * kHashMul;
+    const uint4 e = lds128(((h >> 19) & 0x1F80u) | lut_lane);   // selectors x, y; byte masks of the flipped positions z, w
+    qa = (prmt_b32(pa, pb, e.x) & ~e.z) | (prmt_b32(na, nb, e.x) & e.z);   // a flipped zero stays zero
+    qb = (prmt_b32(pa, pb, e.y) & ~e.w) | (prmt_b32(na, nb, e.y) & e.w);
+}
+
 // first tile of linear `it` that belongs to CTA `cta` (tiles cta-congruent modulo the grid, numbered across linears)
 __device__ __forceinline__ int first_tile(const Item& it, int cta, int n_ctas) {
     int r = (cta - it.tile_base) % n_ctas;
@@ -67,7 +107,7 @@ __device__ unsigned long long g_seq_trace[512][8][8];   // [cta][item][event], w
 #define GOQ_TRI0 0
 #endif
 
-template <int WB, int CPG>
+template <int WB, int CPG, bool I8>
 __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_constant__ Params p) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* lut = smem + ((8192u - (smem_u32(smem) & 8191u)) & 8191u);   // 8 KiB boundary: slot offsets are OR-ed in
@@ -77,7 +117,8 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(red + kRedSlots * kConsumerWarps * 32 * 4);
     uint64_t* empty_bar = full_bar + p.n_stages;
     uint64_t* x_bar = empty_bar + p.n_stages;
-    uint16_t* xs = reinterpret_cast<uint16_t*>(x_bar + 2);
+    uint16_t* xs = reinterpret_cast<uint16_t*>(x_bar + 2);   // bf16 rows, or (I8) int8 rows 2*token + slice
+    float* xscale = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(xs) + kXBufBytes);   // (I8) [k-block][4 tokens]
     __shared__ volatile int abort_flag;
     __shared__ int arrive_cnt[kRedSlots];
     __shared__ int done_gen[kRedSlots];
@@ -120,7 +161,8 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
     // ---------------- consumers ----------------
     for (int i = tid; i < 64 * kLutCopies; i += kConsumerWarps * 32) {
         const uint32_t* e = c_exchange_lut.v[i / kLutCopies];
-        *reinterpret_cast<uint4*>(lut + (size_t)i * 16) = make_uint4(e[0], e[1], e[2], e[3]);
+        *reinterpret_cast<uint4*>(lut + (size_t)i * 16) =
+            I8 ? make_uint4(e[0], e[1], byte_mask(e[2]), byte_mask(e[3])) : make_uint4(e[0], e[1], e[2], e[3]);
     }
     const int g = lane >> 2, t = lane & 3;
     const uint32_t lut_lane = smem_u32(lut) + (lane & (kLutCopies - 1)) * 16;
@@ -157,25 +199,68 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
                     }
                 }
                 GOQ_ST(i, 2);
-                if (ok) {
+                if (ok && !I8) {
                     const uint32_t row_bytes = (uint32_t)it.k_in * 2;
                     mbar_arrive_expect_tx(x_bar, row_bytes * it.m_total);
                     for (int r = 0; r < it.m_total; ++r) bulk_copy_g2s(xs + (size_t)r * k_pad, it.x + (size_t)r * it.k_in, row_bytes, x_bar);
                 }
             }
+            if (I8 && have_work) mbar_arrive(x_bar);   // the activations may be read now (or the CTA has given up)
         }
         if (!have_work) continue;
-        {   // zero the padding [k_in, k_pad) of every staged activation row (the copies do not touch it)
-            const int tail = k_pad - it.k_in;
-            for (int j = tid; j < tail * it.m_total; j += kConsumerWarps * 32) xs[(size_t)(j / tail) * k_pad + it.k_in + (j % tail)] = 0;
+        bool x_ok;
+        if constexpr (I8) {
+            // ---- fetch the activations and make them integers (see above): 16-byte chunks of 8 bf16, 16 chunks = one k-block ----
+            x_ok = mbar_wait_bounded(x_bar, x_phase, &abort_flag) && abort_flag == 0;
+            unsigned char* xb = reinterpret_cast<unsigned char*>(xs);
+            const int cpt = k_pad / 8, total = cpt * it.m_total;
+            for (int c0 = warp * 32; c0 < total; c0 += kConsumerWarps * 32) {
+                const int c = c0 + lane;
+                const bool in = c < total;
+                const int r = in ? c / cpt : 0, k0 = in ? (c - r * cpt) * 8 : 0;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (in && x_ok && k0 < it.k_in) v = __ldcg(reinterpret_cast<const uint4*>(it.x + (size_t)r * it.k_in + k0));   // L2: written by other SMs
+                const uint32_t in32[4] = {v.x, v.y, v.z, v.w};
+                uint32_t amax = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) amax = max(amax, max(in32[j] & 0x7FFFu, (in32[j] >> 16) & 0x7FFFu));
+#pragma unroll
+                for (int o = 1; o < 16; o <<= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+                int sfield = 268 - (int)(amax >> 7);   // 2^s: the block's largest magnitude lands in [2^14, 2^15)
+                sfield = sfield < 1 ? 1 : (sfield > 253 ? 253 : sfield);
+                const float mult = __uint_as_float((uint32_t)sfield << 23);
+                uint32_t q0[2] = {0u, 0u}, q1[2] = {0u, 0u};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t bits = (j & 1) ? (in32[j >> 1] & 0xFFFF0000u) : (in32[j >> 1] << 16);
+                    int Q = __float2int_rn(__uint_as_float(bits) * mult);
+                    Q = max(-32639, min(32639, Q));
+                    const int lo = ((Q + 128) & 255) - 128, hi = (Q - lo) >> 8;   // Q = 256 hi + lo, both int8
+                    q0[j >> 2] |= (uint32_t)(hi & 255) << (8 * (j & 3));
+                    q1[j >> 2] |= (uint32_t)(lo & 255) << (8 * (j & 3));
+                }
+                if (in) {
+                    *reinterpret_cast<uint2*>(xb + (size_t)(2 * r) * k_pad + k0) = make_uint2(q0[0], q0[1]);
+                    *reinterpret_cast<uint2*>(xb + (size_t)(2 * r + 1) * k_pad + k0) = make_uint2(q1[0], q1[1]);
+                    // 2^-s, and 2^-emax for the integer weights
+                    if ((lane & 15) == 0) xscale[(k0 >> 7) * 4 + r] = __uint_as_float((uint32_t)(254 - sfield) << 23) * (1.0f / (float)(1 << ((1 << (WB - 1)) - 1)));
+                }
+            }
+            consumer_bar_sync();
+        } else {
+            {   // zero the padding [k_in, k_pad) of every staged activation row (the copies do not touch it)
+                const int tail = k_pad - it.k_in;
+                for (int j = tid; j < tail * it.m_total; j += kConsumerWarps * 32) xs[(size_t)(j / tail) * k_pad + it.k_in + (j % tail)] = 0;
+            }
+            consumer_bar_sync();
+            x_ok = mbar_wait_bounded(x_bar, x_phase, &abort_flag);
         }
-        consumer_bar_sync();
-        const bool x_ok = mbar_wait_bounded(x_bar, x_phase, &abort_flag);
         GOQ_ST(i, 3);
         x_phase ^= 1u;
         // lanes whose token does not exist read the last token's row: an MMA output column depends only on its own
         // B column, and columns of missing tokens are never stored
-        const uint32_t xrow_s = order_after_wait(smem_u32(xs) + (uint32_t)(min(g, it.m_total - 1) * k_pad + t * 8) * 2);
+        const uint32_t xrow_s = I8 ? order_after_wait(smem_u32(xs) + (uint32_t)(min(g, 2 * it.m_total - 1) * k_pad + t * 8))
+                                   : order_after_wait(smem_u32(xs) + (uint32_t)(min(g, it.m_total - 1) * k_pad + t * 8) * 2);
 
         for (int T = T0; T < it.n_tiles; T += n_ctas) {
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -187,30 +272,61 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
                     const uint4 wv0 = lds128(unit), wv1 = lds128(unit + 512);
                     const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
                     const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
-                    float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f};
+                    if constexpr (I8) {
+                        int s1[4] = {0, 0, 0, 0}, s2[4] = {0, 0, 0, 0};
+                        float rec0 = 0.f, rec2 = 0.f;   // this record's sums for token t: row g, row g+8
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const uint4 xa = lds128(xrow_s + (kb0 + c * 32) * 2);
-                        uint32_t R0[4], Q0[4], R1[4], Q1[4];
-                        expand_word<WB>(w0[c], lut_lane, R0, Q0);
-                        expand_word<WB>(w1[c], lut_lane, R1, Q1);
-                        mma_bf16(d1, R0[0], R1[0], R0[1], R1[1], xa.x, xa.y);
-                        mma_bf16(d2, Q0[0], Q1[0], Q0[1], Q1[1], xa.x, xa.y);
-                        mma_bf16(d1, R0[2], R1[2], R0[3], R1[3], xa.z, xa.w);
-                        mma_bf16(d2, Q0[2], Q1[2], Q0[3], Q1[3], xa.z, xa.w);
-                        if (((c + 1) % CPG) == 0) {   // end of a macro-block: the coefficient multiply, outside the inner product
-                            const int jj = c / CPG;
-                            const uint32_t cfa = lds32(coef_addr + jj * 64), cfb = lds32(coef_addr + jj * 64 + 32);
-                            const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
-                            const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
-                            const float c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
-                            const float c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
-                            acc[0] += c1a * d1[0] + c2a * d2[0];
-                            acc[1] += c1a * d1[1] + c2a * d2[1];
-                            acc[2] += c1b * d1[2] + c2b * d2[2];
-                            acc[3] += c1b * d1[3] + c2b * d2[3];
+                        for (int c = 0; c < 4; ++c) {
+                            const uint2 xb = lds64(xrow_s + kb0 + c * 32);
+                            uint32_t pa0, pb0, qa0, qb0, pa1, pb1, qa1, qb1;
+                            decode_i8<WB>(w0[c], lut_lane, pa0, pb0, qa0, qb0);
+                            decode_i8<WB>(w1[c], lut_lane, pa1, pb1, qa1, qb1);
+                            // A fragment: a0/a1 = bytes k 0..3 of the micro-block for rows g / g+8, a2/a3 = bytes 4..7
+                            mma_s8(s1, pa0, pa1, pb0, pb1, xb.x, xb.y);
+                            mma_s8(s2, qa0, qa1, qb0, qb1, xb.x, xb.y);
+                            if (((c + 1) % CPG) == 0) {   // end of a macro-block: the coefficient multiply, outside the inner product
+                                const int jj = c / CPG;
+                                const uint32_t cfa = lds32(coef_addr + jj * 64), cfb = lds32(coef_addr + jj * 64 + 32);
+                                const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
+                                const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
+                                const float c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
+                                const float c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
+                                // columns 2t, 2t+1 hold the high and low activation slices of token t: S = 256 S_hi + S_lo, exact in int32
+                                rec0 += c1a * (float)(s1[0] * 256 + s1[1]) + c2a * (float)(s2[0] * 256 + s2[1]);
+                                rec2 += c1b * (float)(s1[2] * 256 + s1[3]) + c2b * (float)(s2[2] * 256 + s2[3]);
 #pragma unroll
-                            for (int r = 0; r < 4; ++r) d1[r] = d2[r] = 0.f;
+                                for (int r = 0; r < 4; ++r) s1[r] = s2[r] = 0;
+                            }
+                        }
+                        const float sv = xscale[(u0 + warp) * 4 + (t < it.m_total ? t : 0)];   // undo the activation scale of this k-block
+                        acc[0] = fmaf(sv, rec0, acc[0]);
+                        acc[2] = fmaf(sv, rec2, acc[2]);
+                    } else {
+                        float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f};
+    #pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const uint4 xa = lds128(xrow_s + (kb0 + c * 32) * 2);
+                            uint32_t R0[4], Q0[4], R1[4], Q1[4];
+                            expand_word<WB>(w0[c], lut_lane, R0, Q0);
+                            expand_word<WB>(w1[c], lut_lane, R1, Q1);
+                            mma_bf16(d1, R0[0], R1[0], R0[1], R1[1], xa.x, xa.y);
+                            mma_bf16(d2, Q0[0], Q1[0], Q0[1], Q1[1], xa.x, xa.y);
+                            mma_bf16(d1, R0[2], R1[2], R0[3], R1[3], xa.z, xa.w);
+                            mma_bf16(d2, Q0[2], Q1[2], Q0[3], Q1[3], xa.z, xa.w);
+                            if (((c + 1) % CPG) == 0) {   // end of a macro-block: the coefficient multiply, outside the inner product
+                                const int jj = c / CPG;
+                                const uint32_t cfa = lds32(coef_addr + jj * 64), cfb = lds32(coef_addr + jj * 64 + 32);
+                                const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
+                                const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
+                                const float c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
+                                const float c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
+                                acc[0] += c1a * d1[0] + c2a * d2[0];
+                                acc[1] += c1a * d1[1] + c2a * d2[1];
+                                acc[2] += c1b * d1[2] + c2b * d2[2];
+                                acc[3] += c1b * d1[3] + c2b * d2[3];
+    #pragma unroll
+                                for (int r = 0; r < 4; ++r) d1[r] = d2[r] = 0.f;
+                            }
                         }
                     }
                 }
@@ -252,8 +368,8 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
 #pragma unroll
                             for (int r = 0; r < 4; ++r) {
                                 const int row = T * 16 + g + ((r & 2) ? 8 : 0);
-                                const int tok = t * 2 + (r & 1);
-                                if (row < it.n_out && tok < it.m_total) {
+                                const int tok = I8 ? t : t * 2 + (r & 1);   // (I8) one token per lane, in elements 0 and 2
+                                if (row < it.n_out && tok < it.m_total && !(I8 && (r & 1))) {
                                     if (it.y_dtype == GOQ_F32) reinterpret_cast<float*>(it.y)[(size_t)tok * it.n_out + row] = out[r];
                                     else reinterpret_cast<uint16_t*>(it.y)[(size_t)tok * it.n_out + row] = f32_to_bf16_rne(out[r]);
                                 }
@@ -280,6 +396,8 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
 // ---- host side -------------------------------------------------------------------------------------
 namespace goq {
 
+bool g_seq_int8 = true;   // integer operands for sequences whose items all have batch <= 4 (tests force both forms)
+
 static int seq_sm_count() {
     int dev = 0, n = 0;
     cudaGetDevice(&dev);
@@ -292,13 +410,13 @@ bool gemv_seq_supported(const Geometry& g, int m) {
 }
 size_t gemv_seq_workspace(int n_items) { return 256 + (size_t)(n_items > 0 ? n_items : 0) * sizeof(int); }
 
-template <int WB, int CPG>
+template <int WB, int CPG, bool I8>
 static cudaError_t launch_seq_cfg(seq::Params& p, cudaStream_t st) {
-    auto kernel = seq::gemv_seq_kernel<WB, CPG>;
+    auto kernel = seq::gemv_seq_kernel<WB, CPG, I8>;
     const int stage_bytes = seq::kStageUnits * p.unit_bytes;
     p.n_stages = 3;
     const size_t smem = (size_t)2 * kLutBytes + (size_t)p.n_stages * stage_bytes + (size_t)seq::kRedSlots * seq::kConsumerWarps * 32 * 4 * sizeof(float) +
-                        (size_t)(2 * p.n_stages + 2) * sizeof(uint64_t) + (size_t)seq::kXBufBytes;
+                        (size_t)(2 * p.n_stages + 2) * sizeof(uint64_t) + (size_t)seq::kXBufBytes + (size_t)seq::kScaleFloats * sizeof(float);
     static size_t attr_smem = 0;
     static int per_sm = 0;
     if (smem > attr_smem) {
@@ -353,8 +471,14 @@ cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, i
         it.tile_base = 0;
     }
     const int cpg = group / 32;
-    if (wbits == 3) return cpg == 1 ? launch_seq_cfg<3, 1>(p, st) : cpg == 2 ? launch_seq_cfg<3, 2>(p, st) : launch_seq_cfg<3, 4>(p, st);
-    return cpg == 1 ? launch_seq_cfg<2, 1>(p, st) : cpg == 2 ? launch_seq_cfg<2, 2>(p, st) : launch_seq_cfg<2, 4>(p, st);
+    bool i8 = g_seq_int8;   // the integer form serves batch <= 4; one kernel per launch, so every item must qualify
+    for (int i = 0; i < n; ++i) i8 = i8 && calls[i].m <= 4;
+    if (i8) {
+        if (wbits == 3) return cpg == 1 ? launch_seq_cfg<3, 1, true>(p, st) : cpg == 2 ? launch_seq_cfg<3, 2, true>(p, st) : launch_seq_cfg<3, 4, true>(p, st);
+        return cpg == 1 ? launch_seq_cfg<2, 1, true>(p, st) : cpg == 2 ? launch_seq_cfg<2, 2, true>(p, st) : launch_seq_cfg<2, 4, true>(p, st);
+    }
+    if (wbits == 3) return cpg == 1 ? launch_seq_cfg<3, 1, false>(p, st) : cpg == 2 ? launch_seq_cfg<3, 2, false>(p, st) : launch_seq_cfg<3, 4, false>(p, st);
+    return cpg == 1 ? launch_seq_cfg<2, 1, false>(p, st) : cpg == 2 ? launch_seq_cfg<2, 2, false>(p, st) : launch_seq_cfg<2, 4, false>(p, st);
 }
 
 }  // namespace goq

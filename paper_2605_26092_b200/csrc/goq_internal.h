@@ -45,6 +45,7 @@ struct SeqCall {
     void* y;
     int m, y_dtype, depends;
 };
+extern bool g_seq_int8;   // false: never use the integer-operand form (tests)
 bool gemv_seq_supported(const Geometry& g, int m);
 size_t gemv_seq_workspace(int n_items);
 cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, int unit_bytes, void* ws, cudaStream_t st);

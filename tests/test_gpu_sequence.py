@@ -33,7 +33,15 @@ def _ws(goq, n_items):
     return ws
 
 
-def test_chain_with_real_dependencies_matches_oracle_stage_by_stage(goq):
+@pytest.fixture(params=[0, 5], ids=["auto", "bf16-operands"])
+def form(goq, request):
+    """0: the kernel picks integer operands when every item has batch <= 4; 5: always bf16 operands."""
+    prev = goq.set_gemv_variant(request.param)
+    yield request.param
+    goq.set_gemv_variant(prev)
+
+
+def test_chain_with_real_dependencies_matches_oracle_stage_by_stage(goq, form):
     """y0 = W0 x0 (bf16 out) feeds W1, whose bf16 output feeds W2: every stage is checked against the oracle
     evaluated on the bits the previous stage actually produced."""
     from tests.gpu_util import dev
@@ -63,7 +71,7 @@ def test_chain_with_real_dependencies_matches_oracle_stage_by_stage(goq):
 
 
 @pytest.mark.parametrize("g,b", [(128, 3), (32, 2)])
-def test_independent_items_of_mixed_shapes(goq, g, b):
+def test_independent_items_of_mixed_shapes(goq, g, b, form):
     """Ragged rows and k, fewer and more than 16 k-blocks per tile, batch 1..8, both output types."""
     from tests.gpu_util import dev
     shapes = [(40, 256, 1), (300, 4224, 2), (16, 128, 8), (1000, 1152, 5), (257, 2048 + 128, 3)]
@@ -92,7 +100,37 @@ def test_independent_items_of_mixed_shapes(goq, g, b):
     del keep
 
 
-def test_one_7b_shaped_layer_sampled_rows(goq):
+@pytest.mark.parametrize("g,b", [(128, 3), (64, 2)])
+def test_small_batches_integer_operand_form(goq, g, b, form):
+    """Every item has batch <= 4, so the automatic choice is the integer-operand form; extreme activations included."""
+    from tests.gpu_util import dev
+    shapes = [(40, 256, 1), (300, 4224, 2), (16, 128, 4), (1000, 1152, 3), (257, 2048 + 128, 1)]
+    keep, checks, items = [], [], []
+    for i, (n, k, m) in enumerate(shapes):
+        L = _layer(goq, n, k, g, b, seed=190 + i)
+        x = si.bf16_bits_to_f64(si.bf16_activations(m, k, seed=160 + i))
+        if i == 1:
+            x[0, ::3] = 0.0
+            x[0, 1::7] *= 2.0 ** -60
+            x[1, ::5] *= 2.0 ** 40
+        xb = si.f32_to_bf16_bits(x.astype(np.float32))
+        y = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda")
+        xd = dev(xb)
+        keep.append(xd)
+        items.append((L["d"], L["packed"], xd, m, y, goq.F32, False))
+        checks.append((L, xb, y))
+    ws = _ws(goq, len(items))
+    goq.gemv_sequence(goq.make_sequence(items), ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    for L, xb, y in checks:
+        y_ref = O.linear_f64(L["codes"], L["meta"], L["coef"], si.bf16_bits_to_f64(xb), g, b)
+        err = O.normwise_rel_err(y.cpu().numpy().astype(np.float64), y_ref)
+        print("sequence form %d: normwise error %.3e" % (form, err))
+        assert err <= TIGHT, err
+
+
+def test_one_7b_shaped_layer_sampled_rows(goq, form):
     from tests.gpu_util import dev
     items, checks = [], []
     for i, (name, n, k) in enumerate(si.LLAMA2_7B_LINEARS):
