@@ -233,7 +233,8 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const uint32_t bits = (j & 1) ? (in32[j >> 1] & 0xFFFF0000u) : (in32[j >> 1] << 16);
-                    int Q = __float2int_rn(__uint_as_float(bits) * mult);
+                    // rne to an integer without the quarter-rate convert: adding 1.5 * 2^23 leaves it in the low mantissa bits
+                    int Q = __float_as_int(fmaf(__uint_as_float(bits), mult, 12582912.0f)) - 0x4B400000;
                     Q = max(-32639, min(32639, Q));
                     const int lo = ((Q + 128) & 255) - 128, hi = (Q - lo) >> 8;   // Q = 256 hi + lo, both int8
                     q0[j >> 2] |= (uint32_t)(hi & 255) << (8 * (j & 3));
