@@ -304,23 +304,49 @@ def run_cuda(args):
     ms = e0.elapsed_time(e1) / args.steps
     ms_max, value = aggregate_replicas(ms, step_bytes, world, "cuda")
 
-    # ---- end to end: host buffers in, host buffers out, through goq_gemv_host -------------------
-    host = []
-    for s in stack:
-        xh = s["x"].cpu().pin_memory()
-        yh = torch.empty((1, s["n"]), dtype=torch.float32).pin_memory()
-        host.append((xh, yh))
+    # ---- end to end: host buffers in, host buffers out, through the C ABI's host entry points ---------
+    if args.launch == "sequence":
+        # one pinned host block with every linear's activations, one with every output; goq_gemv_sequence_host
+        # copies the first in, runs the sequence kernel on views of the device blocks, copies the second out
+        x_off, y_off, xo, yo = [], [], 0, 0
+        for s in stack:
+            x_off.append(xo); xo += (s["k"] * 2 + 255) // 256 * 256
+            y_off.append(yo); yo += (s["n"] * 4 + 255) // 256 * 256
+        x_stage = torch.zeros(xo, dtype=torch.uint8, device="cuda")
+        y_stage = torch.zeros(yo, dtype=torch.uint8, device="cuda")
+        x_host = torch.zeros(xo, dtype=torch.uint8).pin_memory()
+        y_host = torch.zeros(yo, dtype=torch.uint8).pin_memory()
+        views = []
+        for s, a, b in zip(stack, x_off, y_off):
+            x_host[a:a + s["k"] * 2] = s["x"].view(torch.uint8).flatten().cpu()
+            views.append((x_stage[a:a + s["k"] * 2].view(torch.bfloat16).view(1, s["k"]),
+                          y_stage[b:b + s["n"] * 4].view(torch.float32).view(1, s["n"])))
+        seq_e2e = goq.make_sequence([(s["d"], s["packed"], xv, 1, yv, goq.F32, True) for s, (xv, yv) in zip(stack, views)])
+        e2e_desc = "one CUDA graph holding one goq_gemv_sequence_host call (one pinned H2D block, the sequence kernel, one D2H block)"
 
-    def step_e2e():
-        for s, (xh, yh) in zip(stack, host):
-            goq.gemv_host(s["d"], s["packed"], xh, 1, yh, goq.F32, s["x"], s["y"], ws=ws)
+        def step_e2e():
+            goq.gemv_sequence_host(seq_e2e, x_host, x_stage, y_host, y_stage, ws_seq)
+    else:
+        host = []
+        for s in stack:
+            xh = s["x"].cpu().pin_memory()
+            yh = torch.empty((1, s["n"]), dtype=torch.float32).pin_memory()
+            host.append((xh, yh))
+        e2e_desc = "one CUDA graph of goq_gemv_host calls (pinned H2D, kernel, D2H per linear)"
+
+        def step_e2e():
+            for s, (xh, yh) in zip(stack, host):
+                goq.gemv_host(s["d"], s["packed"], xh, 1, yh, goq.F32, s["x"], s["y"], ws=ws)
 
     g2 = capture(torch, step_e2e)
     e2e_steps = max(3, args.steps // 4)
     ms_e2e = time_graph(torch, g2, e2e_steps, 3)
     _, e2e_val = aggregate_replicas(ms_e2e, step_bytes, world, "cuda")
-    h2d = sum(s["k"] * 2 for s in stack)
-    d2h = sum(s["n"] * 4 for s in stack)
+    if args.launch == "sequence":
+        h2d, d2h = x_stage.numel(), y_stage.numel()   # the blocks as copied (each linear's slice padded to 256 bytes)
+    else:
+        h2d = sum(s["k"] * 2 for s in stack)
+        d2h = sum(s["n"] * 4 for s in stack)
 
     if rank != 0:
         if world > 1:
@@ -370,7 +396,7 @@ def run_cuda(args):
                      "kernel": kernel_name, "bytes_per_launch_avg": launch_bytes, "us_per_launch_avg": launch_ms * 1e3},
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "launch": "one CUDA graph of goq_gemv_host calls (pinned H2D, kernel, D2H per linear)"},
+                "launch": e2e_desc},
         "gpu_launches": args.steps * kernels_per_step,
         "clocks": sampler.summary(),
         "extras": extras,

@@ -197,6 +197,18 @@ typedef struct {
 size_t goq_sequence_workspace_bytes(int n_items);
 goq_status goq_gemv_sequence(const goq_gemv_item* items, int n_items, void* ws, size_t ws_bytes, void* stream);
 
+/* goq_gemv_sequence_host: goq_gemv_sequence for callers whose activations and results live in HOST memory.
+ * All activations of the sequence sit in one host block and all outputs in another; the call enqueues, on `stream`,
+ *   one copy x_host -> x_stage (x_bytes), the sequence kernel, one copy y_stage -> y_host (y_bytes).
+ *   items     as in goq_gemv_sequence; every items[i].x_bf16 must point inside [x_stage, x_stage + x_bytes) or, for
+ *             an item fed by an earlier item, inside [y_stage, y_stage + y_bytes); every items[i].y inside the y block
+ *             (else GOQ_ERR_INVALID_ARG). The layout of the two blocks is the caller's.
+ *   x_host, y_host   host pointers (pinned memory makes the copies asynchronous); x_stage, y_stage device blocks.
+ * Asynchronous like every other entry point: y_host is valid once the stream has been synchronised. */
+goq_status goq_gemv_sequence_host(const goq_gemv_item* items, int n_items, const void* x_host, void* x_stage,
+                                  size_t x_bytes, void* y_host, void* y_stage, size_t y_bytes, void* ws,
+                                  size_t ws_bytes, void* stream);
+
 /* The cudaError_t value behind the most recent GOQ_ERR_CUDA returned in this process (0 if none). */
 int goq_last_cuda_error(void);
 

@@ -237,6 +237,28 @@ goq_status goq_gemv_sequence(const goq_gemv_item* items, int n_items, void* ws, 
     return GOQ_OK;
 }
 
+goq_status goq_gemv_sequence_host(const goq_gemv_item* items, int n_items, const void* x_host, void* x_stage,
+                                  size_t x_bytes, void* y_host, void* y_stage, size_t y_bytes, void* ws,
+                                  size_t ws_bytes, void* stream) {
+    if (!items || n_items < 1 || !x_host || !x_stage || !y_host || !y_stage || !x_bytes || !y_bytes) return GOQ_ERR_INVALID_ARG;
+    const uintptr_t xs = (uintptr_t)x_stage, ys = (uintptr_t)y_stage;
+    for (int i = 0; i < n_items; ++i) {
+        const goq_gemv_item& it = items[i];
+        if (it.batch < 1 || it.desc.k_in <= 0 || it.desc.n_out <= 0) return GOQ_ERR_INVALID_ARG;
+        const size_t xb = (size_t)it.batch * it.desc.k_in * 2;
+        const size_t yb = (size_t)it.batch * it.desc.n_out * (it.y_dtype == GOQ_F32 ? 4 : 2);
+        const uintptr_t x = (uintptr_t)it.x_bf16, y = (uintptr_t)it.y;
+        const bool x_in_x = x >= xs && x + xb <= xs + x_bytes, x_in_y = x >= ys && x + xb <= ys + y_bytes;
+        if (!(x_in_x || (x_in_y && i > 0 && it.depends)) || !(y >= ys && y + yb <= ys + y_bytes)) return GOQ_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(x_stage, x_host, x_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return from_cuda(cudaGetLastError());
+    goq_status s = goq_gemv_sequence(items, n_items, ws, ws_bytes, stream);
+    if (s != GOQ_OK) return s;
+    if (cudaMemcpyAsync(y_host, y_stage, y_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return from_cuda(cudaGetLastError());
+    return GOQ_OK;
+}
+
 goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x_host, int batch, void* y_host,
                          int y_dtype, void* x_stage, void* y_stage, void* ws, size_t ws_bytes, void* stream) {
     Geometry g;

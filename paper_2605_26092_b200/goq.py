@@ -23,7 +23,7 @@ EXPORTS = (
     "goq_status_string", "goq_packed_bytes", "goq_algorithmic_bytes", "goq_workspace_bytes", "goq_pack",
     "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant", "goq_workspace_init",
     "goq_workspace_status", "goq_gemv_static", "goq_last_cuda_error", "goq_sequence_workspace_bytes",
-    "goq_gemv_sequence",
+    "goq_gemv_sequence", "goq_gemv_sequence_host",
 )
 
 
@@ -84,6 +84,9 @@ def lib() -> ctypes.CDLL:
         L.goq_sequence_workspace_bytes.argtypes = [c_int]
         L.goq_gemv_sequence.restype = c_int
         L.goq_gemv_sequence.argtypes = [POINTER(GemvItem), c_int, c_void_p, ctypes.c_size_t, c_void_p]
+        L.goq_gemv_sequence_host.restype = c_int
+        L.goq_gemv_sequence_host.argtypes = [POINTER(GemvItem), c_int, c_void_p, c_void_p, ctypes.c_size_t, c_void_p,
+                                             c_void_p, ctypes.c_size_t, c_void_p, ctypes.c_size_t, c_void_p]
         L.goq_set_gemv_variant.restype = c_int
         L.goq_set_gemv_variant.argtypes = [c_int]
         _lib = L
@@ -194,6 +197,15 @@ def gemv_sequence(seq, ws, stream=None):
     """goq_gemv_sequence: a chain of decode GEMVs in one persistent kernel. `seq` comes from make_sequence."""
     _check(lib().goq_gemv_sequence(seq, len(seq), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
            "goq_gemv_sequence")
+
+
+def gemv_sequence_host(seq, x_host, x_stage, y_host, y_stage, ws, stream=None):
+    """goq_gemv_sequence_host: one copy of the activation block in, the sequence kernel, one copy of the output
+    block out. x_host / y_host are (pinned) host tensors, x_stage / y_stage the device blocks the items point into."""
+    xb, yb = x_stage.numel() * x_stage.element_size(), y_stage.numel() * y_stage.element_size()
+    _check(lib().goq_gemv_sequence_host(seq, len(seq), _ptr(x_host), _ptr(x_stage), xb, _ptr(y_host), _ptr(y_stage), yb,
+                                        _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
+           "goq_gemv_sequence_host")
 
 
 def gemm(d: Desc, packed, x, m: int, x_dtype: int, y=None, y_dtype: int = F32, sx=None, cq=None, sc=None,

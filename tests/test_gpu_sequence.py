@@ -174,3 +174,36 @@ def test_unsupported_and_invalid_sequences_return_a_status(goq):
     with pytest.raises(goq.GoqError) as e:
         goq.gemv_sequence(goq.make_sequence(mixed[:1] * 2), small)
     assert e.value.status == goq.ERR_WORKSPACE
+
+
+def test_host_block_entry_point(goq):
+    """goq_gemv_sequence_host: activations in one pinned host block, outputs in another; a two-linear chain whose
+    second item reads the first one's bf16 output inside the output block."""
+    n0, k0, n1, m = 256, 384, 100, 2
+    L0, L1 = _layer(goq, n0, k0, 64, 3, seed=11), _layer(goq, n1, n0, 64, 3, seed=12)
+    xb = si.bf16_activations(m, k0, seed=9)
+    x_bytes, y0_bytes, y1_bytes = m * k0 * 2, m * n0 * 2, m * n1 * 4
+    x_stage = torch.zeros(x_bytes, dtype=torch.uint8, device="cuda")
+    y_stage = torch.zeros(y0_bytes + y1_bytes, dtype=torch.uint8, device="cuda")
+    x_host = torch.from_numpy(xb.view(np.uint8).reshape(-1).copy()).pin_memory()
+    y_host = torch.zeros(y0_bytes + y1_bytes, dtype=torch.uint8).pin_memory()
+    xv = x_stage.view(torch.bfloat16).view(m, k0)
+    y0v = y_stage[:y0_bytes].view(torch.bfloat16).view(m, n0)
+    y1v = y_stage[y0_bytes:].view(torch.float32).view(m, n1)
+    seq = goq.make_sequence([(L0["d"], L0["packed"], xv, m, y0v, goq.BF16, False), (L1["d"], L1["packed"], y0v, m, y1v, goq.F32, True)])
+    ws = _ws(goq, 2)
+    goq.gemv_sequence_host(seq, x_host, x_stage, y_host, y_stage, ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    mid_bits = y_host[:y0_bytes].numpy().view(np.uint16).reshape(m, n0)
+    y0_ref = O.linear_f64(L0["codes"], L0["meta"], L0["coef"], si.bf16_bits_to_f64(xb), 64, 3)
+    assert O.normwise_rel_err(si.bf16_bits_to_f64(mid_bits), y0_ref) <= 4e-3
+    y1 = y_host[y0_bytes:].numpy().view(np.float32).reshape(m, n1).astype(np.float64)
+    y1_ref = O.linear_f64(L1["codes"], L1["meta"], L1["coef"], si.bf16_bits_to_f64(mid_bits), 64, 3)
+    assert O.normwise_rel_err(y1, y1_ref) <= TIGHT
+    # an item whose buffers lie outside the blocks is refused on the host
+    stray = torch.zeros((m, n1), dtype=torch.float32, device="cuda")
+    bad = goq.make_sequence([(L0["d"], L0["packed"], xv, m, y0v, goq.BF16, False), (L1["d"], L1["packed"], y0v, m, stray, goq.F32, True)])
+    with pytest.raises(goq.GoqError) as e:
+        goq.gemv_sequence_host(bad, x_host, x_stage, y_host, y_stage, ws)
+    assert e.value.status == goq.ERR_INVALID_ARG
