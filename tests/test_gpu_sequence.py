@@ -207,3 +207,28 @@ def test_host_block_entry_point(goq):
     with pytest.raises(goq.GoqError) as e:
         goq.gemv_sequence_host(bad, x_host, x_stage, y_host, y_stage, ws)
     assert e.value.status == goq.ERR_INVALID_ARG
+
+
+def test_long_sequence_is_split_into_launches_and_small_grids_work(goq, form):
+    """300 items (more than one launch holds) over two tiny layers: 8 row tiles in all per launch chunk would leave most
+    CTAs without work, so the grid shrinks to the tile count; every item is checked."""
+    from tests.gpu_util import dev
+    La, Lb = _layer(goq, 48, 128, 64, 3, seed=501), _layer(goq, 80, 256, 64, 3, seed=502)
+    xa, xb_ = si.bf16_activations(2, 128, seed=21), si.bf16_activations(2, 256, seed=22)
+    xad, xbd = dev(xa), dev(xb_)
+    ys, items = [], []
+    for i in range(300):
+        L, x, k = (La, xad, 128) if i % 2 == 0 else (Lb, xbd, 256)
+        y = torch.full((2, L["n"]), float("nan"), dtype=torch.float32, device="cuda")
+        ys.append(y)
+        items.append((L["d"], L["packed"], x, 2, y, goq.F32, i % 3 != 0))
+    ws = _ws(goq, len(items))
+    goq.gemv_sequence(goq.make_sequence(items), ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    ref_a = O.linear_f64(La["codes"], La["meta"], La["coef"], si.bf16_bits_to_f64(xa), 64, 3)
+    ref_b = O.linear_f64(Lb["codes"], Lb["meta"], Lb["coef"], si.bf16_bits_to_f64(xb_), 64, 3)
+    for i, y in enumerate(ys):
+        ref = ref_a if i % 2 == 0 else ref_b
+        assert O.normwise_rel_err(y.cpu().numpy().astype(np.float64), ref) <= TIGHT, i
+    assert torch.equal(ys[0], ys[298]) and torch.equal(ys[1], ys[299])
