@@ -267,10 +267,12 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
             int n_rec = p.n_tiles - T0;
             if (n_rec > kExpanders) n_rec = kExpanders;
             bool ok = true;
+            int pk_issued = 0, b_issued = 0;   // record blocks / activation chunks whose copies have been issued
             for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
                 const int ps = kb & 1;
                 if (kb >= 2) ok = mbar_wait(&pk_empty[ps], ((kb >> 1) - 1) & 1, &abort_flag);
                 if (!ok) break;
+                pk_issued = kb + 1;
                 mbar_expect_tx(&pk_full[ps], (uint32_t)n_rec * p.unit_bytes);
                 for (int r = 0; r < n_rec; ++r)
                     bulk_g2s(pk_ring + ps * pk_slot_bytes + r * p.unit_bytes,
@@ -279,10 +281,18 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                     const int chunk = 2 * kb + half, s = chunk % kStages;
                     if (chunk >= kStages) ok = mbar_wait(&empty[s], ((chunk / kStages) - 1) & 1, &abort_flag);
                     if (!ok) break;
+                    b_issued = chunk + 1;
                     mbar_expect_tx(&full_b[s], kBTileBytes);
                     tma_load_2d(b_tiles + s * kBTileBytes, &x_map, chunk * kChunkK, tok0, &full_b[s]);
                     tma_load_2d(b_tiles + s * kBTileBytes + kBTileBytes / 2, &x_map, chunk * kChunkK, tok0 + 256, &full_b[s]);
                 }
+            }
+            if (!ok || abort_flag) {
+                // after a give-up: copies already issued must land before the CTA's shared memory goes away (bounded waits)
+                for (int i = pk_issued > 2 ? pk_issued - 2 : 0; i < pk_issued; ++i)
+                    for (int it = 0; it < kSpin && !mbar_try(&pk_full[i & 1], (uint32_t)(i >> 1) & 1u); ++it) { }
+                for (int i = b_issued > kStages ? b_issued - kStages : 0; i < b_issued; ++i)
+                    for (int it = 0; it < kSpin && !mbar_try(&full_b[i % kStages], (uint32_t)(i / kStages) & 1u); ++it) { }
             }
         }
     } else if (warp == 1) {

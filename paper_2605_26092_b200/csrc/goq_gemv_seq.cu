@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
     if (warp == kConsumerWarps) {
         // ---------------- producer: the weight stream of every tile this CTA owns, linear after linear ----------------
         if (lane == 0) {
-            int slot = 0, round = 0;
+            int slot = 0, round = 0, issued = 0;
             bool ok = true;
             for (int i = 0; i < p.n_items && ok; ++i) {
                 const Item& it = p.item[i];
@@ -151,9 +151,11 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
                         mbar_arrive_expect_tx(&full_bar[slot], bytes);
                         bulk_copy_g2s(ring + (size_t)slot * stage_bytes, src + (size_t)u0 * p.unit_bytes, bytes, &full_bar[slot]);
                         if (++slot == p.n_stages) { slot = 0; ++round; }
+                        ++issued;
                     }
                 }
             }
+            if (!ok || abort_flag) drain_issued_stages(full_bar, issued, p.n_stages);
         }
         return;
     }

@@ -130,11 +130,12 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
             const uint8_t* src = p.packed + (size_t)u_begin * p.unit_bytes;
             int slot = 0, round = 0;
             bool x_issued = (p.x_smem_bytes == 0);
+            int issued = 0;
             for (int s = 0; s < my_stages; ++s) {
-
                 if (round > 0) {
                     if (!mbar_wait_bounded(&empty_bar[slot], (round - 1) & 1, &abort_flag)) break;
                 }
+                issued = s + 1;
                 const int units = min(kStageUnits, my_units - s * kStageUnits);
                 const uint32_t bytes = (uint32_t)units * p.unit_bytes;
                 mbar_arrive_expect_tx(&full_bar[slot], bytes);
@@ -153,6 +154,7 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
                 }
             }
             GOQ_TR(3);
+            if (abort_flag) drain_issued_stages(full_bar, issued, p.n_stages);
         }
         return;
     }

@@ -56,6 +56,17 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     *abort_flag = 1;
     return false;
 }
+// After a give-up: the bulk copies this thread has already issued must land before the CTA (and its shared
+// memory) goes away. `issued` stages were issued in ring order over `n_stages` slots; the last min(issued, n_stages)
+// may still be in flight. Bounded, and deliberately blind to the abort flag.
+__device__ __forceinline__ void drain_issued_stages(uint64_t* full_bar, int issued, int n_stages) {
+    const int first = issued > n_stages ? issued - n_stages : 0;
+    for (int s = first; s < issued; ++s) {
+        const int slot = s % n_stages;
+        const uint32_t parity = (uint32_t)(s / n_stages) & 1u;
+        for (int it = 0; it < kSpinLimit && !mbar_try_wait(&full_bar[slot], parity); ++it) { }
+    }
+}
 // Device-scope fetch-add that releases this warp's earlier writes (ordered before it by __syncwarp) and
 // acquires the writes of the CTAs that incremented before.
 __device__ __forceinline__ int atomic_add_acq_rel_gpu(int* addr, int v) {
