@@ -192,7 +192,7 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
     if (x_dtype == GOQ_I8) {
         if (!cq || (!y && !acc)) return GOQ_ERR_INVALID_ARG;
         if (y && (!sx || !sc)) return GOQ_ERR_INVALID_ARG;
-        if (!aligned(acc, 4) || !aligned(sx, 4) || !aligned(sc, 4)) return GOQ_ERR_ALIGNMENT;
+        if (!aligned(acc, 4) || !aligned(sx, 4) || !aligned(sc, 4) || !aligned(cq, 2)) return GOQ_ERR_ALIGNMENT;
         if (g.wbits > 3 || g.group < 16 || (g.k_in % 16)) return GOQ_ERR_UNSUPPORTED;
         // |ACC| <= k_in * 127 (x~) * 127 (c~) * 2^emax must stay below 2^31
         const long long bound = (long long)g.k_in * 127 * 127 * (1ll << ((1 << (g.wbits - 1)) - 1));

@@ -157,52 +157,122 @@ template <> struct IntTables<2> {  // codes 0..3 -> 2 0 -2 -1
 };
 
 constexpr int kA8Warps = 8;
-constexpr int kA8NT = 8;  // 8-token column tiles per warp: 64 tokens
+constexpr int kA8NT = 8;          // 8-token column tiles per warp: 64 tokens per CTA
+constexpr int kA8Tok = 8 * kA8NT;
+constexpr int kA8XStride = 160;   // bytes per token row of the staged activation tile: 128 + 32, so that the 16 lanes of a
+                                  // half-warp (4 token rows x 4 eight-byte pieces) hit 32 different banks
+constexpr uint32_t kA8HashMul = 0x01008420u;   // (record bits in place) * this >> 26 is a bijection onto 0..63
 
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ uint2 a8_lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint4 a8_lds128(uint32_t addr) {
+    uint4 v;
+    asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// CTA = 8 warps: warp w owns the 16-row tile 8*blockIdx.x + w, all warps share the same 64 tokens. Per 128-wide
+// k-block the activation tile (64 tokens x 128 int8) is staged in shared memory with cp.async, double-buffered; each
+// warp reads its unit record straight from global memory one k-block ahead. Row sums S1, S2 per macro-block on the
+// int8 tensor cores, then ACC += c~ * S in int32: every order of these integer operations gives the same bits.
 template <int WB>
 __global__ void __launch_bounds__(kA8Warps * 32, 1)
 gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int8_t* __restrict__ x,
                    const float* __restrict__ sx, const int8_t* __restrict__ cq, const float* __restrict__ sc,
                    void* __restrict__ y, int y_dtype, int32_t* __restrict__ acc_out, int n_out, int n_tiles, int k_in,
                    int k_blocks, int group, int m_total) {
-    __shared__ uint4 lut[64];  // per record: byte selectors for positions 0..3 / 4..7, byte masks of flipped positions
-    if (threadIdx.x < 64) {
-        const uint32_t meta = threadIdx.x;
+    // record table: byte selectors for positions 0..3 / 4..7 and byte masks of the flipped positions, indexed by the
+    // hash of the record bits, eight bank-disjoint copies (entry e, copy c at e*128 + c*16)
+    __shared__ __align__(16) unsigned char lut[64 * 8 * 16];
+    __shared__ __align__(16) unsigned char xs[2][kA8Tok * kA8XStride];
+    for (int i = threadIdx.x; i < 512; i += kA8Warps * 32) {
+        const uint32_t meta = i >> 3;
         const int s = (int)(meta & 3u) + 1;
         const uint32_t flips = flip_mask(meta);
         uint32_t sel_a = 0, sel_b = 0, m_a = 0, m_b = 0;
-        for (int i = 0; i < 4; ++i) {
-            sel_a |= (uint32_t)(i ^ s) << (4 * i);
-            sel_b |= (uint32_t)((4 + i) ^ s) << (4 * i);
-            if ((flips >> i) & 1u) m_a |= 0xFFu << (8 * i);
-            if ((flips >> (4 + i)) & 1u) m_b |= 0xFFu << (8 * i);
+        for (int j = 0; j < 4; ++j) {
+            sel_a |= (uint32_t)(j ^ s) << (4 * j);
+            sel_b |= (uint32_t)((4 + j) ^ s) << (4 * j);
+            if ((flips >> j) & 1u) m_a |= 0xFFu << (8 * j);
+            if ((flips >> (4 + j)) & 1u) m_b |= 0xFFu << (8 * j);
         }
-        lut[meta] = make_uint4(sel_a, sel_b, m_a, m_b);
+        const uint32_t slot = (scatter_meta(meta) * kA8HashMul) >> 26;
+        *reinterpret_cast<uint4*>(lut + slot * 128 + (i & 7) * 16) = make_uint4(sel_a, sel_b, m_a, m_b);
     }
-    __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int T = blockIdx.x * kA8Warps + warp;
-    if (T >= n_tiles) return;
-    const int tok0 = blockIdx.y * (8 * kA8NT);
+    const bool have_tile = T < n_tiles;
+    const int tok0 = blockIdx.y * kA8Tok;
     const int groups_in = k_in / group, cpg = group >> 5;
     const int row_a = T * 16 + g, row_b = row_a + 8;
+    const uint32_t lut_lane = (uint32_t)__cvta_generic_to_shared(lut) + (uint32_t)(lane & 7) * 16u;
+    const uint32_t xs_base = (uint32_t)__cvta_generic_to_shared(&xs[0][0]);
+
+    // the whole CTA copies the activation tile of k-block bk into buffer bk & 1: 512 chunks of 16 bytes, two per thread
+    auto stage_x = [&](int bk) {
+        const uint32_t dst0 = xs_base + (uint32_t)(bk & 1) * (kA8Tok * kA8XStride);
+#pragma unroll
+        for (int j = 0; j < (kA8Tok * 8) / (kA8Warps * 32); ++j) {
+            const int q = threadIdx.x + j * kA8Warps * 32, tok = q >> 3, part = q & 7;
+            const int k0 = bk * kBlockK + part * 16;
+            const uint32_t dst = dst0 + (uint32_t)(tok * kA8XStride + part * 16);
+            if (k0 < k_in) cp_async16(dst, x + (size_t)min(tok0 + tok, m_total - 1) * k_in + k0);   // k_in % 16 == 0: a chunk is all in or all out
+            else asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(dst), "r"(0u) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
 
     int acc1[kA8NT][4], acc2[kA8NT][4], s1[kA8NT][4], s2[kA8NT][4];
 #pragma unroll
     for (int nt = 0; nt < kA8NT; ++nt)
 #pragma unroll
         for (int r = 0; r < 4; ++r) acc1[nt][r] = acc2[nt][r] = s1[nt][r] = s2[nt][r] = 0;
-    const int8_t* xrow[kA8NT];
-#pragma unroll
-    for (int nt = 0; nt < kA8NT; ++nt) xrow[nt] = x + (size_t)min(tok0 + nt * 8 + g, m_total - 1) * k_in + t * 8;
 
+    // integer coefficient pairs (c1, c2) of rows g and g+8 for the up to four macro-blocks of k-block bk, fetched one
+    // k-block ahead like the words: element jj = c1a | c2a << 8 | c1b << 16 | c2b << 24 (as unsigned bytes)
+    const int gpb = 4 / cpg;
+    auto fetch_coef = [&](int bk, uint32_t (&cf)[4]) {
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            cf[jj] = 0u;
+            const int j = bk * gpb + jj;
+            if (jj < gpb && j < groups_in) {
+                uint32_t lo = 0u, hi = 0u;
+                if (row_a < n_out) lo = *reinterpret_cast<const uint16_t*>(cq + ((size_t)row_a * groups_in + j) * 2);
+                if (row_b < n_out) hi = *reinterpret_cast<const uint16_t*>(cq + ((size_t)row_b * groups_in + j) * 2);
+                cf[jj] = lo | (hi << 16);
+            }
+        }
+    };
+    stage_x(0);
+    uint32_t ncf[4] = {0u, 0u, 0u, 0u};
+    if (have_tile) fetch_coef(0, ncf);
+    uint4 nw0 = make_uint4(0, 0, 0, 0), nw1 = nw0;   // the next k-block's words of this warp's record
+    if (have_tile) {
+        const uint4* unit = reinterpret_cast<const uint4*>(packed + unit_offset(T, 0, k_blocks, unit_bytes));
+        nw0 = unit[lane]; nw1 = unit[32 + lane];
+    }
     for (int bk = 0; bk < k_blocks; ++bk) {
-        const uint8_t* unit = packed + unit_offset(T, bk, k_blocks, unit_bytes);
-        const uint4 wv0 = reinterpret_cast<const uint4*>(unit)[lane], wv1 = reinterpret_cast<const uint4*>(unit)[32 + lane];
-        const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();   // tile bk has landed for everyone; everyone has finished reading tile bk - 1
+        if (bk + 1 < k_blocks) stage_x(bk + 1);
+        const uint32_t w0[4] = {nw0.x, nw0.y, nw0.z, nw0.w}, w1[4] = {nw1.x, nw1.y, nw1.z, nw1.w};
+        const uint32_t cf[4] = {ncf[0], ncf[1], ncf[2], ncf[3]};
+        if (have_tile && bk + 1 < k_blocks) {
+            fetch_coef(bk + 1, ncf);
+            const uint4* unit = reinterpret_cast<const uint4*>(packed + unit_offset(T, bk + 1, k_blocks, unit_bytes));
+            nw0 = unit[lane]; nw1 = unit[32 + lane];
+        }
+        if (!have_tile) continue;
+        const uint32_t xt = xs_base + (uint32_t)(bk & 1) * (kA8Tok * kA8XStride) + (uint32_t)(g * kA8XStride + t * 8);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            const int k0 = bk * kBlockK + c * 32;
             uint32_t a[4], q[4];
 #pragma unroll
             for (int v = 0; v < 2; ++v) {
@@ -210,7 +280,8 @@ gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int
                 const uint32_t m = w & 0x77777777u, mh = m >> 16;
                 const uint32_t p_lo = prmt8(IntTables<WB>::P0, IntTables<WB>::P1, m), p_hi = prmt8(IntTables<WB>::P0, IntTables<WB>::P1, mh);
                 const uint32_t n_lo = prmt8(IntTables<WB>::N0, IntTables<WB>::N1, m), n_hi = prmt8(IntTables<WB>::N0, IntTables<WB>::N1, mh);
-                const uint4 e = lut[gather_meta(w)];
+                const uint32_t h = (w - m) * kA8HashMul;
+                const uint4 e = a8_lds128((((h >> 26) * 128u)) + lut_lane);
                 a[v] = p_lo;          // m16n8k32 A fragment: a0/a1 = k 4t..4t+3 of rows g / g+8, a2/a3 = k 16+4t..
                 a[2 + v] = p_hi;
                 const uint32_t qp_lo = prmt8(p_lo, p_hi, e.x), qn_lo = prmt8(n_lo, n_hi, e.x);
@@ -218,21 +289,16 @@ gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int
                 q[v] = (qp_lo & ~e.z) | (qn_lo & e.z);
                 q[2 + v] = (qp_hi & ~e.w) | (qn_hi & e.w);
             }
-            const bool in_k = (k0 + t * 8) < k_in;
 #pragma unroll
             for (int nt = 0; nt < kA8NT; ++nt) {
-                uint2 b = make_uint2(0, 0);
-                if (in_k) b = *reinterpret_cast<const uint2*>(xrow[nt] + k0);
+                const uint2 b = a8_lds64(xt + (uint32_t)(nt * 8 * kA8XStride + c * 32));
                 mma_s8(s1[nt], a[0], a[1], a[2], a[3], b.x, b.y);
                 mma_s8(s2[nt], q[0], q[1], q[2], q[3], b.x, b.y);
             }
             if (((c + 1) % cpg) == 0) {
-                const int j = k0 / group;
-                int c1a = 0, c2a = 0, c1b = 0, c2b = 0;
-                if (j < groups_in) {
-                    if (row_a < n_out) { c1a = cq[((size_t)row_a * groups_in + j) * 2]; c2a = cq[((size_t)row_a * groups_in + j) * 2 + 1]; }
-                    if (row_b < n_out) { c1b = cq[((size_t)row_b * groups_in + j) * 2]; c2b = cq[((size_t)row_b * groups_in + j) * 2 + 1]; }
-                }
+                const uint32_t cw = cf[c / cpg];
+                const int c1a = (int)(int8_t)(cw & 255u), c2a = (int)(int8_t)((cw >> 8) & 255u);
+                const int c1b = (int)(int8_t)((cw >> 16) & 255u), c2b = (int)(int8_t)(cw >> 24);
 #pragma unroll
                 for (int nt = 0; nt < kA8NT; ++nt) {
                     acc1[nt][0] += c1a * s1[nt][0]; acc1[nt][1] += c1a * s1[nt][1];
@@ -245,6 +311,7 @@ gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int
             }
         }
     }
+    if (!have_tile) return;
     constexpr float kInvScale = 1.0f / (float)(1u << ((1u << (WB - 1)) - 1u));
 #pragma unroll
     for (int nt = 0; nt < kA8NT; ++nt)
@@ -270,7 +337,7 @@ cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* 
                            const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, cudaStream_t st) {
     auto* words = (const uint8_t*)packed;
     if (g.group >= 32) {
-        dim3 grid2((g.n_tiles + kA8Warps - 1) / kA8Warps, (m + 8 * kA8NT - 1) / (8 * kA8NT)), block2(kA8Warps * 32);
+        dim3 grid2((g.n_tiles + kA8Warps - 1) / kA8Warps, (m + kA8Tok - 1) / kA8Tok), block2(kA8Warps * 32);
         if (g.wbits == 3)
             gemm_a8_mma_kernel<3><<<grid2, block2, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, g.n_out,
                                                             g.n_tiles, g.k_in, g.k_blocks, g.group, m);
