@@ -258,6 +258,8 @@ def run_cuda(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     hbm_peak, tf_peak, peak_src = measured_peaks()
 
+    if args.gemv_variant:
+        goq.set_gemv_variant(args.gemv_variant)
     layers = args.layers
     stack = build_stack(goq, torch, layers, seed0=replica_seed(rank), batch=1)
     n_lin = len(stack)
@@ -572,6 +574,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--launch", choices=("sequence", "graph"), default="sequence",
                     help="how a step is issued: one goq_gemv_sequence call, or a CUDA graph of per-linear goq_gemv launches")
+    ap.add_argument("--gemv-variant", type=int, default=0,
+                    help="force a kernel variant (goq_set_gemv_variant): 0 automatic, 3 streaming, 4 tcgen05 tensor-memory GEMV, ...")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="dram bytes per launch of the dominant kernel from an ncu capture (reported as-is)")
     args = ap.parse_args()
