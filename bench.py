@@ -376,7 +376,8 @@ def run_cuda(args):
         if int(goq.workspace_status(ws_seq)) != 0:
             raise RuntimeError("sequence kernel reported a device-side timeout")
     else:
-        kernel_name = "gemv_stream_kernel<3,1,4,true>"
+        kernel_name = {4: "gemv_tc_kernel<3,1,16>", 2: "linear_mma_kernel<3,1>", 1: "gemv_scalar_kernel"}.get(
+            args.gemv_variant, "gemv_stream_kernel<3,1,4,true>")
         launch_desc = "one CUDA graph of %d goq_gemv nodes per step" % n_lin
         # one ncu capture of the 4096x4096 launch read 8.96 MB of DRAM for 8.39 MB of algorithmic bytes;
         # the packed image grows in proportion to n*k, so the ratio is applied to the average launch
