@@ -274,6 +274,13 @@ def run_cuda(args):
         ws_seq = torch.empty(goq.sequence_workspace_bytes(n_lin), dtype=torch.uint8, device="cuda")
         goq.workspace_init(ws_seq)
         kernels_per_step = (n_lin + 255) // 256
+        try:   # a device that refuses the cooperative launch still gets a number, from the per-linear launches
+            goq.gemv_sequence(seq, ws_seq)
+            torch.cuda.synchronize()
+        except goq.GoqError as e:
+            print("goq_gemv_sequence unavailable (%s): timing per-linear launches instead" % e, file=sys.stderr)
+            args.launch = "graph"
+    if args.launch == "sequence":
 
         def step():
             goq.gemv_sequence(seq, ws_seq)
