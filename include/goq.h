@@ -116,7 +116,10 @@ goq_status goq_unpack(const goq_desc* desc, const void* packed, uint8_t* codes_b
  *   y        out [batch][n_out], y_dtype GOQ_BF16 or GOQ_F32
  *   ws       scratch of goq_workspace_bytes(desc, GOQ_OP_GEMV, batch) bytes, 256-byte aligned,
  *            initialised once with goq_workspace_init (may be NULL if the size is 0)
- * Each PoT term is applied to the activation as an exponent shift; sums are fp32. */
+ * Each PoT term is applied to the activation as an exponent shift; sums are fp32. Up to 4 tokens
+ * whose activations fit the sequence kernel's staging buffer run as a one-linear goq_gemv_sequence
+ * in its integer-operand form (same rounding and saturation of non-finite activations as stated
+ * there); the other cases take the bf16-operand streaming kernel. */
 goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16, int batch, void* y,
                     int y_dtype, void* ws, size_t ws_bytes, void* stream);
 
