@@ -42,6 +42,10 @@ struct Params {
     int n_items, unit_bytes, n_stages;
     int* status;
     int* done;   // [n_items] CTAs that have finished each linear; zero on entry, left zero
+    // 255, read from the constant bank: 0/1 bytes times a value the compiler cannot see stays one multiply (on the
+    // multiply-add pipe) instead of a shift and a subtract on the logic pipe, which bounds the decode. (The same
+    // trick for the right shifts, as mul.hi by 2^16 and 2^13, was measured slower.)
+    uint32_t mul_255;
 };
 
 __device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory"); }
@@ -75,19 +79,25 @@ __device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, ui
     asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-// The record table holds sign-bit masks (bit 7 of each flipped byte); (mask >> 7) * 255 makes them byte masks.
-__device__ __forceinline__ uint32_t byte_mask(uint32_t sign_bits) { return (sign_bits >> 7) * 255u; }
-// one micro-block word -> b1 bytes (pa: weights 0..3, pb: 4..7) and b2 bytes, as int8 = value * 2^emax
+// The record table holds sign-bit masks (bit 7 of each flipped byte); >> 7 leaves a 1 in each flipped byte.
+__device__ __forceinline__ uint32_t flip_ones(uint32_t sign_bits) { return sign_bits >> 7; }
+// One micro-block word -> b1 bytes (pa: weights 0..3, pb: 4..7), int8 = value * 2^emax, and b2 as two operands:
+// the permuted b1 bytes with every flipped byte complemented (ra, rb), and a 1 in every flipped byte (za, zb).
+// ~v = -v - 1, so sum_i (~v_i) x_i + sum_i 1 x_i = -sum_i v_i x_i over the flipped positions: accumulating both
+// operands against the same activations gives the signed sum exactly (a flipped zero contributes -x + x = 0),
+// for one xor per register in place of a second table lookup, a second permute and a select.
 template <int WB>
-__device__ __forceinline__ void decode_i8(uint32_t w, uint32_t lut_lane, uint32_t& pa, uint32_t& pb, uint32_t& qa, uint32_t& qb) {
+__device__ __forceinline__ void decode_i8(const Params& p, uint32_t w, uint32_t lut_lane, uint32_t& pa, uint32_t& pb,
+                                          uint32_t& ra, uint32_t& rb, uint32_t& za, uint32_t& zb) {
     const uint32_t m = w & 0x77777777u, mh = m >> 16;
     pa = prmt_b32(IntTables<WB>::P0, IntTables<WB>::P1, m);
     pb = prmt_b32(IntTables<WB>::P0, IntTables<WB>::P1, mh);
-    const uint32_t na = prmt_b32(IntTables<WB>::N0, IntTables<WB>::N1, m), nb = prmt_b32(IntTables<WB>::N0, IntTables<WB>::N1, mh);
     const uint32_t h = (w - m) * kHashMul;
-    const uint4 e = lds128(((h >> 19) & 0x1F80u) | lut_lane);   // selectors x, y; byte masks of the flipped positions z, w
-    qa = (prmt_b32(pa, pb, e.x) & ~e.z) | (prmt_b32(na, nb, e.x) & e.z);   // a flipped zero stays zero
-    qb = (prmt_b32(pa, pb, e.y) & ~e.w) | (prmt_b32(na, nb, e.y) & e.w);
+    const uint4 e = lds128(((h >> 19) & 0x1F80u) | lut_lane);   // selectors x, y; ones at the flipped bytes z, w
+    za = e.z;
+    zb = e.w;
+    ra = prmt_b32(pa, pb, e.x) ^ (e.z * p.mul_255);
+    rb = prmt_b32(pa, pb, e.y) ^ (e.w * p.mul_255);
 }
 
 // first tile of linear `it` that belongs to CTA `cta` (tiles cta-congruent modulo the grid, numbered across linears)
@@ -164,7 +174,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
     for (int i = tid; i < 64 * kLutCopies; i += kConsumerWarps * 32) {
         const uint32_t* e = c_exchange_lut.v[i / kLutCopies];
         *reinterpret_cast<uint4*>(lut + (size_t)i * 16) =
-            I8 ? make_uint4(e[0], e[1], byte_mask(e[2]), byte_mask(e[3])) : make_uint4(e[0], e[1], e[2], e[3]);
+            I8 ? make_uint4(e[0], e[1], flip_ones(e[2]), flip_ones(e[3])) : make_uint4(e[0], e[1], e[2], e[3]);
     }
     const int g = lane >> 2, t = lane & 3;
     const uint32_t lut_lane = smem_u32(lut) + (lane & (kLutCopies - 1)) * 16;
@@ -276,17 +286,18 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
                     const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
                     const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
                     if constexpr (I8) {
-                        int s1[4] = {0, 0, 0, 0}, s2[4] = {0, 0, 0, 0};
+                        int s1[4] = {0, 0, 0, 0}, s2[4] = {0, 0, 0, 0}, s3[4] = {0, 0, 0, 0};
                         float rec0 = 0.f, rec2 = 0.f;   // this record's sums for token t: row g, row g+8
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             const uint2 xb = lds64(xrow_s + kb0 + c * 32);
-                            uint32_t pa0, pb0, qa0, qb0, pa1, pb1, qa1, qb1;
-                            decode_i8<WB>(w0[c], lut_lane, pa0, pb0, qa0, qb0);
-                            decode_i8<WB>(w1[c], lut_lane, pa1, pb1, qa1, qb1);
+                            uint32_t pa0, pb0, ra0, rb0, za0, zb0, pa1, pb1, ra1, rb1, za1, zb1;
+                            decode_i8<WB>(p, w0[c], lut_lane, pa0, pb0, ra0, rb0, za0, zb0);
+                            decode_i8<WB>(p, w1[c], lut_lane, pa1, pb1, ra1, rb1, za1, zb1);
                             // A fragment: a0/a1 = bytes k 0..3 of the micro-block for rows g / g+8, a2/a3 = bytes 4..7
                             mma_s8(s1, pa0, pa1, pb0, pb1, xb.x, xb.y);
-                            mma_s8(s2, qa0, qa1, qb0, qb1, xb.x, xb.y);
+                            mma_s8(s2, ra0, ra1, rb0, rb1, xb.x, xb.y);
+                            mma_s8(s3, za0, za1, zb0, zb1, xb.x, xb.y);
                             if (((c + 1) % CPG) == 0) {   // end of a macro-block: the coefficient multiply, outside the inner product
                                 const int jj = c / CPG;
                                 const uint32_t cfa = lds32(coef_addr + jj * 64), cfb = lds32(coef_addr + jj * 64 + 32);
@@ -295,10 +306,10 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
                                 const float c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
                                 const float c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
                                 // columns 2t, 2t+1 hold the high and low activation slices of token t: S = 256 S_hi + S_lo, exact in int32
-                                rec0 += c1a * (float)(s1[0] * 256 + s1[1]) + c2a * (float)(s2[0] * 256 + s2[1]);
-                                rec2 += c1b * (float)(s1[2] * 256 + s1[3]) + c2b * (float)(s2[2] * 256 + s2[3]);
+                                rec0 += c1a * (float)(s1[0] * 256 + s1[1]) + c2a * (float)((s2[0] + s3[0]) * 256 + s2[1] + s3[1]);
+                                rec2 += c1b * (float)(s1[2] * 256 + s1[3]) + c2b * (float)((s2[2] + s3[2]) * 256 + s2[3] + s3[3]);
 #pragma unroll
-                                for (int r = 0; r < 4; ++r) s1[r] = s2[r] = 0;
+                                for (int r = 0; r < 4; ++r) s1[r] = s2[r] = s3[r] = 0;
                             }
                         }
                         const float sv = xscale[(u0 + warp) * 4 + (t < it.m_total ? t : 0)];   // undo the activation scale of this k-block
@@ -459,6 +470,7 @@ cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, i
     p.unit_bytes = unit_bytes;
     p.status = (int*)wsb;
     p.done = (int*)(wsb + 256);
+    p.mul_255 = 255u;
     for (int i = 0; i < n; ++i) {
         seq::Item& it = p.item[i];
         it.packed = (const uint8_t*)calls[i].packed;
