@@ -511,9 +511,12 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
     xs = [torch.randn((m, s["k"]), device="cuda").to(torch.bfloat16) for s in layer0]
     ys = [torch.empty((m, s["n"]), dtype=torch.float32, device="cuda") for s in layer0]
 
+    ws_gemm = torch.empty(max(goq.workspace_bytes(s["d"], goq.OP_GEMM, m) for s in layer0), dtype=torch.uint8, device="cuda")
+    goq.workspace_init(ws_gemm)
+
     def step_gemm():
         for s, x, y in zip(layer0, xs, ys):
-            goq.gemm(s["d"], s["packed"], x, m, goq.BF16, y=y, y_dtype=goq.F32, ws=ws)
+            goq.gemm(s["d"], s["packed"], x, m, goq.BF16, y=y, y_dtype=goq.F32, ws=ws_gemm)
 
     step_gemm()
     torch.cuda.synchronize()
@@ -527,7 +530,23 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
     flops = sum(2.0 * m * s["n"] * s["k"] for s in layer0)
     out["gemm_m2048_layer_tflops"] = flops / (ms * 1e-3) / 1e12
     out["gemm_m2048_frac_of_bf16_peak"] = out["gemm_m2048_layer_tflops"] / tf_peak
-    del xs, ys
+    # the same layer with bf16 outputs (half the bytes of the epilogue's store burst)
+    yb = [torch.empty((m, s["n"]), dtype=torch.bfloat16, device="cuda") for s in layer0]
+
+    def step_gemm_bf16_out():
+        for s, x, y in zip(layer0, xs, yb):
+            goq.gemm(s["d"], s["packed"], x, m, goq.BF16, y=y, y_dtype=goq.BF16, ws=ws_gemm)
+
+    step_gemm_bf16_out()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(3):
+        step_gemm_bf16_out()
+    e1.record()
+    torch.cuda.synchronize()
+    out["gemm_m2048_layer_tflops_bf16_out"] = flops / (e0.elapsed_time(e1) / 3 * 1e-3) / 1e12
+    del yb
+    del xs, ys, ws_gemm
     # integer path: ViT-B/16-shaped linears, 197 x 64 tokens, W3 group 64, int8 activations and coefficients
     mt = si.VIT_B16_TOKENS
     vit = []

@@ -7,15 +7,19 @@
 //     128 k) and loads the 512 x 64 bf16 activation tile with two 2-D TMA copies (128-byte swizzle);
 //   - eight expander warps decode the records (same byte-table decode and record lookup as the GEMV:
 //     b1 from the code bytes, b2 = byte-permuted b1 with pair signs, Section 3.3), form
-//     w_hat = c1*b1 + c2*b2 in fp32, round once to bf16 and store the 128 x 64 operand tile to shared
+//     w_hat = c1*b1 + c2*b2 in fp32, round once to fp16 and store the 128 x 64 operand tile to shared
 //     memory in the K-major, 128-byte-swizzled layout the tensor core reads;
-//   - one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 x bf16 -> fp32) into a 128 x 512 fp32
+//   - one thread issues tcgen05.mma (M=128, N=256, K=16, fp16 x fp16 -> fp32) into a 128 x 512 fp32
 //     accumulator that fills the SM's tensor memory, and commits each stage back to the producers.
 // After the last chunk the warps read the accumulator with tcgen05.ld and store y.
-// bf16 keeps 8 significant bits, so one rounding of w_hat costs about 2e-3 normwise on the output
-// (measured), which is the whole error budget. The operand is therefore carried as two bf16 tiles,
-// w_hi = bf16(w_hat) and w_lo = bf16(w_hat - w_hi), multiplied against the same activation tile into the
-// same accumulator: w_hi + w_lo holds w_hat to about 2^-16, at the price of twice the tensor work.
+//
+// Operand precision. One rounding of w_hat to bf16 (8 significant bits) costs about 2e-3 normwise on the
+// output, the whole error budget; fp16 keeps 11 bits (about 2.5e-4) for the same tensor work, where a
+// bf16 hi + lo pair needs twice the MMAs. Both MMA operands must then be fp16, so a pre-pass rewrites
+// the bf16 activations as fp16, each token scaled by the power of two that puts its largest magnitude in
+// [2^14, 2^15): bf16's 8 significant bits are kept exactly, and only elements more than 2^-28 below the
+// token's largest lose bits to fp16's range (they vanish below 2^-39 of it). The epilogue undoes the scale.
+// |w_hat| above 65504 overflows to infinity (coefficients that large do not occur: they scale fp16 weights).
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, skips the remaining work,
 // still frees its tensor memory and records GOQ_ERR_TIMEOUT in the status word.
@@ -33,7 +37,7 @@ constexpr int kChunkK = 64;     // k per pipeline stage: 128 bytes of bf16 = one
 constexpr int kStages = 2;
 constexpr int kExpanders = 8;   // expander warps; each owns one 16-row unit record per k-block
 constexpr int kThreads = (2 + kExpanders) * 32;
-constexpr int kATileBytes = kTileN * kChunkK * 2;   // 16 KiB, one of the two operand tiles (hi, lo) of a stage
+constexpr int kATileBytes = kTileN * kChunkK * 2;   // 16 KiB, the weight operand tile of a stage
 constexpr int kBTileBytes = kTileM * kChunkK * 2;   // 64 KiB
 constexpr int kLutCopies = 1;   // the expanders are not the bottleneck here: one 1 KiB copy, bank conflicts accepted
 constexpr int kLutBytes = 64 * kLutCopies * 16;
@@ -96,9 +100,9 @@ __device__ __forceinline__ uint32_t after_wait(uint32_t addr) {
     asm volatile("mov.u32 %0, %1;" : "=r"(r) : "r"(addr) : "memory");
     return r;
 }
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
     uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
 
@@ -120,9 +124,9 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
     return d;
 }
-// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, M = 128, N = 256
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+// kind::f16 instruction descriptor: fp32 accumulate, fp16 x fp16 (format fields 0), both K-major, M = 128, N = 256
+constexpr uint32_t kIdesc = (1u << 4) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
@@ -145,12 +149,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 
 
 // ---- record decode (same tables as the decode GEMV) --------------------------------------------
+// High byte of the fp16 number of every PoT state, by code (the low byte of a power of two is zero).
 template <int WB> struct PotBytes;
-template <> struct PotBytes<3> {  // +1 +.5 +.25 0 -1 -.5 -.25 -.125 : bf16 high / low bytes by code
-    static constexpr uint32_t H0 = 0x003E3F3Fu, H1 = 0xBEBEBFBFu, L0 = 0x00800080u, L1 = 0x00800080u;
+template <> struct PotBytes<3> {  // +1 +.5 +.25 0 -1 -.5 -.25 -.125
+    static constexpr uint32_t H0 = 0x0034383Cu, H1 = 0xB0B4B8BCu;
 };
 template <> struct PotBytes<2> {  // +1 0 -1 -.5
-    static constexpr uint32_t H0 = 0xBFBF003Fu, H1 = 0u, L0 = 0x00800080u, L1 = 0u;
+    static constexpr uint32_t H0 = 0xB8BC003Cu, H1 = 0u;
 };
 constexpr uint32_t kHashMul = 0x01008420u;  // (record bits in place) * kHashMul >> 26 is a bijection onto 0..63
 
@@ -186,35 +191,38 @@ constexpr ExchangeLut make_exchange_lut() {
 }
 __constant__ ExchangeLut c_lut = make_exchange_lut();
 
-// eight weights of one micro-block -> w_hat = c1*b1 + c2*b2 as bf16 hi + bf16 lo, four bf16x2 words each
+__device__ __forceinline__ uint32_t hmul2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t hfma2(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t r;
+    asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    return r;
+}
+// Eight weights of one micro-block -> w_hat = c1*b1 + c2*b2 in fp16, four f16x2 words. c1, c2: the coefficient in both
+// halves of a register. b1 and b2 are built as fp16 directly (table high byte over a zero low byte), c1*b1 is a
+// power-of-two scaling (exact) and the fused multiply-add rounds once: the same value as fp32 arithmetic rounded
+// to fp16, for a quarter of the instructions.
 template <int WB>
-__device__ __forceinline__ void expand_what(uint32_t w, uint32_t lut_lane, float c1, float c2, uint32_t (&out_hi)[4],
-                                            uint32_t (&out_lo)[4]) {
+__device__ __forceinline__ void expand_what(uint32_t w, uint32_t lut_lane, uint32_t c1, uint32_t c2, uint32_t (&out)[4]) {
     const uint32_t m = w & 0x77777777u, mh = m >> 16;
     const uint32_t ha = prmt(PotBytes<WB>::H0, PotBytes<WB>::H1, m), hb = prmt(PotBytes<WB>::H0, PotBytes<WB>::H1, mh);
-    const uint32_t la = prmt(PotBytes<WB>::L0, PotBytes<WB>::L1, m), lb = prmt(PotBytes<WB>::L0, PotBytes<WB>::L1, mh);
     const uint32_t h = (w - m) * kHashMul;
     const uint4 e = lds128(((h >> 22) & 0x3F0u) | lut_lane);  // table is 1 KiB aligned
-    const uint32_t qha = prmt(ha, hb, e.x) ^ e.z, qhb = prmt(ha, hb, e.y) ^ e.w;
-    const uint32_t qla = prmt(la, lb, e.x), qlb = prmt(la, lb, e.y);
-    uint32_t R[4], Q[4];
-    R[0] = prmt(la, ha, 0x5140u); R[1] = prmt(la, ha, 0x7362u); R[2] = prmt(lb, hb, 0x5140u); R[3] = prmt(lb, hb, 0x7362u);
-    Q[0] = prmt(qla, qha, 0x5140u); Q[1] = prmt(qla, qha, 0x7362u); Q[2] = prmt(qlb, qhb, 0x5140u); Q[3] = prmt(qlb, qhb, 0x7362u);
+    const uint32_t qa = prmt(ha, hb, e.x) ^ e.z, qb = prmt(ha, hb, e.y) ^ e.w;   // b2: permuted, pair signs applied
+    // bytes {0, h[2q], 0, h[2q+1]}: weights 2q, 2q+1 as one f16x2 word
+    const uint32_t R[4] = {prmt(ha, 0u, 0x1404u), prmt(ha, 0u, 0x3424u), prmt(hb, 0u, 0x1404u), prmt(hb, 0u, 0x3424u)};
+    const uint32_t Q[4] = {prmt(qa, 0u, 0x1404u), prmt(qa, 0u, 0x3424u), prmt(qb, 0u, 0x1404u), prmt(qb, 0u, 0x3424u)};
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const float b1lo = __uint_as_float(R[q] << 16), b1hi = __uint_as_float(R[q] & 0xFFFF0000u);
-        const float b2lo = __uint_as_float(Q[q] << 16), b2hi = __uint_as_float(Q[q] & 0xFFFF0000u);
-        const float wlo = fmaf(c2, b2lo, c1 * b1lo), whi = fmaf(c2, b2hi, c1 * b1hi);
-        const uint32_t h2 = pack_bf16x2(wlo, whi);
-        out_hi[q] = h2;
-        // residual of the rounding, exact in fp32, rounded to bf16 itself
-        out_lo[q] = pack_bf16x2(wlo - __uint_as_float(h2 << 16), whi - __uint_as_float(h2 & 0xFFFF0000u));
-    }
+    for (int q = 0; q < 4; ++q) out[q] = hfma2(c2, Q[q], hmul2(c1, R[q]));
 }
 
 struct GemmParams {
     const uint8_t* packed;
     void* y;
+    const float* inv_scale;   // [m_total] 2^-s of each token (the activations the tensor map covers are x * 2^s in fp16)
     int* status;
     int unit_bytes, k_blocks, n_tiles, n_out, m_total, y_dtype, group_log2;
 };
@@ -226,7 +234,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
     unsigned char* base = smem_raw + ((1024u - (s32(smem_raw) & 1023u)) & 1023u);  // 1 KiB boundary
     unsigned char* lut = base;
     unsigned char* a_tiles = lut + kLutBytes;
-    unsigned char* b_tiles = a_tiles + kStages * 2 * kATileBytes;
+    unsigned char* b_tiles = a_tiles + kStages * kATileBytes;
     unsigned char* pk_ring = b_tiles + kStages * kBTileBytes;
     const int pk_slot_bytes = kExpanders * p.unit_bytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(pk_ring + 2 * pk_slot_bytes);
@@ -236,7 +244,9 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
     uint64_t* pk_full = bars + 6;       // [2] packed records landed
     uint64_t* pk_empty = bars + 8;      // [2] expanders finished with the records
     uint64_t* tmem_full = bars + 10;    // accumulator complete
+    uint64_t* epi_bar = bars + 11;      // [2] epilogue rendezvous of the four warps of a token half
     __shared__ uint32_t tmem_base_slot;
+    __shared__ __align__(16) float inv_s[kTileM];   // 2^-s of this CTA's tokens (1 for tokens past the end)
     __shared__ volatile int abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -249,12 +259,15 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&full_b[i], 1); mbar_init(&full_a[i], kExpanders); mbar_init(&empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], kExpanders); }
         mbar_init(tmem_full, 1);
+        mbar_init(&epi_bar[0], 4);
+        mbar_init(&epi_bar[1], 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < 64 * kLutCopies; i += kThreads) {
         const uint32_t* e = c_lut.v[i / kLutCopies];
         *reinterpret_cast<uint4*>(lut + (size_t)i * 16) = make_uint4(e[0], e[1], e[2], e[3]);
     }
+    for (int i = tid; i < kTileM; i += kThreads) inv_s[i] = (tok0 + i < p.m_total) ? __ldg(&p.inv_scale[tok0 + i]) : 1.0f;
     if (warp == 1) tmem_alloc_512(&tmem_base_slot);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -305,17 +318,14 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                 ok = mbar_wait(&full_b[s], par, &abort_flag) && mbar_wait(&full_a[s], par, &abort_flag);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint64_t ahi = smem_desc_sw128(s32(a_tiles + s * 2 * kATileBytes));
-                const uint64_t alo = smem_desc_sw128(s32(a_tiles + s * 2 * kATileBytes + kATileBytes));
+                const uint64_t adesc = smem_desc_sw128(s32(a_tiles + s * kATileBytes));
                 const uint64_t bdesc0 = smem_desc_sw128(s32(b_tiles + s * kBTileBytes));
                 const uint64_t bdesc1 = smem_desc_sw128(s32(b_tiles + s * kBTileBytes + kBTileBytes / 2));
 #pragma unroll
                 for (int ks = 0; ks < kChunkK / 16; ++ks) {
                     const uint32_t acc = (chunk > 0 || ks > 0) ? 1u : 0u;
-                    umma_bf16(tmem_base, ahi + 2 * ks, bdesc0 + 2 * ks, acc);         // tokens   0..255
-                    umma_bf16(tmem_base + 256, ahi + 2 * ks, bdesc1 + 2 * ks, acc);   // tokens 256..511
-                    umma_bf16(tmem_base, alo + 2 * ks, bdesc0 + 2 * ks, 1u);
-                    umma_bf16(tmem_base + 256, alo + 2 * ks, bdesc1 + 2 * ks, 1u);
+                    umma_f16(tmem_base, adesc + 2 * ks, bdesc0 + 2 * ks, acc);         // tokens   0..255
+                    umma_f16(tmem_base + 256, adesc + 2 * ks, bdesc1 + 2 * ks, acc);   // tokens 256..511
                 }
                 umma_commit(&empty[s]);
             }
@@ -341,31 +351,27 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                 const int chunk = 2 * kb + half, s = chunk % kStages;
                 if (chunk >= kStages) ok = __all_sync(0xFFFFFFFFu, mbar_wait(&empty[s], ((chunk / kStages) - 1) & 1, &abort_flag));
                 if (!ok) break;
-                const uint32_t a_tile = s32(a_tiles + s * 2 * kATileBytes);
+                const uint32_t a_tile = s32(a_tiles + s * kATileBytes);
 #pragma unroll
                 for (int cc = 0; cc < 2; ++cc) {
                     const int c = half * 2 + cc;
                     const int jj = (c * 32 + t * 8) >> p.group_log2;  // macro-block of this micro-block inside the k-block
-                    float c1a = 0.f, c2a = 0.f, c1b = 0.f, c2b = 0.f;
+                    uint32_t cfa = 0u, cfb = 0u;   // {c1, c2} as stored: fp16 pairs
                     if (valid) {
-                        const uint32_t cfa = lds32(unit + kCodeBytesPerUnit + (jj * 16 + g) * 4);
-                        const uint32_t cfb = lds32(unit + kCodeBytesPerUnit + (jj * 16 + 8 + g) * 4);
-                        c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
-                        c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
-                        c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
-                        c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
+                        cfa = lds32(unit + kCodeBytesPerUnit + (jj * 16 + g) * 4);
+                        cfb = lds32(unit + kCodeBytesPerUnit + (jj * 16 + 8 + g) * 4);
                     }
-                    uint32_t oa[4], ob[4], la[4], lb[4];
-                    expand_what<WB>(w0[c], lut_lane, c1a, c2a, oa, la);
-                    expand_what<WB>(w1[c], lut_lane, c1b, c2b, ob, lb);
+                    const uint32_t c1a = prmt(cfa, cfa, 0x1010u), c2a = prmt(cfa, cfa, 0x3232u);
+                    const uint32_t c1b = prmt(cfb, cfb, 0x1010u), c2b = prmt(cfb, cfb, 0x3232u);
+                    uint32_t oa[4], ob[4];
+                    expand_what<WB>(w0[c], lut_lane, c1a, c2a, oa);
+                    expand_what<WB>(w1[c], lut_lane, c1b, c2b, ob);
                     // K-major tile, 128-byte rows, 16-byte chunk j of row r stored at chunk j ^ (r & 7)
                     const int j = cc * 4 + t;
                     const int ra = e * 16 + g, rb = ra + 8;  // (ra & 7) == (rb & 7) == g
                     const uint32_t off = (uint32_t)((j ^ g) << 4);
                     sts128(a_tile + ra * 128 + off, oa[0], oa[1], oa[2], oa[3]);
                     sts128(a_tile + rb * 128 + off, ob[0], ob[1], ob[2], ob[3]);
-                    sts128(a_tile + kATileBytes + ra * 128 + off, la[0], la[1], la[2], la[3]);
-                    sts128(a_tile + kATileBytes + rb * 128 + off, lb[0], lb[1], lb[2], lb[3]);
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> tensor-core reads
                 __syncwarp();
@@ -379,20 +385,58 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
         ok = __all_sync(0xFFFFFFFFu, ok);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok) {
+            // Each thread holds one output channel (a TMEM lane) for 32 tokens; stored directly that is one 4-byte store
+            // per token and thread, 2048 128-byte requests per CTA, and the request rate of that burst, not its bytes,
+            // set the epilogue's time. So the four warps of a token half transpose 32 tokens x 128 channels through
+            // shared memory (the activation ring is idle by now) and store 16 bytes per thread: a quarter of the requests.
             const int q = warp & 3, col_half = (e >= 4) ? 1 : 0;
-            const int row = blockIdx.x * kTileN + q * 32 + lane;
+            const int row4 = blockIdx.x * kTileN + 4 * lane;
+            const bool f32 = p.y_dtype == GOQ_F32;
+            const bool vec = (blockIdx.x + 1) * kTileN <= p.n_out && (p.n_out & 3) == 0 &&
+                             (reinterpret_cast<uintptr_t>(p.y) & (f32 ? 15u : 7u)) == 0;
 #pragma unroll 1
-            for (int cb = 0; cb < 8; ++cb) {
+            for (int cb = 0; cb < 8 && ok; ++cb) {
                 uint32_t v[32];
                 const int col0 = col_half * 256 + cb * 32;
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)col0, v);
-                if (row < p.n_out) {
+                float* st = reinterpret_cast<float*>(b_tiles) + (col_half * 2 + (cb & 1)) * (32 * kTileN);
 #pragma unroll
-                    for (int jx = 0; jx < 32; ++jx) {
-                        const int tok = tok0 + col0 + jx;
-                        if (tok < p.m_total) {
-                            if (p.y_dtype == GOQ_F32) reinterpret_cast<float*>(p.y)[(size_t)tok * p.n_out + row] = __uint_as_float(v[jx]);
-                            else reinterpret_cast<uint16_t*>(p.y)[(size_t)tok * p.n_out + row] = f32_to_bf16_rne(__uint_as_float(v[jx]));
+                for (int j4 = 0; j4 < 8; ++j4) {   // the 32 tokens' inverse scales: eight broadcast 16-byte loads
+                    const float4 f = *reinterpret_cast<const float4*>(&inv_s[col0 + 4 * j4]);
+                    st[(4 * j4 + 0) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 0]) * f.x;
+                    st[(4 * j4 + 1) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 1]) * f.y;
+                    st[(4 * j4 + 2) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 2]) * f.z;
+                    st[(4 * j4 + 3) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 3]) * f.w;
+                }
+                // bounded rendezvous of the half's four warps (a named barrier could not give up)
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&epi_bar[col_half]);
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&epi_bar[col_half], cb & 1, &abort_flag));
+                if (!ok) break;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int jt = q * 8 + i, tok = tok0 + col0 + jt;
+                    if (tok >= p.m_total) continue;
+                    const float4 f = *reinterpret_cast<const float4*>(&st[jt * kTileN + 4 * lane]);
+                    const size_t o = (size_t)tok * p.n_out + row4;
+                    if (f32) {
+                        float* y = reinterpret_cast<float*>(p.y);
+                        if (vec) *reinterpret_cast<float4*>(y + o) = f;
+                        else {
+                            if (row4 + 0 < p.n_out) y[o + 0] = f.x;
+                            if (row4 + 1 < p.n_out) y[o + 1] = f.y;
+                            if (row4 + 2 < p.n_out) y[o + 2] = f.z;
+                            if (row4 + 3 < p.n_out) y[o + 3] = f.w;
+                        }
+                    } else {
+                        uint16_t* y = reinterpret_cast<uint16_t*>(p.y);
+                        const uint16_t h0 = f32_to_bf16_rne(f.x), h1 = f32_to_bf16_rne(f.y), h2 = f32_to_bf16_rne(f.z), h3 = f32_to_bf16_rne(f.w);
+                        if (vec) *reinterpret_cast<uint2*>(y + o) = make_uint2((uint32_t)h0 | ((uint32_t)h1 << 16), (uint32_t)h2 | ((uint32_t)h3 << 16));
+                        else {
+                            if (row4 + 0 < p.n_out) y[o + 0] = h0;
+                            if (row4 + 1 < p.n_out) y[o + 1] = h1;
+                            if (row4 + 2 < p.n_out) y[o + 2] = h2;
+                            if (row4 + 3 < p.n_out) y[o + 3] = h3;
                         }
                     }
                 }
@@ -408,6 +452,45 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
     if (tid == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
 }
 
+
+// ---- activation pre-pass: bf16 -> scaled fp16, one CTA per token ------------------------------------
+// xh[tok][k] = fp16(x[tok][k] * 2^s), inv_scale[tok] = 2^-s, s chosen from the exponent field of the token's largest
+// magnitude (an all-zero token gets the largest scale, harmlessly; inf / nan stay inf / nan).
+constexpr int kPrepThreads = 256;
+__global__ void __launch_bounds__(kPrepThreads) x_to_f16_kernel(const uint16_t* __restrict__ x, int k_in, uint16_t* __restrict__ xh,
+                                                                float* __restrict__ inv_scale) {
+    const int tok = blockIdx.x, tid = threadIdx.x;
+    const uint4* row = reinterpret_cast<const uint4*>(x + (size_t)tok * k_in);
+    uint4* out = reinterpret_cast<uint4*>(xh + (size_t)tok * k_in);
+    const int n_vec = k_in / 8;   // k_in is a multiple of 8 (checked by the launcher)
+    __shared__ uint32_t warp_max[kPrepThreads / 32];
+    uint32_t amax = 0;
+    for (int i = tid; i < n_vec; i += kPrepThreads) {
+        const uint4 v = __ldg(&row[i]);
+        const uint32_t in32[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) amax = max(amax, max(in32[j] & 0x7FFFu, (in32[j] >> 16) & 0x7FFFu));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+    if ((tid & 31) == 0) warp_max[tid >> 5] = amax;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kPrepThreads / 32; ++w) amax = max(amax, warp_max[w]);
+    int sfield = 268 - (int)(amax >> 7);   // exponent field of 2^s: the largest magnitude lands in [2^14, 2^15)
+    sfield = sfield < 1 ? 1 : (sfield > 253 ? 253 : sfield);
+    const float mult = __uint_as_float((uint32_t)sfield << 23);
+    for (int i = tid; i < n_vec; i += kPrepThreads) {
+        const uint4 v = __ldg(&row[i]);
+        const uint32_t in32[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o32[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            o32[j] = pack_f16x2(__uint_as_float(in32[j] << 16) * mult, __uint_as_float(in32[j] & 0xFFFF0000u) * mult);
+        out[i] = make_uint4(o32[0], o32[1], o32[2], o32[3]);
+    }
+    if (tid == 0) inv_scale[tok] = __uint_as_float((uint32_t)(254 - sfield) << 23);
+}
 
 // ---- host side ------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -426,21 +509,23 @@ static EncodeTiledFn encode_tiled_fn() {
 }
 
 static size_t smem_bytes(const Geometry& g) {
-    return 1024 /* alignment slack */ + kLutBytes + (size_t)kStages * (2 * kATileBytes + kBTileBytes) +
+    return 1024 /* alignment slack */ + kLutBytes + (size_t)kStages * (kATileBytes + kBTileBytes) +
            (size_t)2 * kExpanders * g.unit_bytes + 16 * sizeof(uint64_t);
 }
 
 template <int WB>
 static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* x, int m, void* y, int y_dtype, int* status,
-                             cudaStream_t st) {
+                             float* inv_scale, uint16_t* xh, cudaStream_t st) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return cudaErrorNotSupported;
+    if (g.k_in % 8 != 0) return cudaErrorInvalidValue;
+    x_to_f16_kernel<<<m, kPrepThreads, 0, st>>>((const uint16_t*)x, g.k_in, xh, inv_scale);
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)g.k_in, (cuuint64_t)m};
     const cuuint64_t strides[1] = {(cuuint64_t)g.k_in * 2};
     const cuuint32_t box[2] = {(cuuint32_t)kChunkK, 256};
     const cuuint32_t estr[2] = {1, 1};
-    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, xh, dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidTexture;  // distinct code: the tensor map could not be encoded
@@ -454,6 +539,7 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
     GemmParams p;
     p.packed = (const uint8_t*)packed;
     p.y = y;
+    p.inv_scale = inv_scale;
     p.status = status;
     p.unit_bytes = g.unit_bytes;
     p.k_blocks = g.k_blocks;
@@ -474,11 +560,19 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
 
 namespace goq {
 bool gemm_tc_supported(const Geometry& g) { return g.wbits <= 3 && tc::smem_bytes(g) + 2048 <= 227 * 1024; }
-size_t gemm_tc_workspace(const Geometry&) { return 256; }  // status word
+// Scratch: [0, base) is left to the other kernels that may share the buffer (status word at 0, their zeroed counters);
+// then the per-token inverse scales and the fp16 copy of the activations.
+static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+size_t gemm_tc_workspace(const Geometry& g, int m, size_t base) {
+    return align256(base < 256 ? 256 : base) + align256((size_t)m * sizeof(float)) + (size_t)m * g.k_in * 2;
+}
 cudaError_t launch_gemm_tc(const Geometry& g, const void* packed, const void* x, int m, void* y, int y_dtype, void* ws,
-                           cudaStream_t st) {
+                           size_t base, cudaStream_t st) {
     int* status = (int*)ws;
-    return g.wbits == 3 ? tc::launch_wb<3>(g, packed, x, m, y, y_dtype, status, st)
-                        : tc::launch_wb<2>(g, packed, x, m, y, y_dtype, status, st);
+    uint8_t* b = (uint8_t*)ws + align256(base < 256 ? 256 : base);
+    float* inv_scale = (float*)b;
+    uint16_t* xh = (uint16_t*)(b + align256((size_t)m * sizeof(float)));
+    return g.wbits == 3 ? tc::launch_wb<3>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, st)
+                        : tc::launch_wb<2>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, st);
 }
 }  // namespace goq
