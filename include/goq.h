@@ -125,6 +125,11 @@ goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16
 
 /* goq_gemm - the same layer for m activation rows.
  *  x_dtype GOQ_BF16: x [m][k_in] bf16; y out [m][n_out] (GOQ_BF16 or GOQ_F32); sx, cq, sc, acc unused (NULL).
+ *      ws: goq_workspace_bytes(desc, GOQ_OP_GEMM, m) bytes, 256-byte aligned, initialised once with
+ *      goq_workspace_init. From 65 rows on (W <= 3) the tensor-core kernel runs: it keeps an fp16 copy of x
+ *      (each row scaled by a power of two, undone in the output) in ws, so the size grows with m * k_in, and it
+ *      rounds c1*b1 + c2*b2 once to fp16 (normwise output error about 1.5e-4; |c1*b1 + c2*b2| must stay below
+ *      65504).
  *  x_dtype GOQ_I8 (Eq. 4 with integer X~ and c~; left shifts x~ << (emax-e), exact int32):
  *      x    [m][k_in] int8         sx [m] fp32 per-token scale
  *      cq   [n_out][k_in/group][2] int8 integer coefficients,  sc [n_out][2] fp32 their per-channel scales

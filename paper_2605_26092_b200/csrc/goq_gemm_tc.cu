@@ -39,7 +39,8 @@ constexpr int kExpanders = 8;   // expander warps; each owns one 16-row unit rec
 constexpr int kThreads = (2 + kExpanders) * 32;
 constexpr int kATileBytes = kTileN * kChunkK * 2;   // 16 KiB, the weight operand tile of a stage
 constexpr int kBTileBytes = kTileM * kChunkK * 2;   // 64 KiB
-constexpr int kLutCopies = 1;   // the expanders are not the bottleneck here: one 1 KiB copy, bank conflicts accepted
+constexpr int kLutCopies = 8;   // record table, one copy per lane & 7: lookups are bank-conflict free (shared-memory
+                                // bandwidth, shared with the tensor core's operand reads, bounds this kernel)
 constexpr int kLutBytes = 64 * kLutCopies * 16;
 constexpr int kSpin = 1 << 22;
 
@@ -210,7 +211,7 @@ __device__ __forceinline__ void expand_what(uint32_t w, uint32_t lut_lane, uint3
     const uint32_t m = w & 0x77777777u, mh = m >> 16;
     const uint32_t ha = prmt(PotBytes<WB>::H0, PotBytes<WB>::H1, m), hb = prmt(PotBytes<WB>::H0, PotBytes<WB>::H1, mh);
     const uint32_t h = (w - m) * kHashMul;
-    const uint4 e = lds128(((h >> 22) & 0x3F0u) | lut_lane);  // table is 1 KiB aligned
+    const uint4 e = lds128(((h >> 19) & 0x1F80u) | lut_lane);  // table is 8 KiB aligned, lut_lane selects the copy
     const uint32_t qa = prmt(ha, hb, e.x) ^ e.z, qb = prmt(ha, hb, e.y) ^ e.w;   // b2: permuted, pair signs applied
     // bytes {0, h[2q], 0, h[2q+1]}: weights 2q, 2q+1 as one f16x2 word
     const uint32_t R[4] = {prmt(ha, 0u, 0x1404u), prmt(ha, 0u, 0x3424u), prmt(hb, 0u, 0x1404u), prmt(hb, 0u, 0x3424u)};
@@ -225,13 +226,17 @@ struct GemmParams {
     const float* inv_scale;   // [m_total] 2^-s of each token (the activations the tensor map covers are x * 2^s in fp16)
     int* status;
     int unit_bytes, k_blocks, n_tiles, n_out, m_total, y_dtype, group_log2;
+    // Tile schedule (1-D grid). CTAs [0, n_full) take 128 x 512 tiles, numbered channel-tile fastest; the remaining
+    // CTAs take the last tiles as halves of 256 tokens each, so that a last wave that would fill less than half of
+    // the SMs runs for half as long on twice as many.
+    int n_full, n_tiles_x;
 };
 
 template <int WB>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    unsigned char* base = smem_raw + ((1024u - (s32(smem_raw) & 1023u)) & 1023u);  // 1 KiB boundary
+    unsigned char* base = smem_raw + ((8192u - (s32(smem_raw) & 8191u)) & 8191u);  // 8 KiB boundary: table offsets are OR-ed in
     unsigned char* lut = base;
     unsigned char* a_tiles = lut + kLutBytes;
     unsigned char* b_tiles = a_tiles + kStages * kATileBytes;
@@ -250,8 +255,12 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
     __shared__ volatile int abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int T0 = blockIdx.x * (kTileN / kTileRows);  // first 16-row tile of this CTA
-    const int tok0 = blockIdx.y * kTileM;
+    const int bid = blockIdx.x;
+    const int tile = bid < p.n_full ? bid : p.n_full + ((bid - p.n_full) >> 1);
+    const int n_half = bid < p.n_full ? 2 : 1;   // token halves (of 256) this CTA computes
+    const int tile_x = tile % p.n_tiles_x;
+    const int T0 = tile_x * (kTileN / kTileRows);  // first 16-row tile of this CTA
+    const int tok0 = (tile / p.n_tiles_x) * kTileM + (bid < p.n_full ? 0 : ((bid - p.n_full) & 1) * 256);
     const int n_chunks = 2 * p.k_blocks;
 
     if (tid == 0) {
@@ -295,9 +304,10 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                     if (chunk >= kStages) ok = mbar_wait(&empty[s], ((chunk / kStages) - 1) & 1, &abort_flag);
                     if (!ok) break;
                     b_issued = chunk + 1;
-                    mbar_expect_tx(&full_b[s], kBTileBytes);
+                    mbar_expect_tx(&full_b[s], (uint32_t)n_half * (kBTileBytes / 2));
                     tma_load_2d(b_tiles + s * kBTileBytes, &x_map, chunk * kChunkK, tok0, &full_b[s]);
-                    tma_load_2d(b_tiles + s * kBTileBytes + kBTileBytes / 2, &x_map, chunk * kChunkK, tok0 + 256, &full_b[s]);
+                    if (n_half == 2)
+                        tma_load_2d(b_tiles + s * kBTileBytes + kBTileBytes / 2, &x_map, chunk * kChunkK, tok0 + 256, &full_b[s]);
                 }
             }
             if (!ok || abort_flag) {
@@ -325,7 +335,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                 for (int ks = 0; ks < kChunkK / 16; ++ks) {
                     const uint32_t acc = (chunk > 0 || ks > 0) ? 1u : 0u;
                     umma_f16(tmem_base, adesc + 2 * ks, bdesc0 + 2 * ks, acc);         // tokens   0..255
-                    umma_f16(tmem_base + 256, adesc + 2 * ks, bdesc1 + 2 * ks, acc);   // tokens 256..511
+                    if (n_half == 2) umma_f16(tmem_base + 256, adesc + 2 * ks, bdesc1 + 2 * ks, acc);   // tokens 256..511
                 }
                 umma_commit(&empty[s]);
             }
@@ -334,7 +344,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
     } else {
         // ------------------------------ expanders, then epilogue ------------------------------
         const int e = warp - 2, g = lane >> 2, t = lane & 3;
-        const uint32_t lut_lane = s32(lut);
+        const uint32_t lut_lane = s32(lut) + (uint32_t)(lane & (kLutCopies - 1)) * 16;
         const bool valid = (T0 + e) < p.n_tiles;
         constexpr uint32_t kZeroWord = (WB == 3) ? 0x33333333u : 0x11111111u;  // every code = the zero state
         bool ok = true;
@@ -353,8 +363,13 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                 if (!ok) break;
                 const uint32_t a_tile = s32(a_tiles + s * kATileBytes);
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
+                for (int cci = 0; cci < 2; ++cci) {
+                    // odd rows take the chunk's two 32-wide slices in the other order: the eight lanes of a quarter warp
+                    // (two rows) then store to all eight 16-byte columns of the swizzled rows instead of four, twice
+                    const int cc = cci ^ (g & 1);
                     const int c = half * 2 + cc;
+                    const uint32_t wa = (g & 1) ? w0[half * 2 + (cci ^ 1)] : w0[half * 2 + cci];
+                    const uint32_t wb = (g & 1) ? w1[half * 2 + (cci ^ 1)] : w1[half * 2 + cci];
                     const int jj = (c * 32 + t * 8) >> p.group_log2;  // macro-block of this micro-block inside the k-block
                     uint32_t cfa = 0u, cfb = 0u;   // {c1, c2} as stored: fp16 pairs
                     if (valid) {
@@ -364,8 +379,8 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                     const uint32_t c1a = prmt(cfa, cfa, 0x1010u), c2a = prmt(cfa, cfa, 0x3232u);
                     const uint32_t c1b = prmt(cfb, cfb, 0x1010u), c2b = prmt(cfb, cfb, 0x3232u);
                     uint32_t oa[4], ob[4];
-                    expand_what<WB>(w0[c], lut_lane, c1a, c2a, oa);
-                    expand_what<WB>(w1[c], lut_lane, c1b, c2b, ob);
+                    expand_what<WB>(wa, lut_lane, c1a, c2a, oa);
+                    expand_what<WB>(wb, lut_lane, c1b, c2b, ob);
                     // K-major tile, 128-byte rows, 16-byte chunk j of row r stored at chunk j ^ (r & 7)
                     const int j = cc * 4 + t;
                     const int ra = e * 16 + g, rb = ra + 8;  // (ra & 7) == (rb & 7) == g
@@ -384,15 +399,15 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
         if (ok) ok = mbar_wait(tmem_full, 0, &abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok) {
+        if (ok && (e < 4 || n_half == 2)) {
             // Each thread holds one output channel (a TMEM lane) for 32 tokens; stored directly that is one 4-byte store
             // per token and thread, 2048 128-byte requests per CTA, and the request rate of that burst, not its bytes,
             // set the epilogue's time. So the four warps of a token half transpose 32 tokens x 128 channels through
             // shared memory (the activation ring is idle by now) and store 16 bytes per thread: a quarter of the requests.
             const int q = warp & 3, col_half = (e >= 4) ? 1 : 0;
-            const int row4 = blockIdx.x * kTileN + 4 * lane;
+            const int row4 = tile_x * kTileN + 4 * lane;
             const bool f32 = p.y_dtype == GOQ_F32;
-            const bool vec = (blockIdx.x + 1) * kTileN <= p.n_out && (p.n_out & 3) == 0 &&
+            const bool vec = (tile_x + 1) * kTileN <= p.n_out && (p.n_out & 3) == 0 &&
                              (reinterpret_cast<uintptr_t>(p.y) & (f32 ? 15u : 7u)) == 0;
 #pragma unroll 1
             for (int cb = 0; cb < 8 && ok; ++cb) {
@@ -509,7 +524,7 @@ static EncodeTiledFn encode_tiled_fn() {
 }
 
 static size_t smem_bytes(const Geometry& g) {
-    return 1024 /* alignment slack */ + kLutBytes + (size_t)kStages * (kATileBytes + kBTileBytes) +
+    return 8192 /* alignment slack */ + kLutBytes + (size_t)kStages * (kATileBytes + kBTileBytes) +
            (size_t)2 * kExpanders * g.unit_bytes + 16 * sizeof(uint64_t);
 }
 
@@ -550,8 +565,18 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
     int lg = 3;
     while ((1 << lg) < g.group) ++lg;
     p.group_log2 = lg;
-    dim3 grid((g.n_pad + kTileN - 1) / kTileN, (m + kTileM - 1) / kTileM);
-    gemm_tc_kernel<WB><<<grid, kThreads, smem, st>>>(p, map);
+    const int tiles_x = (g.n_pad + kTileN - 1) / kTileN, tiles = tiles_x * ((m + kTileM - 1) / kTileM);
+    static int sm_count = 0;
+    if (sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            sm_count = 148;
+    }
+    const int tail = tiles % sm_count;   // tiles of the last, partial wave
+    const int split = (tiles > sm_count && tail > 0 && 2 * tail <= sm_count) ? tail : 0;
+    p.n_tiles_x = tiles_x;
+    p.n_full = tiles - split;
+    gemm_tc_kernel<WB><<<p.n_full + 2 * split, kThreads, smem, st>>>(p, map);
     return cudaGetLastError();
 }
 
@@ -559,7 +584,7 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
 }  // namespace goq
 
 namespace goq {
-bool gemm_tc_supported(const Geometry& g) { return g.wbits <= 3 && tc::smem_bytes(g) + 2048 <= 227 * 1024; }
+bool gemm_tc_supported(const Geometry& g) { return g.wbits <= 3 && g.k_in % 8 == 0 && tc::smem_bytes(g) + 2048 <= 227 * 1024; }
 // Scratch: [0, base) is left to the other kernels that may share the buffer (status word at 0, their zeroed counters);
 // then the per-token inverse scales and the fp16 copy of the activations.
 static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }

@@ -237,6 +237,22 @@ def test_config4_prefill_2048_tokens_sampled_rows(goq):
     assert O.normwise_rel_err(y[:, rows], y_ref) <= TOL
 
 
+def test_gemm_tail_wave_runs_as_half_tiles(goq):
+    """160 output tiles (20 channel tiles x 8 token tiles) on 148 SMs: the 12 tiles of the last wave are scheduled
+    as 24 half tiles of 256 tokens; 3900 tokens make the last token tile ragged. Sampled channels, all tokens."""
+    from tests.gpu_util import pack_weights, run_gemm_bf16
+    n, k, m = 2560, 256, 3900
+    codes, meta, coef = si.random_quantized(n, k, 64, 3, seed=41)
+    rows = np.unique(np.concatenate([si.sample_rows(n, 48, seed=4), np.arange(n - 130, n)]))   # the split tiles are the last ones
+    d, packed = pack_weights(n, k, 64, 3, codes, meta, coef)
+    xb = si.bf16_activations(m, k, seed=42)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 64, 3, rows=rows)
+    y = run_gemm_bf16(d, packed, xb)
+    assert O.normwise_rel_err(y[:, rows], y_ref) <= GEMM_TC_TOL
+    # every token of the ragged last tile, channel by channel
+    assert np.max(np.abs(y[3584:, rows] - y_ref[3584:])) <= 5e-3 * np.max(np.abs(y_ref))
+
+
 # ------------------------------------------------------------------------------------- integer path
 @pytest.mark.parametrize("n,k,g,b,m", [(48, 256, 64, 3, 200), (20, 192, 32, 2, 130), (16, 128, 128, 3, 1),
                                        (40, 128, 16, 3, 70), (200, 384, 128, 3, 333)])
