@@ -237,6 +237,35 @@ def test_config4_prefill_2048_tokens_sampled_rows(goq):
     assert O.normwise_rel_err(y[:, rows], y_ref) <= TOL
 
 
+def test_gemm_token_scaling_extreme_activations(goq):
+    """The tcgen05 GEMM feeds fp16 activations scaled per token by a power of two. Tokens of very different
+    magnitude (2^100, 2^-100), an all-zero token, a token whose elements span 2^24 and one with many zeros must
+    all come out at the kernel's usual accuracy, each token judged on its own norm."""
+    from tests.gpu_util import pack_weights, run_gemm_bf16
+    n, k, m, g, b = 144, 512, 200, 64, 3
+    codes, meta, coef = _quantized(n, k, g, b, seed=51)
+    d, packed = pack_weights(n, k, g, b, codes, meta, coef)
+    x = si.bf16_bits_to_f64(si.bf16_activations(m, k, seed=52))
+    x[3] *= 2.0 ** 100
+    x[4] *= 2.0 ** -100
+    x[5] = 0.0
+    x[6, ::2] *= 2.0 ** 24       # half of the token 2^24 above the rest: the small half is still above 2^-28 of the largest
+    x[7, 1::3] = 0.0
+    x[8, :] = 0.0
+    x[8, 17] = -3.0              # a single non-zero element
+    xb = si.f32_to_bf16_bits(x.astype(np.float32))
+    xr = si.bf16_bits_to_f64(xb)
+    y_ref = O.linear_f64(codes, meta, coef, xr, g, b)
+    y = run_gemm_bf16(d, packed, xb)
+    assert np.all(np.isfinite(y))
+    assert np.all(y[5] == 0.0)
+    for tok in range(m):
+        if tok == 5:
+            continue
+        e = np.linalg.norm(y[tok] - y_ref[tok]) / np.linalg.norm(y_ref[tok])
+        assert e <= GEMM_TC_TOL, (tok, e)
+
+
 def test_gemm_tail_wave_runs_as_half_tiles(goq):
     """160 output tiles (20 channel tiles x 8 token tiles) on 148 SMs: the 12 tiles of the last wave are scheduled
     as 24 half tiles of 256 tokens; 3900 tokens make the last token tile ragged. Sampled channels, all tokens."""
