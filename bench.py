@@ -469,42 +469,6 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
         shapes[(n, k)] = {"us": us, "gbs": algorithmic_bytes(n, k, 1) / (us * 1e-6) / 1e9}
         del g
     out["gemv_batch1_per_shape"] = {"%dx%d" % k: v for k, v in shapes.items()}
-    # batch-size crossover on one 70B-shaped linear (8192 x 8192, W3 g128): the GEMV kernels up to batch 16,
-    # the tensor-core GEMM from there on; eight copies of the weights are rotated so every call reads cold weights
-    n = k = 8192
-    d70 = goq.desc(n, k, GROUP, WBITS)
-    gen = torch.Generator(device="cuda")
-    copies = []
-    for c in range(8):
-        gen.manual_seed(7000 + c)
-        codes = torch.randint(0, 1 << WBITS, (n, k), dtype=torch.uint8, device="cuda", generator=gen)
-        meta = torch.randint(0, 64, (n, k // 8), dtype=torch.uint8, device="cuda", generator=gen)
-        coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * 0.03).to(torch.float16)
-        pk = torch.empty(goq.packed_bytes(d70), dtype=torch.uint8, device="cuda")
-        goq.pack(d70, codes, meta, coef, pk)
-        copies.append(pk)
-        del codes, meta, coef
-    cross = {}
-    for batch in (1, 4, 16, 64, 256):
-        x = torch.randn((batch, k), device="cuda").to(torch.bfloat16)
-        y = torch.empty((batch, n), dtype=torch.float32, device="cuda")
-        paths = (["gemv"] if batch <= 16 else []) + (["gemm"] if batch >= 16 else [])
-        for path in paths:
-            wsx = goq.new_workspace(d70, goq.OP_GEMV if path == "gemv" else goq.OP_GEMM, batch)
-
-            def step_x():
-                for pk in copies:
-                    if path == "gemv":
-                        goq.gemv(d70, pk, x, batch, y, goq.F32, ws=wsx)
-                    else:
-                        goq.gemm(d70, pk, x, batch, goq.BF16, y=y, y_dtype=goq.F32, ws=wsx)
-
-            g = capture(torch, step_x)
-            us = time_graph(torch, g, 10, 3) * 1e3 / len(copies)
-            cross["batch%d_%s_us" % (batch, path)] = us
-            del g
-    out["crossover_8192x8192_w3"] = cross
-    del copies
     # prefill GEMM, M = 2048, one layer's seven linears
     m = 2048
     layer0 = stack[:7]
@@ -547,6 +511,43 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
     out["gemm_m2048_layer_tflops_bf16_out"] = flops / (e0.elapsed_time(e1) / 3 * 1e-3) / 1e12
     del yb
     del xs, ys, ws_gemm
+    # batch-size crossover on one 70B-shaped linear (8192 x 8192, g128) at W3, W2 and W4: goq_gemv up to batch 16,
+    # goq_gemm from there on; eight copies of the weights are rotated so every call reads cold weights
+    n = k = 8192
+    for wb in (3, 2, 4):
+        d70 = goq.desc(n, k, GROUP, wb)
+        gen = torch.Generator(device="cuda")
+        copies = []
+        for c in range(8):
+            gen.manual_seed(7000 + c)
+            codes = torch.randint(0, 1 << wb, (n, k), dtype=torch.uint8, device="cuda", generator=gen)
+            meta = torch.randint(0, 64, (n, k // 8), dtype=torch.uint8, device="cuda", generator=gen)
+            coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * 0.03).to(torch.float16)
+            pk = torch.empty(goq.packed_bytes(d70), dtype=torch.uint8, device="cuda")
+            goq.pack(d70, codes, meta, coef, pk)
+            copies.append(pk)
+            del codes, meta, coef
+        cross = {}
+        for batch in (1, 4, 16, 48, 64, 256):
+            x = torch.randn((batch, k), device="cuda").to(torch.bfloat16)
+            y = torch.empty((batch, n), dtype=torch.float32, device="cuda")
+            paths = (["gemv"] if batch <= 16 else []) + (["gemm"] if batch >= 16 else [])
+            for path in paths:
+                wsx = goq.new_workspace(d70, goq.OP_GEMV if path == "gemv" else goq.OP_GEMM, batch)
+
+                def step_x():
+                    for pk in copies:
+                        if path == "gemv":
+                            goq.gemv(d70, pk, x, batch, y, goq.F32, ws=wsx)
+                        else:
+                            goq.gemm(d70, pk, x, batch, goq.BF16, y=y, y_dtype=goq.F32, ws=wsx)
+
+                g = capture(torch, step_x)
+                us = time_graph(torch, g, 10, 3) * 1e3 / len(copies)
+                cross["batch%d_%s_us" % (batch, path)] = us
+                del g
+        out["crossover_8192x8192_w%d" % wb] = cross
+        del copies
     # integer path: ViT-B/16-shaped linears, 197 x 64 tokens, W3 group 64, int8 activations and coefficients
     mt = si.VIT_B16_TOKENS
     vit = []

@@ -10,7 +10,7 @@ using goq::Geometry;
 namespace {
 
 std::atomic<int> g_gemv_variant{0};
-constexpr int kGemmViaGemvMaxTokens = 64;
+constexpr int kGemmViaGemvMaxTokens = 48;
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -174,8 +174,8 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
         if (!y) return GOQ_ERR_INVALID_ARG;
         if (goq_status s = check_arch()) return s;
         const int variant = g_gemv_variant.load(std::memory_order_relaxed);
-        // Few tokens (17..64): the streaming GEMV kernel, 16 tokens per launch, is several times faster than a
-        // 128 x 512 tensor-core tile that would be mostly padding (measured crossover on 8192 x 8192: ~80 tokens).
+        // Few tokens (17..48): the streaming GEMV kernel, 16 tokens per launch (36 us each on 8192 x 8192), against a
+        // tensor-core tile that is mostly padding (one 256-token half tile per CTA, measured below).
         if (m <= kGemmViaGemvMaxTokens && variant == 0 && goq::gemv_stream_supported(g)) {
             if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
             if (ws_bytes < goq::gemv_stream_workspace(g)) return GOQ_ERR_WORKSPACE;

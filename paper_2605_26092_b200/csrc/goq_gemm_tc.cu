@@ -229,7 +229,8 @@ struct GemmParams {
     // Tile schedule (1-D grid). CTAs [0, n_full) take 128 x 512 tiles, numbered channel-tile fastest; the remaining
     // CTAs take the last tiles as halves of 256 tokens each, so that a last wave that would fill less than half of
     // the SMs runs for half as long on twice as many.
-    int n_full, n_tiles_x;
+    // With at most 256 tokens in all, every tile is one half (halves_per_tile = 1).
+    int n_full, n_tiles_x, halves_per_tile;
 };
 
 template <int WB>
@@ -256,11 +257,11 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bid = blockIdx.x;
-    const int tile = bid < p.n_full ? bid : p.n_full + ((bid - p.n_full) >> 1);
+    const int tile = bid < p.n_full ? bid : p.n_full + (bid - p.n_full) / p.halves_per_tile;
     const int n_half = bid < p.n_full ? 2 : 1;   // token halves (of 256) this CTA computes
     const int tile_x = tile % p.n_tiles_x;
     const int T0 = tile_x * (kTileN / kTileRows);  // first 16-row tile of this CTA
-    const int tok0 = (tile / p.n_tiles_x) * kTileM + (bid < p.n_full ? 0 : ((bid - p.n_full) & 1) * 256);
+    const int tok0 = (tile / p.n_tiles_x) * kTileM + (bid < p.n_full ? 0 : ((bid - p.n_full) % p.halves_per_tile) * 256);
     const int n_chunks = 2 * p.k_blocks;
 
     if (tid == 0) {
@@ -575,8 +576,10 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
     const int tail = tiles % sm_count;   // tiles of the last, partial wave
     const int split = (tiles > sm_count && tail > 0 && 2 * tail <= sm_count) ? tail : 0;
     p.n_tiles_x = tiles_x;
-    p.n_full = tiles - split;
-    gemm_tc_kernel<WB><<<p.n_full + 2 * split, kThreads, smem, st>>>(p, map);
+    p.halves_per_tile = (m <= 256) ? 1 : 2;
+    p.n_full = (m <= 256) ? 0 : tiles - split;
+    const int n_ctas = (m <= 256) ? tiles : p.n_full + 2 * split;
+    gemm_tc_kernel<WB><<<n_ctas, kThreads, smem, st>>>(p, map);
     return cudaGetLastError();
 }
 
