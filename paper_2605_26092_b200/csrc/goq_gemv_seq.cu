@@ -364,8 +364,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
                 }
                 if (ok) {
                     float* rb = red + (size_t)rs * kConsumerWarps * 32 * 4;
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) rb[(warp * 32 + lane) * 4 + r] = acc[r];
+                    reinterpret_cast<float4*>(rb)[warp * 32 + lane] = make_float4(acc[0], acc[1], acc[2], acc[3]);
                     __threadfence_block();
                     __syncwarp();
                     int old = 0;
@@ -374,9 +373,9 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
                     if (old == contributors - 1) {
                         __threadfence_block();
                         float out[4] = {0.f, 0.f, 0.f, 0.f};
-                        for (int w = 0; w < contributors; ++w) {
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) out[r] += rb[(w * 32 + lane) * 4 + r];
+                        for (int w = 0; w < contributors; ++w) {   // warp order: the sum does not depend on which warp came last
+                            const float4 f = reinterpret_cast<const float4*>(rb)[w * 32 + lane];
+                            out[0] += f.x; out[1] += f.y; out[2] += f.z; out[3] += f.w;
                         }
                         if (abort_flag == 0) {
 #pragma unroll
