@@ -432,7 +432,20 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
         ms = time_graph(torch, g, 20, 3)
         nbytes = sum(algorithmic_bytes(s["n"], s["k"], batch) for s in stack)
         out["gemv_batch%d_gbs" % batch] = nbytes / (ms * 1e-3) / 1e9
-        del g, xs, ys
+        del g
+        if batch <= 4:   # the same step as one dependent sequence (the integer-operand form takes up to 4 tokens)
+            try:
+                seq_b = goq.make_sequence([(s["d"], s["packed"], x, batch, y, goq.F32, j > 0)
+                                           for j, (s, x, y) in enumerate(zip(stack, xs, ys))])
+                ws_b = torch.empty(goq.sequence_workspace_bytes(len(stack)), dtype=torch.uint8, device="cuda")
+                goq.workspace_init(ws_b)
+                g = capture(torch, lambda: goq.gemv_sequence(seq_b, ws_b))
+                ms = time_graph(torch, g, 20, 3)
+                out["gemv_sequence_batch%d_gbs" % batch] = nbytes / (ms * 1e-3) / 1e9
+                del g
+            except goq.GoqError as e:
+                out["gemv_sequence_batch%d_gbs" % batch] = "unavailable: %s" % e
+        del xs, ys
     # the same decode step issued the other way (per-linear launches in a CUDA graph)
     def step_graph():
         for s in stack:

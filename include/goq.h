@@ -187,7 +187,8 @@ goq_status goq_gemv_static(const goq_desc* desc, const void* packed, const void*
  *            depends == 0 : x and y are independent of every earlier item (their buffers must not overlap the
  *                           outputs of earlier items).
  *   Constraints (else GOQ_ERR_UNSUPPORTED): every item has the same wbits (2 or 3) and group (32, 64, 128),
- *   batch <= 8, and batch * round_up(k_in, 128) * 2 bytes <= 23040 (the activations are staged in shared memory).
+ *   batch <= 8, and batch * round_up(k_in, 128) * 2 bytes <= 139264 (the activations are staged in shared memory;
+ *   up to 23040 bytes two CTAs share an SM, above that the launch takes one CTA per SM), k_in <= 12288.
  *   ws       goq_sequence_workspace_bytes(n_items) bytes, 256-byte aligned, zeroed once with goq_workspace_init;
  *            the call leaves it zero. One status word as for goq_gemv (goq_workspace_status).
  * Sequences longer than GOQ_SEQUENCE_MAX_ITEMS are split into several launches. The device must support

@@ -27,7 +27,8 @@ constexpr int kConsumerWarps = 16;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kStageUnits = kConsumerWarps;
 constexpr int kRedSlots = 2;
-constexpr int kXBufBytes = 22 * 1024 + 512;   // staged activations of one linear: batch * k_pad * 2 bytes
+constexpr int kXBufBytes = 22 * 1024 + 512;   // staged activations of one linear (batch * k_pad * 2 bytes) with two CTAs per SM
+constexpr int kXBufBytesMax = 136 * 1024;      // ... with one CTA per SM, for the batches and widths that need more
 constexpr int kScaleFloats = 96 * 4;           // (integer form) one 2^-s per k-block and token: k_blocks <= 90, batch <= 4
 constexpr int kGlobalSpin = 1 << 20;          // polls (with a short sleep) of a completion counter
 
@@ -127,8 +128,8 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_seq_kernel(const __grid_cons
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(red + kRedSlots * kConsumerWarps * 32 * 4);
     uint64_t* empty_bar = full_bar + p.n_stages;
     uint64_t* x_bar = empty_bar + p.n_stages;
-    uint16_t* xs = reinterpret_cast<uint16_t*>(x_bar + 2);   // bf16 rows, or (I8) int8 rows 2*token + slice
-    float* xscale = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(xs) + kXBufBytes);   // (I8) [k-block][4 tokens]
+    float* xscale = reinterpret_cast<float*>(x_bar + 2);   // (I8) [k-block][4 tokens]
+    uint16_t* xs = reinterpret_cast<uint16_t*>(xscale + kScaleFloats);   // bf16 rows, or (I8) int8 rows 2*token + slice; last: its size varies per launch
     __shared__ volatile int abort_flag;
     __shared__ int arrive_cnt[kRedSlots];
     __shared__ int done_gen[kRedSlots];
@@ -419,7 +420,8 @@ static int seq_sm_count() {
 }
 
 bool gemv_seq_supported(const Geometry& g, int m) {
-    return g.group >= 32 && g.wbits <= 3 && m >= 1 && m <= 8 && (size_t)m * g.k_pad * 2 <= (size_t)seq::kXBufBytes;
+    return g.group >= 32 && g.wbits <= 3 && m >= 1 && m <= 8 && (size_t)m * g.k_pad * 2 <= (size_t)seq::kXBufBytesMax &&
+           g.k_blocks * 4 <= seq::kScaleFloats;
 }
 size_t gemv_seq_workspace(int n_items) { return 256 + (size_t)(n_items > 0 ? n_items : 0) * sizeof(int); }
 
@@ -428,17 +430,31 @@ static cudaError_t launch_seq_cfg(seq::Params& p, cudaStream_t st) {
     auto kernel = seq::gemv_seq_kernel<WB, CPG, I8>;
     const int stage_bytes = seq::kStageUnits * p.unit_bytes;
     p.n_stages = 3;
+    // The activations of the widest linear decide the buffer: the usual size leaves room for two CTAs per SM; a
+    // larger batch or width gets what it needs and one CTA per SM (the grid follows from the occupancy query).
+    size_t x_need = 0;
+    for (int i = 0; i < p.n_items; ++i) {
+        const size_t b = (size_t)p.item[i].m_total * p.item[i].k_blocks * kBlockK * 2;
+        if (b > x_need) x_need = b;
+    }
+    const int xbuf_bytes = x_need <= (size_t)seq::kXBufBytes ? seq::kXBufBytes : (int)((x_need + 1023) & ~(size_t)1023);
     const size_t smem = (size_t)2 * kLutBytes + (size_t)p.n_stages * stage_bytes + (size_t)seq::kRedSlots * seq::kConsumerWarps * 32 * 4 * sizeof(float) +
-                        (size_t)(2 * p.n_stages + 2) * sizeof(uint64_t) + (size_t)seq::kXBufBytes + (size_t)seq::kScaleFloats * sizeof(float);
-    static size_t attr_smem = 0;
-    static int per_sm = 0;
+                        (size_t)(2 * p.n_stages + 2) * sizeof(uint64_t) + (size_t)xbuf_bytes + (size_t)seq::kScaleFloats * sizeof(float);
+    static size_t attr_smem = 0;   // largest size the attribute has been raised to
+    static size_t occ_smem[2] = {0, 0};   // occupancy cache: [0] the two-per-SM size, [1] the last larger size
+    static int occ_per_sm[2] = {0, 0};
     if (smem > attr_smem) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, seq::kThreads, smem);
-        if (e != cudaSuccess) return e;
         attr_smem = smem;
     }
+    const int slot = xbuf_bytes == seq::kXBufBytes ? 0 : 1;
+    if (occ_smem[slot] != smem) {
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_per_sm[slot], kernel, seq::kThreads, smem);
+        if (e != cudaSuccess) return e;
+        occ_smem[slot] = smem;
+    }
+    const int per_sm = occ_per_sm[slot];
     if (per_sm < 1) return cudaErrorLaunchOutOfResources;
     long long total_tiles = 0;
     for (int i = 0; i < p.n_items; ++i) total_tiles += p.item[i].n_tiles;

@@ -130,6 +130,33 @@ def test_small_batches_integer_operand_form(goq, g, b, form):
         assert err <= TIGHT, err
 
 
+@pytest.mark.parametrize("shapes", [
+    [(64, 4224, 4), (48, 11008, 3), (300, 256, 1)],      # batch <= 4: integer form unless bf16 operands are forced
+    [(32, 4096, 8), (500, 2304, 7), (40, 128, 2)],       # batch up to 8: bf16 operands
+])
+def test_activations_beyond_the_two_cta_buffer(goq, shapes, form):
+    """Batches and widths whose staged activations exceed the buffer that leaves room for two CTAs per SM run
+    with a buffer sized for the launch and one CTA per SM; a dependent chain inside exercises the counters."""
+    from tests.gpu_util import dev
+    keep, checks, items = [], [], []
+    for i, (n, k, m) in enumerate(shapes):
+        L = _layer(goq, n, k, 128, 3, seed=290 + i)
+        xb = si.bf16_activations(m, k, seed=260 + i)
+        y = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda")
+        xd = dev(xb)
+        keep.append(xd)
+        items.append((L["d"], L["packed"], xd, m, y, goq.F32, i > 0))
+        checks.append((L, xb, y))
+    ws = _ws(goq, len(items))
+    goq.gemv_sequence(goq.make_sequence(items), ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    for L, xb, y in checks:
+        y_ref = O.linear_f64(L["codes"], L["meta"], L["coef"], si.bf16_bits_to_f64(xb), 128, 3)
+        assert O.normwise_rel_err(y.cpu().numpy().astype(np.float64), y_ref) <= TIGHT
+    del keep
+
+
 def test_one_7b_shaped_layer_sampled_rows(goq, form):
     from tests.gpu_util import dev
     items, checks = [], []
