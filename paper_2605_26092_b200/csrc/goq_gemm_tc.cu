@@ -231,6 +231,13 @@ struct GemmParams {
     // the SMs runs for half as long on twice as many.
     // With at most 256 tokens in all, every tile is one half (halves_per_tile = 1).
     int n_full, n_tiles_x, halves_per_tile;
+    // Split-K (only with at most 256 tokens, where the tiles alone would leave most SMs idle): n_split CTAs share a
+    // tile, each takes kb_per_split k-blocks and parks its fp32 partial tile in `partial`; the CTA that arrives last
+    // at the tile's counter adds the partials in split order (the result does not depend on timing), scales and
+    // stores, and leaves the counter zero.
+    int n_split, kb_per_split;
+    float* partial;      // [tile][split][256 tokens][128 channels]
+    int* tile_counter;   // [tile], zero on entry, left zero
 };
 
 template <int WB>
@@ -254,15 +261,19 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
     __shared__ uint32_t tmem_base_slot;
     __shared__ __align__(16) float inv_s[kTileM];   // 2^-s of this CTA's tokens (1 for tokens past the end)
     __shared__ volatile int abort_flag;
+    __shared__ volatile int split_last;   // (split-K) this CTA completed its tile's counter
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bid = blockIdx.x;
-    const int tile = bid < p.n_full ? bid : p.n_full + (bid - p.n_full) / p.halves_per_tile;
-    const int n_half = bid < p.n_full ? 2 : 1;   // token halves (of 256) this CTA computes
+    const int unit_id = bid / p.n_split, split = bid - unit_id * p.n_split;   // n_split > 1 only when every tile is one half
+    const int tile = unit_id < p.n_full ? unit_id : p.n_full + (unit_id - p.n_full) / p.halves_per_tile;
+    const int n_half = unit_id < p.n_full ? 2 : 1;   // token halves (of 256) this CTA computes
+    const int kb0 = split * p.kb_per_split;            // this CTA's k-blocks: [kb0, kb0 + nkb)
+    const int nkb = min(p.kb_per_split, p.k_blocks - kb0);
     const int tile_x = tile % p.n_tiles_x;
     const int T0 = tile_x * (kTileN / kTileRows);  // first 16-row tile of this CTA
-    const int tok0 = (tile / p.n_tiles_x) * kTileM + (bid < p.n_full ? 0 : ((bid - p.n_full) % p.halves_per_tile) * 256);
-    const int n_chunks = 2 * p.k_blocks;
+    const int tok0 = (tile / p.n_tiles_x) * kTileM + (unit_id < p.n_full ? 0 : ((unit_id - p.n_full) % p.halves_per_tile) * 256);
+    const int n_chunks = 2 * nkb;
 
     if (tid == 0) {
         abort_flag = 0;
@@ -291,7 +302,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
             if (n_rec > kExpanders) n_rec = kExpanders;
             bool ok = true;
             int pk_issued = 0, b_issued = 0;   // record blocks / activation chunks whose copies have been issued
-            for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
+            for (int kb = 0; kb < nkb && ok; ++kb) {
                 const int ps = kb & 1;
                 if (kb >= 2) ok = mbar_wait(&pk_empty[ps], ((kb >> 1) - 1) & 1, &abort_flag);
                 if (!ok) break;
@@ -299,16 +310,16 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                 mbar_expect_tx(&pk_full[ps], (uint32_t)n_rec * p.unit_bytes);
                 for (int r = 0; r < n_rec; ++r)
                     bulk_g2s(pk_ring + ps * pk_slot_bytes + r * p.unit_bytes,
-                             p.packed + unit_offset(T0 + r, kb, p.k_blocks, p.unit_bytes), p.unit_bytes, &pk_full[ps]);
+                             p.packed + unit_offset(T0 + r, kb0 + kb, p.k_blocks, p.unit_bytes), p.unit_bytes, &pk_full[ps]);
                 for (int half = 0; half < 2 && ok; ++half) {
                     const int chunk = 2 * kb + half, s = chunk % kStages;
                     if (chunk >= kStages) ok = mbar_wait(&empty[s], ((chunk / kStages) - 1) & 1, &abort_flag);
                     if (!ok) break;
                     b_issued = chunk + 1;
                     mbar_expect_tx(&full_b[s], (uint32_t)n_half * (kBTileBytes / 2));
-                    tma_load_2d(b_tiles + s * kBTileBytes, &x_map, chunk * kChunkK, tok0, &full_b[s]);
+                    tma_load_2d(b_tiles + s * kBTileBytes, &x_map, (2 * kb0 + chunk) * kChunkK, tok0, &full_b[s]);
                     if (n_half == 2)
-                        tma_load_2d(b_tiles + s * kBTileBytes + kBTileBytes / 2, &x_map, chunk * kChunkK, tok0 + 256, &full_b[s]);
+                        tma_load_2d(b_tiles + s * kBTileBytes + kBTileBytes / 2, &x_map, (2 * kb0 + chunk) * kChunkK, tok0 + 256, &full_b[s]);
                 }
             }
             if (!ok || abort_flag) {
@@ -349,7 +360,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
         const bool valid = (T0 + e) < p.n_tiles;
         constexpr uint32_t kZeroWord = (WB == 3) ? 0x33333333u : 0x11111111u;  // every code = the zero state
         bool ok = true;
-        for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
+        for (int kb = 0; kb < nkb && ok; ++kb) {
             const int ps = kb & 1;
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(&pk_full[ps], (kb >> 1) & 1, &abort_flag));
             if (!ok) break;
@@ -410,6 +421,29 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
             const bool f32 = p.y_dtype == GOQ_F32;
             const bool vec = (tile_x + 1) * kTileN <= p.n_out && (p.n_out & 3) == 0 &&
                              (reinterpret_cast<uintptr_t>(p.y) & (f32 ? 15u : 7u)) == 0;
+            auto store4 = [&](int tok, float4 f) {   // four channels of one token
+                const size_t o = (size_t)tok * p.n_out + row4;
+                if (f32) {
+                    float* y = reinterpret_cast<float*>(p.y);
+                    if (vec) *reinterpret_cast<float4*>(y + o) = f;
+                    else {
+                        if (row4 + 0 < p.n_out) y[o + 0] = f.x;
+                        if (row4 + 1 < p.n_out) y[o + 1] = f.y;
+                        if (row4 + 2 < p.n_out) y[o + 2] = f.z;
+                        if (row4 + 3 < p.n_out) y[o + 3] = f.w;
+                    }
+                } else {
+                    uint16_t* y = reinterpret_cast<uint16_t*>(p.y);
+                    const uint16_t h0 = f32_to_bf16_rne(f.x), h1 = f32_to_bf16_rne(f.y), h2 = f32_to_bf16_rne(f.z), h3 = f32_to_bf16_rne(f.w);
+                    if (vec) *reinterpret_cast<uint2*>(y + o) = make_uint2((uint32_t)h0 | ((uint32_t)h1 << 16), (uint32_t)h2 | ((uint32_t)h3 << 16));
+                    else {
+                        if (row4 + 0 < p.n_out) y[o + 0] = h0;
+                        if (row4 + 1 < p.n_out) y[o + 1] = h1;
+                        if (row4 + 2 < p.n_out) y[o + 2] = h2;
+                        if (row4 + 3 < p.n_out) y[o + 3] = h3;
+                    }
+                }
+            };
 #pragma unroll 1
             for (int cb = 0; cb < 8 && ok; ++cb) {
                 uint32_t v[32];
@@ -429,32 +463,52 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                 if (lane == 0) mbar_arrive(&epi_bar[col_half]);
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(&epi_bar[col_half], cb & 1, &abort_flag));
                 if (!ok) break;
+                if (p.n_split > 1) {   // park the (already scaled) partial rows: [token][128 channels], 512 bytes per warp store
+                    float* part = p.partial + ((size_t)tile * p.n_split + split) * (256 * kTileN);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int jt = q * 8 + i;
+                        __stcg(reinterpret_cast<float4*>(part + (size_t)(cb * 32 + jt) * kTileN + 4 * lane),
+                               *reinterpret_cast<const float4*>(&st[jt * kTileN + 4 * lane]));
+                    }
+                    continue;
+                }
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int jt = q * 8 + i, tok = tok0 + col0 + jt;
-                    if (tok >= p.m_total) continue;
-                    const float4 f = *reinterpret_cast<const float4*>(&st[jt * kTileN + 4 * lane]);
-                    const size_t o = (size_t)tok * p.n_out + row4;
-                    if (f32) {
-                        float* y = reinterpret_cast<float*>(p.y);
-                        if (vec) *reinterpret_cast<float4*>(y + o) = f;
-                        else {
-                            if (row4 + 0 < p.n_out) y[o + 0] = f.x;
-                            if (row4 + 1 < p.n_out) y[o + 1] = f.y;
-                            if (row4 + 2 < p.n_out) y[o + 2] = f.z;
-                            if (row4 + 3 < p.n_out) y[o + 3] = f.w;
+                    if (tok < p.m_total) store4(tok, *reinterpret_cast<const float4*>(&st[jt * kTileN + 4 * lane]));
+                }
+            }
+            if (p.n_split > 1 && ok) {
+                // Every warp's partial rows are on their way: make them visible, meet, and let one thread count this CTA
+                // in. The epilogue barrier has been through eight phases, so the next two have parities 0 and 1.
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&epi_bar[0]);
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&epi_bar[0], 0, &abort_flag));
+                if (ok) {
+                    if (lane == 0) {
+                        if (q == 0) {
+                            split_last = (atomicAdd(&p.tile_counter[tile], 1) == p.n_split - 1) ? 1 : 0;
+                            __threadfence();
                         }
-                    } else {
-                        uint16_t* y = reinterpret_cast<uint16_t*>(p.y);
-                        const uint16_t h0 = f32_to_bf16_rne(f.x), h1 = f32_to_bf16_rne(f.y), h2 = f32_to_bf16_rne(f.z), h3 = f32_to_bf16_rne(f.w);
-                        if (vec) *reinterpret_cast<uint2*>(y + o) = make_uint2((uint32_t)h0 | ((uint32_t)h1 << 16), (uint32_t)h2 | ((uint32_t)h3 << 16));
-                        else {
-                            if (row4 + 0 < p.n_out) y[o + 0] = h0;
-                            if (row4 + 1 < p.n_out) y[o + 1] = h1;
-                            if (row4 + 2 < p.n_out) y[o + 2] = h2;
-                            if (row4 + 3 < p.n_out) y[o + 3] = h3;
-                        }
+                        mbar_arrive(&epi_bar[0]);
                     }
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(&epi_bar[0], 1, &abort_flag));
+                }
+                if (ok && split_last) {
+                    const float* part = p.partial + (size_t)tile * p.n_split * (256 * kTileN);
+                    for (int jt = q * 64; jt < q * 64 + 64; ++jt) {
+                        const int tok = tok0 + jt;
+                        if (tok >= p.m_total) break;
+                        float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int sp = 0; sp < p.n_split; ++sp) {   // split order: the sum does not depend on which CTA came last
+                            const float4 a = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)sp * 256 + jt) * kTileN + 4 * lane));
+                            f.x += a.x; f.y += a.y; f.z += a.z; f.w += a.w;
+                        }
+                        store4(tok, f);
+                    }
+                    if (q == 0 && lane == 0) p.tile_counter[tile] = 0;
                 }
             }
         }
@@ -524,6 +578,28 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
+static int sm_count_cached() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+// Split-K factor for a call (1 = none): only with at most 256 tokens, when the channel tiles alone would leave at
+// least half of the SMs idle, and never below four k-blocks per CTA.
+static int split_factor(const Geometry& g, int m) {
+    if (m > 256) return 1;
+    const int tiles_x = (g.n_pad + kTileN - 1) / kTileN;
+    int s = sm_count_cached() / tiles_x;
+    if (s > 4) s = 4;
+    if (s > g.k_blocks / 4) s = g.k_blocks / 4;
+    if (s < 2) return 1;
+    const int per = (g.k_blocks + s - 1) / s;
+    return (g.k_blocks + per - 1) / per;   // no empty split
+}
+
 static size_t smem_bytes(const Geometry& g) {
     return 8192 /* alignment slack */ + kLutBytes + (size_t)kStages * (kATileBytes + kBTileBytes) +
            (size_t)2 * kExpanders * g.unit_bytes + 16 * sizeof(uint64_t);
@@ -531,7 +607,7 @@ static size_t smem_bytes(const Geometry& g) {
 
 template <int WB>
 static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* x, int m, void* y, int y_dtype, int* status,
-                             float* inv_scale, uint16_t* xh, cudaStream_t st) {
+                             float* inv_scale, uint16_t* xh, int* tile_counter, float* partial, cudaStream_t st) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return cudaErrorNotSupported;
     if (g.k_in % 8 != 0) return cudaErrorInvalidValue;
@@ -567,18 +643,17 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
     while ((1 << lg) < g.group) ++lg;
     p.group_log2 = lg;
     const int tiles_x = (g.n_pad + kTileN - 1) / kTileN, tiles = tiles_x * ((m + kTileM - 1) / kTileM);
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            sm_count = 148;
-    }
+    const int sm_count = sm_count_cached();
     const int tail = tiles % sm_count;   // tiles of the last, partial wave
     const int split = (tiles > sm_count && tail > 0 && 2 * tail <= sm_count) ? tail : 0;
     p.n_tiles_x = tiles_x;
     p.halves_per_tile = (m <= 256) ? 1 : 2;
     p.n_full = (m <= 256) ? 0 : tiles - split;
-    const int n_ctas = (m <= 256) ? tiles : p.n_full + 2 * split;
+    p.n_split = split_factor(g, m);
+    p.kb_per_split = (g.k_blocks + p.n_split - 1) / p.n_split;
+    p.partial = partial;
+    p.tile_counter = tile_counter;
+    const int n_ctas = (m <= 256) ? tiles * p.n_split : p.n_full + 2 * split;
     gemm_tc_kernel<WB><<<n_ctas, kThreads, smem, st>>>(p, map);
     return cudaGetLastError();
 }
@@ -591,16 +666,31 @@ bool gemm_tc_supported(const Geometry& g) { return g.wbits <= 3 && g.k_in % 8 ==
 // Scratch: [0, base) is left to the other kernels that may share the buffer (status word at 0, their zeroed counters);
 // then the per-token inverse scales and the fp16 copy of the activations.
 static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
-size_t gemm_tc_workspace(const Geometry& g, int m, size_t base) {
-    return align256(base < 256 ? 256 : base) + align256((size_t)m * sizeof(float)) + (size_t)m * g.k_in * 2;
+namespace {
+struct TcScratch { size_t inv_off, xh_off, counter_off, partial_off, total; };
+TcScratch tc_scratch(const Geometry& g, int m, size_t base) {
+    TcScratch t;
+    t.inv_off = align256(base < 256 ? 256 : base);
+    t.xh_off = t.inv_off + align256((size_t)m * sizeof(float));
+    t.counter_off = align256(t.xh_off + (size_t)m * g.k_in * 2);
+    const int split = tc::split_factor(g, m);
+    const size_t tiles_x = (size_t)(g.n_pad + tc::kTileN - 1) / tc::kTileN;
+    t.partial_off = t.counter_off + (split > 1 ? align256(tiles_x * sizeof(int)) : 0);
+    t.total = t.partial_off + (split > 1 ? tiles_x * split * 256 * tc::kTileN * sizeof(float) : 0);
+    return t;
 }
+}  // namespace
+size_t gemm_tc_workspace(const Geometry& g, int m, size_t base) { return tc_scratch(g, m, base).total; }
 cudaError_t launch_gemm_tc(const Geometry& g, const void* packed, const void* x, int m, void* y, int y_dtype, void* ws,
                            size_t base, cudaStream_t st) {
     int* status = (int*)ws;
-    uint8_t* b = (uint8_t*)ws + align256(base < 256 ? 256 : base);
-    float* inv_scale = (float*)b;
-    uint16_t* xh = (uint16_t*)(b + align256((size_t)m * sizeof(float)));
-    return g.wbits == 3 ? tc::launch_wb<3>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, st)
-                        : tc::launch_wb<2>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, st);
+    const TcScratch t = tc_scratch(g, m, base);
+    uint8_t* b = (uint8_t*)ws;
+    float* inv_scale = (float*)(b + t.inv_off);
+    uint16_t* xh = (uint16_t*)(b + t.xh_off);
+    int* counters = (int*)(b + t.counter_off);
+    float* partial = (float*)(b + t.partial_off);
+    return g.wbits == 3 ? tc::launch_wb<3>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, counters, partial, st)
+                        : tc::launch_wb<2>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, counters, partial, st);
 }
 }  // namespace goq

@@ -267,6 +267,30 @@ def test_gemm_token_scaling_extreme_activations(goq):
         assert e <= GEMM_TC_TOL, (tok, e)
 
 
+@pytest.mark.parametrize("n,k,g,m", [(200, 2048, 128, 100), (130, 1152, 64, 256), (520, 4096, 128, 49)])
+def test_gemm_split_k_few_tokens(goq, n, k, g, m):
+    """At most 256 tokens and few channel tiles: several CTAs share a tile along k (4, 2 and 4 splits here, the last
+    one ragged), park partial tiles in the scratch buffer and the last to arrive adds them in split order. Every output
+    compared; a second call on the same scratch buffer must give the same bits (the counters are left zero)."""
+    from tests.gpu_util import pack_weights, dev
+    codes, meta, coef = _quantized(n, k, g, 3, seed=61 + n)
+    d, packed = pack_weights(n, k, g, 3, codes, meta, coef)
+    xb = si.bf16_activations(m, k, seed=62)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), g, 3)
+    x = dev(xb)
+    ws = goq.new_workspace(d, goq.OP_GEMM, m)
+    outs = []
+    for _ in range(2):
+        y = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda")
+        goq.gemm(d, packed, x, m, goq.BF16, y=y, y_dtype=goq.F32, ws=ws)
+        torch.cuda.synchronize()
+        assert goq.workspace_status(ws) == goq.OK
+        outs.append(y)
+    assert torch.equal(outs[0], outs[1])
+    err = O.normwise_rel_err(outs[0].cpu().numpy().astype(np.float64), y_ref)
+    assert err <= GEMM_TC_TOL, err
+
+
 def test_gemm_tail_wave_runs_as_half_tiles(goq):
     """160 output tiles (20 channel tiles x 8 token tiles) on 148 SMs: the 12 tiles of the last wave are scheduled
     as 24 half tiles of 256 tokens; 3900 tokens make the last token tile ragged. Sampled channels, all tokens."""
