@@ -76,7 +76,10 @@ size_t goq_packed_bytes(const goq_desc* desc);
  * This is the figure roofline numbers are quoted against; the packed buffer may be larger. */
 size_t goq_algorithmic_bytes(const goq_desc* desc);
 
-/* Scratch bytes goq_gemv / goq_gemm need for `m` activation rows (may be 0). */
+/* Scratch bytes goq_gemv / goq_gemm need for `m` activation rows (may be 0). Every kernel keeps its counters in
+ * the same leading area and leaves them zero, and nothing else in the buffer is carried from one call to the
+ * next: one buffer of the largest size, initialised once, can serve calls for different layers, ops and m, as
+ * long as those calls cannot overlap on the GPU. */
 size_t goq_workspace_bytes(const goq_desc* desc, int op, int m);
 
 /* Zero-fill a scratch buffer (asynchronous on `stream`). A scratch buffer must be initialised once
@@ -157,9 +160,10 @@ goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x
  * cudaMalloc/cudaFree imply; plain C callers with no device allocator of their own. The scratch lives in a
  * fixed array inside the library image (GOQ_STATIC_SCRATCH_BYTES per GPU that loads the library, held until
  * the process exits); nothing is allocated or freed by this call, by any CUDA call it makes, or through torch.
- *   Arguments and results exactly as goq_gemv (same kernel, same numerics).
- *   Limits: the layer's scratch need, goq_workspace_bytes(desc, GOQ_OP_GEMV, batch), must not exceed
- *   GOQ_STATIC_SCRATCH_BYTES (about 262 000 sixteen-row tiles, i.e. n_out up to ~4 million), otherwise
+ *   Arguments as goq_gemv; always the bf16-operand streaming kernel (goq_gemv takes the integer-operand form for
+ *   up to 4 tokens, so the two can differ in the last bits, both far inside the stated tolerance).
+ *   Limits: the streaming kernel's scratch (status word, tile counters, 1 MiB of parked partial sums) must fit
+ *   GOQ_STATIC_SCRATCH_BYTES (it does for every layer that kernel takes: n_out up to 262 144), otherwise
  *   GOQ_ERR_WORKSPACE is returned and nothing is launched; configurations goq_gemv serves with its
  *   scratch-free kernels (group < 32, wbits = 4) return GOQ_ERR_UNSUPPORTED here - use goq_gemv for them.
  *   First call on each device: looks up the array's device address (once per device, with that device

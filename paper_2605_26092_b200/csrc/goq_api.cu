@@ -31,14 +31,6 @@ goq_status check_arch() {
     return ok ? GOQ_OK : GOQ_ERR_ARCH;
 }
 
-// scratch of the decode kernels that may share a buffer with the prefill GEMM: its activation copy sits behind it
-size_t gemv_scratch(const Geometry& g) {
-    size_t need = 0;
-    if (goq::gemv_stream_supported(g)) need = goq::gemv_stream_workspace(g);
-    if (goq::gemv_tc_supported(g, 1) && goq::gemv_tc_workspace(g) > need) need = goq::gemv_tc_workspace(g);
-    return need;
-}
-
 std::atomic<int> g_last_cuda_error{0};
 goq_status from_cuda(cudaError_t e) {
     if (e == cudaSuccess) return GOQ_OK;
@@ -89,7 +81,7 @@ size_t goq_workspace_bytes(const goq_desc* desc, int op, int m) {
     }
     if (op == GOQ_OP_GEMM) {
         // covers both kernels a call with these arguments may take (few tokens: the streaming GEMV, unless a variant is forced)
-        size_t need = goq::gemm_tc_supported(g) ? goq::gemm_tc_workspace(g, m, gemv_scratch(g)) : 0;
+        size_t need = goq::gemm_tc_supported(g) ? goq::gemm_tc_workspace(g, m) : 0;
         if (m <= kGemmViaGemvMaxTokens && goq::gemv_stream_supported(g) && goq::gemv_stream_workspace(g) > need)
             need = goq::gemv_stream_workspace(g);
         return need;
@@ -192,8 +184,8 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
         }
         if (goq::gemm_tc_supported(g) && variant != 2) {
             if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
-            if (ws_bytes < goq::gemm_tc_workspace(g, m, gemv_scratch(g))) return GOQ_ERR_WORKSPACE;
-            return from_cuda(goq::launch_gemm_tc(g, packed, x, m, y, y_dtype, ws, gemv_scratch(g), (cudaStream_t)stream));
+            if (ws_bytes < goq::gemm_tc_workspace(g, m)) return GOQ_ERR_WORKSPACE;
+            return from_cuda(goq::launch_gemm_tc(g, packed, x, m, y, y_dtype, ws, (cudaStream_t)stream));
         }
         if (goq::linear_mma_supported(g))
             return from_cuda(goq::launch_linear_mma(g, packed, x, m, y, y_dtype, (cudaStream_t)stream));

@@ -25,6 +25,12 @@ namespace goq {
 
 constexpr int kTileRows = 16;
 constexpr int kBlockK = 128;
+// Scratch buffer layout shared by every kernel, so that one buffer (sized for the largest call) can serve calls of
+// different shapes and kernels: [status word, 256 B][counters, kWsCounterBytes: zero on entry, left zero by every
+// kernel][everything else: contents carry nothing from one call to the next].
+constexpr size_t kWsStatusBytes = 256;
+constexpr size_t kWsCounterBytes = 64 * 1024;
+constexpr size_t kWsScratchOff = kWsStatusBytes + kWsCounterBytes;
 constexpr int kWordsPerBlock = 256;
 constexpr int kCodeBytesPerUnit = kWordsPerBlock * 4;
 

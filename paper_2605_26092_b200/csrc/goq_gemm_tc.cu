@@ -663,32 +663,31 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
 
 namespace goq {
 bool gemm_tc_supported(const Geometry& g) { return g.wbits <= 3 && g.k_in % 8 == 0 && tc::smem_bytes(g) + 2048 <= 227 * 1024; }
-// Scratch: [0, base) is left to the other kernels that may share the buffer (status word at 0, their zeroed counters);
-// then the per-token inverse scales and the fp16 copy of the activations.
+// Scratch: status word and tile counters in the common areas; behind them the per-token inverse scales, the fp16
+// copy of the activations and (split-K) the partial tiles.
 static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 namespace {
-struct TcScratch { size_t inv_off, xh_off, counter_off, partial_off, total; };
-TcScratch tc_scratch(const Geometry& g, int m, size_t base) {
+struct TcScratch { size_t inv_off, xh_off, partial_off, total; };
+TcScratch tc_scratch(const Geometry& g, int m) {
     TcScratch t;
-    t.inv_off = align256(base < 256 ? 256 : base);
+    t.inv_off = kWsScratchOff;
     t.xh_off = t.inv_off + align256((size_t)m * sizeof(float));
-    t.counter_off = align256(t.xh_off + (size_t)m * g.k_in * 2);
+    t.partial_off = align256(t.xh_off + (size_t)m * g.k_in * 2);
     const int split = tc::split_factor(g, m);
     const size_t tiles_x = (size_t)(g.n_pad + tc::kTileN - 1) / tc::kTileN;
-    t.partial_off = t.counter_off + (split > 1 ? align256(tiles_x * sizeof(int)) : 0);
     t.total = t.partial_off + (split > 1 ? tiles_x * split * 256 * tc::kTileN * sizeof(float) : 0);
     return t;
 }
 }  // namespace
-size_t gemm_tc_workspace(const Geometry& g, int m, size_t base) { return tc_scratch(g, m, base).total; }
+size_t gemm_tc_workspace(const Geometry& g, int m) { return tc_scratch(g, m).total; }
 cudaError_t launch_gemm_tc(const Geometry& g, const void* packed, const void* x, int m, void* y, int y_dtype, void* ws,
-                           size_t base, cudaStream_t st) {
+                           cudaStream_t st) {
     int* status = (int*)ws;
-    const TcScratch t = tc_scratch(g, m, base);
+    const TcScratch t = tc_scratch(g, m);
     uint8_t* b = (uint8_t*)ws;
     float* inv_scale = (float*)(b + t.inv_off);
     uint16_t* xh = (uint16_t*)(b + t.xh_off);
-    int* counters = (int*)(b + t.counter_off);
+    int* counters = (int*)(b + kWsStatusBytes);   // at most sm_count / 2 tiles when the split is on
     float* partial = (float*)(b + t.partial_off);
     return g.wbits == 3 ? tc::launch_wb<3>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, counters, partial, st)
                         : tc::launch_wb<2>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, counters, partial, st);

@@ -25,7 +25,7 @@
 namespace goq {
 
 // ------------------------------------------------------------------------------------------------
-// scratch layout: [status 256 B][tile counters][partials kMaxCtas x 2 x 256 floats]
+// scratch layout: [status 256 B][tile counters, in the common counter area][partials kMaxCtas x 2 x 256 floats]
 // ------------------------------------------------------------------------------------------------
 constexpr int kMaxCtas = 512;
 constexpr int kStatusBytes = 256;
@@ -37,7 +37,7 @@ struct StreamWs {
 __host__ inline StreamWs stream_ws_layout(const Geometry& g) {
     StreamWs w;
     w.counters_off = kStatusBytes;
-    w.partials_off = align_up(w.counters_off + (size_t)g.n_tiles * 4, 256);
+    w.partials_off = kWsScratchOff;
     w.total = w.partials_off + (size_t)kMaxCtas * 2 * kPartialFloats * sizeof(float);
     return w;
 }
@@ -381,10 +381,10 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
     if (lane == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
 }
 
-bool gemv_stream_supported(const Geometry& g) { return g.group >= 32 && g.wbits <= 3; }
+bool gemv_stream_supported(const Geometry& g) { return g.group >= 32 && g.wbits <= 3 && (size_t)g.n_tiles * 4 <= kWsCounterBytes; }
 
 size_t gemv_stream_workspace(const Geometry& g) { return stream_ws_layout(g).total; }
-size_t gemv_stream_zeroed_prefix(const Geometry& g) { return stream_ws_layout(g).partials_off; }
+size_t gemv_stream_zeroed_prefix(const Geometry& g) { return stream_ws_layout(g).counters_off + (size_t)g.n_tiles * 4; }
 
 bool stream_hash_is_bijective() {
     bool seen[64] = {};

@@ -53,9 +53,8 @@ constexpr int kSlotFloats = 128 * 16;        // parked partial sums of one segme
 struct Ws { size_t counters_off, partials_off, total; };
 __host__ inline Ws ws_layout(const Geometry& g) {
     Ws w;
-    const size_t n_super = (size_t)(g.n_tiles + kRowTiles - 1) / kRowTiles;
     w.counters_off = kStatusBytes;
-    w.partials_off = align_up(w.counters_off + n_super * 4, 256);
+    w.partials_off = kWsScratchOff;
     w.total = w.partials_off + (size_t)kMaxCtas * 2 * kSlotFloats * sizeof(float);
     return w;
 }
@@ -854,7 +853,7 @@ static cudaError_t launch_wb(const Geometry& g, const Params& p, cudaStream_t st
 }  // namespace gtc
 
 bool gemv_tc_supported(const Geometry& g, int m) {
-    return g.wbits <= 3 && (g.group == 128 || g.group == 64) && m >= 1 && m <= 16;
+    return g.wbits <= 3 && (g.group == 128 || g.group == 64) && m >= 1 && m <= 16 && (size_t)g.n_tiles * 4 <= kWsCounterBytes;
 }
 size_t gemv_tc_workspace(const Geometry& g) { return gtc::ws_layout(g).total; }
 

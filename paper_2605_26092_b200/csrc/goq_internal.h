@@ -50,13 +50,13 @@ bool gemv_seq_supported(const Geometry& g, int m);
 size_t gemv_seq_workspace(int n_items);
 cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, int unit_bytes, void* ws, cudaStream_t st);
 
-// Prefill GEMM on tcgen05 tensor cores (wbits <= 3). `ws` holds gemm_tc_workspace(g, m, base) bytes: the status word
-// at 0, `base` bytes the kernel never touches beyond it (the zeroed counters of the decode kernels when the buffer is
-// shared with them), then the per-token scales and the fp16 copy of the m x k_in activations.
+// Prefill GEMM on tcgen05 tensor cores (wbits <= 3). `ws` holds gemm_tc_workspace(g, m) bytes: status word and
+// (split-K) tile counters in the common areas, then the per-token scales, the fp16 copy of the m x k_in activations
+// and the split-K partial tiles.
 bool gemm_tc_supported(const Geometry& g);
-size_t gemm_tc_workspace(const Geometry& g, int m, size_t base);
+size_t gemm_tc_workspace(const Geometry& g, int m);
 cudaError_t launch_gemm_tc(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y, int y_dtype,
-                           void* ws, size_t base, cudaStream_t st);
+                           void* ws, cudaStream_t st);
 
 // Integer-activation layer.
 cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* x, int m, const float* sx,

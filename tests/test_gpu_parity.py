@@ -291,6 +291,45 @@ def test_gemm_split_k_few_tokens(goq, n, k, g, m):
     assert err <= GEMM_TC_TOL, err
 
 
+def test_one_scratch_buffer_serves_calls_of_different_shapes_and_kernels(goq):
+    """Every kernel keeps its counters in the same leading area of the scratch buffer and leaves them zero, and
+    nothing else is carried between calls: a buffer sized for the largest call, initialised once, must give the same
+    bits as a fresh buffer per call - streaming GEMV (tiles that straddle CTAs park partial sums), the sequence
+    kernel behind goq_gemv, the tensor-core GEMM with and without split-K, interleaved and repeated."""
+    from tests.gpu_util import pack_weights, dev
+    layers = []
+    for i, (n, k, g) in enumerate([(1000, 1152, 128), (300, 4224, 64), (130, 2048, 128)]):
+        codes, meta, coef = si.random_quantized(n, k, g, 3, seed=70 + i)
+        d, packed = pack_weights(n, k, g, 3, codes, meta, coef)
+        layers.append((d, packed, n, k))
+    calls = []   # (layer index, op, m)
+    for rep in range(2):
+        for li in range(3):
+            calls += [(li, "gemv", 16), (li, "gemm", 100), (li, "gemv", 1), (li, "gemm", 300), (li, "gemv", 5)]
+    xs = {m: {li: dev(si.bf16_activations(m, layers[li][3], seed=80 + m + li)) for li in range(3)} for m in (1, 5, 16, 100, 300)}
+    need = max(goq.workspace_bytes(layers[li][0], goq.OP_GEMV if op == "gemv" else goq.OP_GEMM, m) for li, op, m in calls)
+    shared = torch.empty(need, dtype=torch.uint8, device="cuda")
+    goq.workspace_init(shared)
+
+    def run(li, op, m, ws):
+        d, packed, n, k = layers[li]
+        y = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda")
+        if op == "gemv":
+            goq.gemv(d, packed, xs[m][li], m, y, goq.F32, ws=ws)
+        else:
+            goq.gemm(d, packed, xs[m][li], m, goq.BF16, y=y, y_dtype=goq.F32, ws=ws)
+        torch.cuda.synchronize()
+        assert goq.workspace_status(ws) == goq.OK
+        return y
+
+    for li, op, m in calls:
+        fresh = goq.new_workspace(layers[li][0], goq.OP_GEMV if op == "gemv" else goq.OP_GEMM, m)
+        want = run(li, op, m, fresh)
+        got = run(li, op, m, shared)
+        assert torch.isfinite(got).all()
+        assert torch.equal(want, got), (li, op, m)
+
+
 def test_gemm_tail_wave_runs_as_half_tiles(goq):
     """160 output tiles (20 channel tiles x 8 token tiles) on 148 SMs: the 12 tiles of the last wave are scheduled
     as 24 half tiles of 256 tokens; 3900 tokens make the last token tile ragged. Sampled channels, all tokens."""
