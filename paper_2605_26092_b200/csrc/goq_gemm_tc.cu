@@ -622,12 +622,8 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidTexture;  // distinct code: the tensor map could not be encoded
     const size_t smem = smem_bytes(g);
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_smem = smem;
-    }
+    static SmemAttrCache smem_attr;
+    if (cudaError_t e = ensure_dynamic_smem(gemm_tc_kernel<WB>, smem, smem_attr)) return e;
     GemmParams p;
     p.packed = (const uint8_t*)packed;
     p.y = y;

@@ -440,14 +440,10 @@ static cudaError_t launch_seq_cfg(seq::Params& p, cudaStream_t st) {
     const int xbuf_bytes = x_need <= (size_t)seq::kXBufBytes ? seq::kXBufBytes : (int)((x_need + 1023) & ~(size_t)1023);
     const size_t smem = (size_t)2 * kLutBytes + (size_t)p.n_stages * stage_bytes + (size_t)seq::kRedSlots * seq::kConsumerWarps * 32 * 4 * sizeof(float) +
                         (size_t)(2 * p.n_stages + 2) * sizeof(uint64_t) + (size_t)xbuf_bytes + (size_t)seq::kScaleFloats * sizeof(float);
-    static size_t attr_smem = 0;   // largest size the attribute has been raised to
     static size_t occ_smem[2] = {0, 0};   // occupancy cache: [0] the two-per-SM size, [1] the last larger size
     static int occ_per_sm[2] = {0, 0};
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_smem = smem;
-    }
+    static SmemAttrCache smem_attr;
+    if (cudaError_t e = ensure_dynamic_smem(kernel, smem, smem_attr)) return e;
     const int slot = xbuf_bytes == seq::kXBufBytes ? 0 : 1;
     if (occ_smem[slot] != smem) {
         cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_per_sm[slot], kernel, seq::kThreads, smem);

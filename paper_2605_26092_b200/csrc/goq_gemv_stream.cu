@@ -432,12 +432,8 @@ static cudaError_t launch_stream(const Geometry& g, const StreamParams& p0, cuda
                         (size_t)kRedSlots * kConsumerWarps * 32 * NT * 4 * sizeof(float) +
                         (size_t)(2 * n_stages + 2) * sizeof(uint64_t) + (size_t)p.x_smem_bytes;
     auto kernel = p.x_smem_bytes ? gemv_stream_kernel<WB, NT, CPG, true> : gemv_stream_kernel<WB, NT, CPG, false>;
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[p.x_smem_bytes ? 1 : 0]) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_set[p.x_smem_bytes ? 1 : 0] = true;
-    }
+    static SmemAttrCache smem_attr[2];
+    if (cudaError_t e = ensure_dynamic_smem(kernel, 160 * 1024, smem_attr[p.x_smem_bytes ? 1 : 0])) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kStreamThreads);

@@ -824,12 +824,8 @@ static cudaError_t launch_cfg(const Geometry& g, Params p, cudaStream_t st) {
     p.n_stages = n_stages;
     const size_t smem = fixed + (size_t)n_stages * stage_bytes;
     auto kernel = gemv_tc_kernel<WB, GPB, N>;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_smem = smem;
-    }
+    static SmemAttrCache smem_attr;
+    if (cudaError_t e = ensure_dynamic_smem(kernel, smem, smem_attr)) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kThreads);

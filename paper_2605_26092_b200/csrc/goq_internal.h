@@ -5,6 +5,21 @@
 
 namespace goq {
 
+// The dynamic shared memory limit of a kernel is a per-device attribute: remember, per device, the largest size it
+// has been raised to (one cache object per kernel instantiation, a function-local static at the call site).
+struct SmemAttrCache { size_t set[64] = {}; };
+template <class Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, size_t smem, SmemAttrCache& cache) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool tracked = dev >= 0 && dev < 64;
+    if (tracked && smem <= cache.set[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess && tracked) cache.set[dev] = smem;
+    return e;
+}
+
 cudaError_t launch_pack(const Geometry& g, const uint8_t* codes, const uint8_t* meta, const uint16_t* coef,
                         void* packed, cudaStream_t st);
 cudaError_t launch_unpack(const Geometry& g, const void* packed, uint8_t* b1, uint8_t* b2, uint16_t* coef,
