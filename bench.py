@@ -597,6 +597,22 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
     ops = sum(2.0 * 2.0 * mt * v["n"] * v["k"] for v in vit)  # two bases, multiply-add = 2 ops
     out["w3a8_vit_b16_int_tops"] = ops / (ms * 1e-3) / 1e12
     out["w3a8_vit_b16_ms"] = ms
+    # the same linears with the scaled bf16 output instead of the two int32 accumulator planes (2 against 8 bytes per output)
+    ys_a8 = [torch.empty((mt, v["n"]), dtype=torch.bfloat16, device="cuda") for v in vit]
+
+    def step_a8_y():
+        for v, yv in zip(vit, ys_a8):
+            goq.gemm(v["d"], v["packed"], v["x"], mt, goq.I8, sx=v["sx"], cq=v["cq"], sc=v["sc"], y=yv, y_dtype=goq.BF16)
+
+    step_a8_y()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(3):
+        step_a8_y()
+    e1.record()
+    torch.cuda.synchronize()
+    out["w3a8_vit_b16_int_tops_bf16_out"] = ops / (e0.elapsed_time(e1) / 3 * 1e-3) / 1e12
+    del ys_a8
     return out
 
 

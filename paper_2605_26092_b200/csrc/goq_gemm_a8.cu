@@ -181,8 +181,11 @@ __device__ __forceinline__ uint4 a8_lds128(uint32_t addr) {
 // k-block the activation tile (64 tokens x 128 int8) is staged in shared memory with cp.async, double-buffered; each
 // warp reads its unit record straight from global memory one k-block ahead. Row sums S1, S2 per macro-block on the
 // int8 tensor cores, then ACC += c~ * S in int32: every order of these integer operations gives the same bits.
-template <int WB>
-__global__ void __launch_bounds__(kA8Warps * 32, 1)
+// A macro-block (CPG 32-wide slices) is decoded whole before its MMAs, so that the row sums of one token tile live
+// only from its first MMA to its coefficient multiply: the 64 registers a full set of S1, S2 would hold buy a
+// second CTA per SM instead.
+template <int WB, int CPG>
+__global__ void __launch_bounds__(kA8Warps * 32, 2)
 gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int8_t* __restrict__ x,
                    const float* __restrict__ sx, const int8_t* __restrict__ cq, const float* __restrict__ sc,
                    void* __restrict__ y, int y_dtype, int32_t* __restrict__ acc_out, int n_out, int n_tiles, int k_in,
@@ -209,7 +212,8 @@ gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int
     const int T = blockIdx.x * kA8Warps + warp;
     const bool have_tile = T < n_tiles;
     const int tok0 = blockIdx.y * kA8Tok;
-    const int groups_in = k_in / group, cpg = group >> 5;
+    const int groups_in = k_in / group;
+    constexpr int cpg = CPG;
     const int row_a = T * 16 + g, row_b = row_a + 8;
     const uint32_t lut_lane = (uint32_t)__cvta_generic_to_shared(lut) + (uint32_t)(lane & 7) * 16u;
     const uint32_t xs_base = (uint32_t)__cvta_generic_to_shared(&xs[0][0]);
@@ -228,11 +232,11 @@ gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
 
-    int acc1[kA8NT][4], acc2[kA8NT][4], s1[kA8NT][4], s2[kA8NT][4];
+    int acc1[kA8NT][4], acc2[kA8NT][4];
 #pragma unroll
     for (int nt = 0; nt < kA8NT; ++nt)
 #pragma unroll
-        for (int r = 0; r < 4; ++r) acc1[nt][r] = acc2[nt][r] = s1[nt][r] = s2[nt][r] = 0;
+        for (int r = 0; r < 4; ++r) acc1[nt][r] = acc2[nt][r] = 0;
 
     // integer coefficient pairs (c1, c2) of rows g and g+8 for the up to four macro-blocks of k-block bk, fetched one
     // k-block ahead like the words: element jj = c1a | c2a << 8 | c1b << 16 | c2b << 24 (as unsigned bytes)
@@ -272,42 +276,43 @@ gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int
         if (!have_tile) continue;
         const uint32_t xt = xs_base + (uint32_t)(bk & 1) * (kA8Tok * kA8XStride) + (uint32_t)(g * kA8XStride + t * 8);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            uint32_t a[4], q[4];
+        for (int mb = 0; mb < 4 / CPG; ++mb) {   // macro-blocks of this k-block
+            uint32_t a[CPG][4], q[CPG][4];
 #pragma unroll
-            for (int v = 0; v < 2; ++v) {
-                const uint32_t w = v ? w1[c] : w0[c];
-                const uint32_t m = w & 0x77777777u, mh = m >> 16;
-                const uint32_t p_lo = prmt8(IntTables<WB>::P0, IntTables<WB>::P1, m), p_hi = prmt8(IntTables<WB>::P0, IntTables<WB>::P1, mh);
-                const uint32_t n_lo = prmt8(IntTables<WB>::N0, IntTables<WB>::N1, m), n_hi = prmt8(IntTables<WB>::N0, IntTables<WB>::N1, mh);
-                const uint32_t h = (w - m) * kA8HashMul;
-                const uint4 e = a8_lds128((((h >> 26) * 128u)) + lut_lane);
-                a[v] = p_lo;          // m16n8k32 A fragment: a0/a1 = k 4t..4t+3 of rows g / g+8, a2/a3 = k 16+4t..
-                a[2 + v] = p_hi;
-                const uint32_t qp_lo = prmt8(p_lo, p_hi, e.x), qn_lo = prmt8(n_lo, n_hi, e.x);
-                const uint32_t qp_hi = prmt8(p_lo, p_hi, e.y), qn_hi = prmt8(n_lo, n_hi, e.y);
-                q[v] = (qp_lo & ~e.z) | (qn_lo & e.z);
-                q[2 + v] = (qp_hi & ~e.w) | (qn_hi & e.w);
+            for (int cc = 0; cc < CPG; ++cc) {
+                const int c = mb * CPG + cc;
+#pragma unroll
+                for (int v = 0; v < 2; ++v) {
+                    const uint32_t w = v ? w1[c] : w0[c];
+                    const uint32_t m = w & 0x77777777u, mh = m >> 16;
+                    const uint32_t p_lo = prmt8(IntTables<WB>::P0, IntTables<WB>::P1, m), p_hi = prmt8(IntTables<WB>::P0, IntTables<WB>::P1, mh);
+                    const uint32_t n_lo = prmt8(IntTables<WB>::N0, IntTables<WB>::N1, m), n_hi = prmt8(IntTables<WB>::N0, IntTables<WB>::N1, mh);
+                    const uint32_t h = (w - m) * kA8HashMul;
+                    const uint4 e = a8_lds128((((h >> 26) * 128u)) + lut_lane);
+                    a[cc][v] = p_lo;          // m16n8k32 A fragment: a0/a1 = k 4t..4t+3 of rows g / g+8, a2/a3 = k 16+4t..
+                    a[cc][2 + v] = p_hi;
+                    const uint32_t qp_lo = prmt8(p_lo, p_hi, e.x), qn_lo = prmt8(n_lo, n_hi, e.x);
+                    const uint32_t qp_hi = prmt8(p_lo, p_hi, e.y), qn_hi = prmt8(n_lo, n_hi, e.y);
+                    q[cc][v] = (qp_lo & ~e.z) | (qn_lo & e.z);
+                    q[cc][2 + v] = (qp_hi & ~e.w) | (qn_hi & e.w);
+                }
             }
+            const uint32_t cw = cf[mb];
+            const int c1a = (int)(int8_t)(cw & 255u), c2a = (int)(int8_t)((cw >> 8) & 255u);
+            const int c1b = (int)(int8_t)((cw >> 16) & 255u), c2b = (int)(int8_t)(cw >> 24);
 #pragma unroll
             for (int nt = 0; nt < kA8NT; ++nt) {
-                const uint2 b = a8_lds64(xt + (uint32_t)(nt * 8 * kA8XStride + c * 32));
-                mma_s8(s1[nt], a[0], a[1], a[2], a[3], b.x, b.y);
-                mma_s8(s2[nt], q[0], q[1], q[2], q[3], b.x, b.y);
-            }
-            if (((c + 1) % cpg) == 0) {
-                const uint32_t cw = cf[c / cpg];
-                const int c1a = (int)(int8_t)(cw & 255u), c2a = (int)(int8_t)((cw >> 8) & 255u);
-                const int c1b = (int)(int8_t)((cw >> 16) & 255u), c2b = (int)(int8_t)(cw >> 24);
+                int s1[4] = {0, 0, 0, 0}, s2[4] = {0, 0, 0, 0};
 #pragma unroll
-                for (int nt = 0; nt < kA8NT; ++nt) {
-                    acc1[nt][0] += c1a * s1[nt][0]; acc1[nt][1] += c1a * s1[nt][1];
-                    acc1[nt][2] += c1b * s1[nt][2]; acc1[nt][3] += c1b * s1[nt][3];
-                    acc2[nt][0] += c2a * s2[nt][0]; acc2[nt][1] += c2a * s2[nt][1];
-                    acc2[nt][2] += c2b * s2[nt][2]; acc2[nt][3] += c2b * s2[nt][3];
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) s1[nt][r] = s2[nt][r] = 0;
+                for (int cc = 0; cc < CPG; ++cc) {
+                    const uint2 b = a8_lds64(xt + (uint32_t)(nt * 8 * kA8XStride + (mb * CPG + cc) * 32));
+                    mma_s8(s1, a[cc][0], a[cc][1], a[cc][2], a[cc][3], b.x, b.y);
+                    mma_s8(s2, q[cc][0], q[cc][1], q[cc][2], q[cc][3], b.x, b.y);
                 }
+                acc1[nt][0] += c1a * s1[0]; acc1[nt][1] += c1a * s1[1];
+                acc1[nt][2] += c1b * s1[2]; acc1[nt][3] += c1b * s1[3];
+                acc2[nt][0] += c2a * s2[0]; acc2[nt][1] += c2a * s2[1];
+                acc2[nt][2] += c2b * s2[2]; acc2[nt][3] += c2b * s2[3];
             }
         }
     }
@@ -338,12 +343,13 @@ cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* 
     auto* words = (const uint8_t*)packed;
     if (g.group >= 32) {
         dim3 grid2((g.n_tiles + kA8Warps - 1) / kA8Warps, (m + kA8Tok - 1) / kA8Tok), block2(kA8Warps * 32);
-        if (g.wbits == 3)
-            gemm_a8_mma_kernel<3><<<grid2, block2, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, g.n_out,
-                                                            g.n_tiles, g.k_in, g.k_blocks, g.group, m);
-        else
-            gemm_a8_mma_kernel<2><<<grid2, block2, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, g.n_out,
-                                                            g.n_tiles, g.k_in, g.k_blocks, g.group, m);
+#define GOQ_A8_LAUNCH(WB_, CPG_)                                                                                          \
+    gemm_a8_mma_kernel<WB_, CPG_><<<grid2, block2, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, g.n_out, \
+                                                           g.n_tiles, g.k_in, g.k_blocks, g.group, m)
+        const int cpg = g.group >> 5;   // 1, 2 or 4
+        if (g.wbits == 3) { if (cpg == 1) GOQ_A8_LAUNCH(3, 1); else if (cpg == 2) GOQ_A8_LAUNCH(3, 2); else GOQ_A8_LAUNCH(3, 4); }
+        else { if (cpg == 1) GOQ_A8_LAUNCH(2, 1); else if (cpg == 2) GOQ_A8_LAUNCH(2, 2); else GOQ_A8_LAUNCH(2, 4); }
+#undef GOQ_A8_LAUNCH
         return cudaGetLastError();
     }
     dim3 grid(g.n_tiles, (m + kA8Tokens - 1) / kA8Tokens), block(kA8Tokens);
