@@ -330,6 +330,32 @@ def test_one_scratch_buffer_serves_calls_of_different_shapes_and_kernels(goq):
         assert torch.equal(want, got), (li, op, m)
 
 
+@pytest.mark.parametrize("m", [100, 700])
+def test_gemm_output_alignment_does_not_change_the_result(goq, m):
+    """The GEMM epilogue stores 16 bytes per thread when the output allows it and element by element otherwise:
+    an output that starts 4 (fp32) or 2 (bf16) bytes off a 16-byte boundary must hold the same bits."""
+    from tests.gpu_util import pack_weights, dev
+    n, k = 256, 1024
+    codes, meta, coef = si.random_quantized(n, k, 128, 3, seed=91)
+    d, packed = pack_weights(n, k, 128, 3, codes, meta, coef)
+    x = dev(si.bf16_activations(m, k, seed=92))
+    ws = goq.new_workspace(d, goq.OP_GEMM, m)
+    for dtype, code in ((torch.float32, goq.F32), (torch.bfloat16, goq.BF16)):
+        flat = torch.zeros(m * n + 8, dtype=dtype, device="cuda")
+        aligned = flat[:m * n].view(m, n)
+        goq.gemm(d, packed, x, m, goq.BF16, y=aligned, y_dtype=code, ws=ws)
+        torch.cuda.synchronize()
+        want = aligned.clone()
+        flat2 = torch.zeros(m * n + 8, dtype=dtype, device="cuda")
+        shifted = flat2[1:m * n + 1].view(m, n)
+        assert shifted.data_ptr() % 16 != 0
+        goq.gemm(d, packed, x, m, goq.BF16, y=shifted, y_dtype=code, ws=ws)
+        torch.cuda.synchronize()
+        assert goq.workspace_status(ws) == goq.OK
+        assert torch.equal(want, shifted)
+        assert float(flat2[0]) == 0.0 and float(flat2[m * n + 1:].abs().sum()) == 0.0
+
+
 def test_gemm_tail_wave_runs_as_half_tiles(goq):
     """160 output tiles (20 channel tiles x 8 token tiles) on 148 SMs: the 12 tiles of the last wave are scheduled
     as 24 half tiles of 256 tokens; 3900 tokens make the last token tile ragged. Sampled channels, all tokens."""
