@@ -101,6 +101,11 @@ __device__ __forceinline__ uint32_t after_wait(uint32_t addr) {
     asm volatile("mov.u32 %0, %1;" : "=r"(r) : "r"(addr) : "memory");
     return r;
 }
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
 __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -434,13 +439,13 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                     }
                 } else {
                     uint16_t* y = reinterpret_cast<uint16_t*>(p.y);
-                    const uint16_t h0 = f32_to_bf16_rne(f.x), h1 = f32_to_bf16_rne(f.y), h2 = f32_to_bf16_rne(f.z), h3 = f32_to_bf16_rne(f.w);
-                    if (vec) *reinterpret_cast<uint2*>(y + o) = make_uint2((uint32_t)h0 | ((uint32_t)h1 << 16), (uint32_t)h2 | ((uint32_t)h3 << 16));
+                    const uint32_t h01 = pack_bf16x2(f.x, f.y), h23 = pack_bf16x2(f.z, f.w);   // round to nearest even, in hardware
+                    if (vec) *reinterpret_cast<uint2*>(y + o) = make_uint2(h01, h23);
                     else {
-                        if (row4 + 0 < p.n_out) y[o + 0] = h0;
-                        if (row4 + 1 < p.n_out) y[o + 1] = h1;
-                        if (row4 + 2 < p.n_out) y[o + 2] = h2;
-                        if (row4 + 3 < p.n_out) y[o + 3] = h3;
+                        if (row4 + 0 < p.n_out) y[o + 0] = (uint16_t)(h01 & 0xFFFFu);
+                        if (row4 + 1 < p.n_out) y[o + 1] = (uint16_t)(h01 >> 16);
+                        if (row4 + 2 < p.n_out) y[o + 2] = (uint16_t)(h23 & 0xFFFFu);
+                        if (row4 + 3 < p.n_out) y[o + 3] = (uint16_t)(h23 >> 16);
                     }
                 }
             };
