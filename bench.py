@@ -465,6 +465,31 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
     ms = time_graph(torch, g, 20, 3)
     out["gemv_sequence_layer_groups_gbs"] = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack) / (ms * 1e-3) / 1e9
     del g
+    # ... and with the usual serving fusions: q, k, v share their input and become one 12288 x 4096 linear, gate and up
+    # one 22016 x 4096 (row-wise quantization groups make the concatenation exact): 4 dependent linears per layer, same bytes
+    fused_shapes = [(3 * 4096, 4096), (4096, 4096), (2 * 11008, 4096), (4096, 11008)]
+    gen = torch.Generator(device="cuda")
+    fused = []
+    for layer in range(layers):
+        for idx, (n, k) in enumerate(fused_shapes):
+            gen.manual_seed(9000 + layer * 4 + idx)
+            d = goq.desc(n, k, GROUP, WBITS)
+            codes = torch.randint(0, 1 << WBITS, (n, k), dtype=torch.uint8, device="cuda", generator=gen)
+            meta = torch.randint(0, 64, (n, k // 8), dtype=torch.uint8, device="cuda", generator=gen)
+            coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * 0.03).to(torch.float16)
+            packed = torch.empty(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
+            goq.pack(d, codes, meta, coef, packed)
+            x = torch.randn((1, k), device="cuda", generator=gen).to(torch.bfloat16)
+            y = torch.empty((1, n), dtype=torch.float32, device="cuda")
+            fused.append({"d": d, "packed": packed, "x": x, "y": y, "n": n, "k": k})
+            del codes, meta, coef
+    seq_f = goq.make_sequence([(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, j > 0) for j, s in enumerate(fused)])
+    ws_f = torch.empty(goq.sequence_workspace_bytes(len(fused)), dtype=torch.uint8, device="cuda")
+    goq.workspace_init(ws_f)
+    g = capture(torch, lambda: goq.gemv_sequence(seq_f, ws_f))
+    ms = time_graph(torch, g, 20, 3)
+    out["gemv_sequence_fused_qkv_gateup_gbs"] = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in fused) / (ms * 1e-3) / 1e9
+    del g, fused, seq_f
     # per-shape batch-1 time (rotating over the layers' copies of that shape, so each launch reads cold weights)
     shapes = {}
     for idx, (name, n, k) in enumerate(si.LLAMA2_7B_LINEARS):
