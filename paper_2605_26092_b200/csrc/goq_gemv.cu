@@ -201,14 +201,18 @@ __device__ __forceinline__ void expand_word(uint32_t w, uint32_t meta4, const ui
         lb = prmt(PotTables<WB>::L0, PotTables<WB>::L1, mh);
         meta = gather_meta(w);
     } else {
-        ha = hb = la = lb = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            uint32_t c = (w >> (4 * i)) & 15u, sg = c >> 3, e = c & 7u;
-            uint32_t bits = (c == 7u) ? 0u : ((sg << 15) | ((127u - e) << 7));
-            if (i < 4) { ha |= (bits >> 8) << (8 * i); la |= (bits & 0xFFu) << (8 * i); }
-            else { hb |= (bits >> 8) << (8 * (i - 4)); lb |= (bits & 0xFFu) << (8 * (i - 4)); }
-        }
+        // W4: code = sign << 3 | e, value (-1)^sign 2^-e, except sign 0, e 7 = zero. bf16(2^-e) = (127 - e) << 7: the low
+        // byte (0x80 for even e) does not depend on the sign, the high byte comes from a table per sign (the positive
+        // one holds 0 at e = 7), chosen per byte by a mask made of the sign bits: prmt's sign-replicate mode turns the
+        // top bit of each byte of w (odd weights) and of w << 4 (even weights) into 0x00 / 0xFF.
+        constexpr uint32_t PH0 = 0x3E3E3F3Fu, PH1 = 0x003C3D3Du, NH0 = 0xBEBEBFBFu, NH1 = 0xBCBCBDBDu, LL = 0x00800080u;
+        const uint32_t m = w & 0x77777777u, mh = m >> 16;
+        const uint32_t s_odd = prmt(w, 0u, 0xBA98u), s_even = prmt(w << 4, 0u, 0xBA98u);
+        const uint32_t ma = prmt(s_even, s_odd, 0x5140u), mb = prmt(s_even, s_odd, 0x7362u);   // weights 0..3, 4..7
+        ha = (prmt(PH0, PH1, m) & ~ma) | (prmt(NH0, NH1, m) & ma);
+        hb = (prmt(PH0, PH1, mh) & ~mb) | (prmt(NH0, NH1, mh) & mb);
+        la = prmt(LL, LL, m);
+        lb = prmt(LL, LL, mh);
         meta = meta4;
     }
     R[0] = prmt(la, ha, 0x5140u);
