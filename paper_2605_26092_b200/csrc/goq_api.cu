@@ -182,7 +182,10 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
             }
             return GOQ_OK;
         }
-        if (goq::gemm_tc_supported(g) && variant != 2) {
+        // W4 has no streaming GEMV: up to 48 tokens its mma.sync kernel is the faster one (41 us at 16 tokens on
+        // 8192 x 8192 against ~105 us for a tensor-core half tile), so the tensor-core kernel takes W4 from 49 tokens on
+        const bool w4_few = g.wbits == 4 && m <= kGemmViaGemvMaxTokens && variant == 0 && goq::linear_mma_supported(g);
+        if (goq::gemm_tc_supported(g) && variant != 2 && !w4_few) {
             if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
             if (ws_bytes < goq::gemm_tc_workspace(g, m)) return GOQ_ERR_WORKSPACE;
             return from_cuda(goq::launch_gemm_tc(g, packed, x, m, y, y_dtype, ws, (cudaStream_t)stream));

@@ -163,6 +163,10 @@ template <> struct PotBytes<3> {  // +1 +.5 +.25 0 -1 -.5 -.25 -.125
 template <> struct PotBytes<2> {  // +1 0 -1 -.5
     static constexpr uint32_t H0 = 0xB8BC003Cu, H1 = 0u;
 };
+// W4: code = sign << 3 | e, value (-1)^sign 2^-e (fp16 high byte (15 - e) << 2), sign 0 with e = 7 is the zero state
+struct PotBytes4 {
+    static constexpr uint32_t PH0 = 0x3034383Cu, PH1 = 0x0024282Cu, NH0 = 0xB0B4B8BCu, NH1 = 0xA0A4A8ACu;
+};
 constexpr uint32_t kHashMul = 0x01008420u;  // (record bits in place) * kHashMul >> 26 is a bijection onto 0..63
 
 struct ExchangeLut { uint32_t v[64][4]; };
@@ -211,12 +215,26 @@ __device__ __forceinline__ uint32_t hfma2(uint32_t a, uint32_t b, uint32_t c) {
 // halves of a register. b1 and b2 are built as fp16 directly (table high byte over a zero low byte), c1*b1 is a
 // power-of-two scaling (exact) and the fused multiply-add rounds once: the same value as fp32 arithmetic rounded
 // to fp16, for a quarter of the instructions.
+// W <= 3: the exchange record sits in the spare bit of the word's nibbles and is hashed into the table slot. W = 4: the
+// nibbles are full (the sign is bit 3), the record comes from the unit's byte plane (`record`) and the table is filled
+// in record order; the high byte is taken from a positive or a negative table per weight, chosen by a byte mask that
+// prmt's sign-replicate mode makes of the sign bits (top bit of each byte of w: odd weights; of w << 4: even weights).
 template <int WB>
-__device__ __forceinline__ void expand_what(uint32_t w, uint32_t lut_lane, uint32_t c1, uint32_t c2, uint32_t (&out)[4]) {
+__device__ __forceinline__ void expand_what(uint32_t w, uint32_t record, uint32_t lut_lane, uint32_t c1, uint32_t c2, uint32_t (&out)[4]) {
     const uint32_t m = w & 0x77777777u, mh = m >> 16;
-    const uint32_t ha = prmt(PotBytes<WB>::H0, PotBytes<WB>::H1, m), hb = prmt(PotBytes<WB>::H0, PotBytes<WB>::H1, mh);
-    const uint32_t h = (w - m) * kHashMul;
-    const uint4 e = lds128(((h >> 19) & 0x1F80u) | lut_lane);  // table is 8 KiB aligned, lut_lane selects the copy
+    uint32_t ha, hb, slot_off;
+    if constexpr (WB <= 3) {
+        ha = prmt(PotBytes<WB>::H0, PotBytes<WB>::H1, m);
+        hb = prmt(PotBytes<WB>::H0, PotBytes<WB>::H1, mh);
+        slot_off = (((w - m) * kHashMul) >> 19) & 0x1F80u;
+    } else {
+        const uint32_t s_odd = prmt(w, 0u, 0xBA98u), s_even = prmt(w << 4, 0u, 0xBA98u);
+        const uint32_t ma = prmt(s_even, s_odd, 0x5140u), mb = prmt(s_even, s_odd, 0x7362u);   // weights 0..3, 4..7
+        ha = (prmt(PotBytes4::PH0, PotBytes4::PH1, m) & ~ma) | (prmt(PotBytes4::NH0, PotBytes4::NH1, m) & ma);
+        hb = (prmt(PotBytes4::PH0, PotBytes4::PH1, mh) & ~mb) | (prmt(PotBytes4::NH0, PotBytes4::NH1, mh) & mb);
+        slot_off = (record & 63u) << 7;
+    }
+    const uint4 e = lds128(slot_off | lut_lane);  // table is 8 KiB aligned, lut_lane selects the copy
     const uint32_t qa = prmt(ha, hb, e.x) ^ e.z, qb = prmt(ha, hb, e.y) ^ e.w;   // b2: permuted, pair signs applied
     // bytes {0, h[2q], 0, h[2q+1]}: weights 2q, 2q+1 as one f16x2 word
     const uint32_t R[4] = {prmt(ha, 0u, 0x1404u), prmt(ha, 0u, 0x3424u), prmt(hb, 0u, 0x1404u), prmt(hb, 0u, 0x3424u)};
@@ -230,7 +248,7 @@ struct GemmParams {
     void* y;
     const float* inv_scale;   // [m_total] 2^-s of each token (the activations the tensor map covers are x * 2^s in fp16)
     int* status;
-    int unit_bytes, k_blocks, n_tiles, n_out, m_total, y_dtype, group_log2;
+    int unit_bytes, meta_off, k_blocks, n_tiles, n_out, m_total, y_dtype, group_log2;
     // Tile schedule (1-D grid). CTAs [0, n_full) take 128 x 512 tiles, numbered channel-tile fastest; the remaining
     // CTAs take the last tiles as halves of 256 tokens each, so that a last wave that would fill less than half of
     // the SMs runs for half as long on twice as many.
@@ -290,7 +308,13 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < 64 * kLutCopies; i += kThreads) {
-        const uint32_t* e = c_lut.v[i / kLutCopies];
+        uint32_t slot = (uint32_t)(i / kLutCopies);
+        if constexpr (WB == 4) {   // table in record order: entry `record` is the hashed table's entry of that record
+            uint32_t spread = 0;
+            for (int b = 0; b < 6; ++b) spread |= ((slot >> b) & 1u) << (4 * b + 3);
+            slot = (spread * kHashMul) >> 26;
+        }
+        const uint32_t* e = c_lut.v[slot];
         *reinterpret_cast<uint4*>(lut + (size_t)i * 16) = make_uint4(e[0], e[1], e[2], e[3]);
     }
     for (int i = tid; i < kTileM; i += kThreads) inv_s[i] = (tok0 + i < p.m_total) ? __ldg(&p.inv_scale[tok0 + i]) : 1.0f;
@@ -363,7 +387,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
         const int e = warp - 2, g = lane >> 2, t = lane & 3;
         const uint32_t lut_lane = s32(lut) + (uint32_t)(lane & (kLutCopies - 1)) * 16;
         const bool valid = (T0 + e) < p.n_tiles;
-        constexpr uint32_t kZeroWord = (WB == 3) ? 0x33333333u : 0x11111111u;  // every code = the zero state
+        constexpr uint32_t kZeroWord = (WB == 4) ? 0x77777777u : (WB == 3) ? 0x33333333u : 0x11111111u;  // every code = the zero state
         bool ok = true;
         for (int kb = 0; kb < nkb && ok; ++kb) {
             const int ps = kb & 1;
@@ -371,7 +395,11 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
             if (!ok) break;
             const uint32_t unit = after_wait(s32(pk_ring) + ps * pk_slot_bytes + e * p.unit_bytes);
             uint4 wv0 = make_uint4(kZeroWord, kZeroWord, kZeroWord, kZeroWord), wv1 = wv0;
-            if (valid) { wv0 = lds128(unit + lane * 16); wv1 = lds128(unit + 512 + lane * 16); }
+            uint32_t mv0 = 0u, mv1 = 0u;   // (W4) the exchange records of this lane's eight words, one byte each
+            if (valid) {
+                wv0 = lds128(unit + lane * 16); wv1 = lds128(unit + 512 + lane * 16);
+                if constexpr (WB == 4) { mv0 = lds32(unit + p.meta_off + lane * 4); mv1 = lds32(unit + p.meta_off + 128 + lane * 4); }
+            }
             const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
@@ -396,8 +424,8 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                     const uint32_t c1a = prmt(cfa, cfa, 0x1010u), c2a = prmt(cfa, cfa, 0x3232u);
                     const uint32_t c1b = prmt(cfb, cfb, 0x1010u), c2b = prmt(cfb, cfb, 0x3232u);
                     uint32_t oa[4], ob[4];
-                    expand_what<WB>(wa, lut_lane, c1a, c2a, oa);
-                    expand_what<WB>(wb, lut_lane, c1b, c2b, ob);
+                    expand_what<WB>(wa, mv0 >> (8 * c), lut_lane, c1a, c2a, oa);
+                    expand_what<WB>(wb, mv1 >> (8 * c), lut_lane, c1b, c2b, ob);
                     // K-major tile, 128-byte rows, 16-byte chunk j of row r stored at chunk j ^ (r & 7)
                     const int j = cc * 4 + t;
                     const int ra = e * 16 + g, rb = ra + 8;  // (ra & 7) == (rb & 7) == g
@@ -635,6 +663,7 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
     p.inv_scale = inv_scale;
     p.status = status;
     p.unit_bytes = g.unit_bytes;
+    p.meta_off = g.meta_off;
     p.k_blocks = g.k_blocks;
     p.n_tiles = g.n_tiles;
     p.n_out = g.n_out;
@@ -663,7 +692,7 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
 }  // namespace goq
 
 namespace goq {
-bool gemm_tc_supported(const Geometry& g) { return g.wbits <= 3 && g.k_in % 8 == 0 && tc::smem_bytes(g) + 2048 <= 227 * 1024; }
+bool gemm_tc_supported(const Geometry& g) { return g.wbits <= 4 && g.k_in % 8 == 0 && tc::smem_bytes(g) + 2048 <= 227 * 1024; }
 // Scratch: status word and tile counters in the common areas; behind them the per-token inverse scales, the fp16
 // copy of the activations and (split-K) the partial tiles.
 static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
@@ -690,6 +719,7 @@ cudaError_t launch_gemm_tc(const Geometry& g, const void* packed, const void* x,
     uint16_t* xh = (uint16_t*)(b + t.xh_off);
     int* counters = (int*)(b + kWsStatusBytes);   // at most sm_count / 2 tiles when the split is on
     float* partial = (float*)(b + t.partial_off);
+    if (g.wbits == 4) return tc::launch_wb<4>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, counters, partial, st);
     return g.wbits == 3 ? tc::launch_wb<3>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, counters, partial, st)
                         : tc::launch_wb<2>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, counters, partial, st);
 }

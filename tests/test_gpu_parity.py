@@ -205,7 +205,7 @@ def test_config5_llama70b_shapes_bit_width_sweep_sampled_rows(goq, name, b, batc
 @pytest.mark.parametrize("n,k,g,b,m,variant", [
     (80, 384, 128, 3, 150, 0), (80, 384, 128, 3, 150, 2), (256, 512, 64, 3, 600, 0), (40, 192, 32, 2, 17, 0),
     (130, 256, 8, 3, 513, 0), (16, 128, 16, 3, 1, 0), (300, 1152, 128, 3, 1030, 0), (96, 256, 64, 3, 60, 0),
-    (64, 256, 64, 3, 256, 0), (64, 256, 64, 3, 257, 0), (80, 384, 128, 4, 150, 0), (40, 256, 32, 4, 20, 0),
+    (64, 256, 64, 3, 256, 0), (64, 256, 64, 3, 257, 0), (80, 384, 128, 4, 150, 0), (40, 256, 32, 4, 20, 0), (300, 1152, 64, 4, 600, 0), (130, 256, 8, 4, 513, 0),
 ])
 def test_gemm_bf16_small_full_parity(goq, n, k, g, b, m, variant):
     """Prefill GEMM, every output compared. variant 2: the two-operand mma.sync kernel, held to the tight bound.
@@ -220,8 +220,8 @@ def test_gemm_bf16_small_full_parity(goq, n, k, g, b, m, variant):
     y = run_gemm_bf16(d, packed, xb, variant=variant)
     err = O.normwise_rel_err(y, y_ref)
     print("gemm variant %d: normwise error %.3e" % (variant, err))
-    on_tc = variant == 0 and b <= 3 and (m > 48 or g < 32)   # W4 runs on the exact two-operand mma.sync kernel; the streaming
-    # GEMV takes the few-token calls it supports (group >= 32)
+    # up to 48 tokens the streaming GEMV (W <= 3, group >= 32) or the exact mma.sync kernel (W4) takes the call
+    on_tc = variant == 0 and (m > 48 or (g < 32 and b <= 3))
     assert err <= TOL and err <= (GEMM_TC_TOL if on_tc else TIGHT), err
 
 
