@@ -201,6 +201,24 @@ def test_config5_llama70b_shapes_bit_width_sweep_sampled_rows(goq, name, b, batc
     assert err <= TOL and err <= TIGHT, err
 
 
+@pytest.mark.parametrize("name,b,m", [("gqa_kv", 4, 256), ("attn_qo", 2, 64), ("attn_qo", 4, 700)])
+def test_config5_llama70b_shapes_crossover_batches_on_the_gemm(goq, name, b, m):
+    """The batch sweep's upper end (64, 256 tokens and beyond) goes through goq_gemm: 70B-shaped linears at W2 / W4
+    on the tensor-core kernel (split-K at 64 and 256 tokens), sampled rows against the oracle."""
+    from tests.gpu_util import pack_weights, run_gemm_bf16
+    n, k = _CFG5[name]
+    codes, meta, coef = si.random_quantized(n, k, 128, b, seed=n + k + b + 1)
+    rows = si.sample_rows(n, 32, seed=5)
+    w = si.weights_with_student_t_channels(len(rows), k, seed=10)
+    codes[rows], meta[rows], coef[rows] = O.quantize_geo(w, 128, b)
+    d, packed = pack_weights(n, k, 128, b, codes, meta, coef)
+    xb = si.bf16_activations(m, k, seed=m + b)
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 128, b, rows=rows)
+    y = run_gemm_bf16(d, packed, xb)
+    err = O.normwise_rel_err(y[:, rows], y_ref)
+    assert err <= GEMM_TC_TOL, err
+
+
 # ------------------------------------------------------------------------------------- prefill GEMM
 @pytest.mark.parametrize("n,k,g,b,m,variant", [
     (80, 384, 128, 3, 150, 0), (80, 384, 128, 3, 150, 2), (256, 512, 64, 3, 600, 0), (40, 192, 32, 2, 17, 0),
