@@ -377,13 +377,13 @@ def run_cuda(args):
     launch_ms = ms / kernels_per_step
     achieved = launch_bytes / (launch_ms * 1e-3) / 1e9
     if args.launch == "sequence":
-        kernel_name = "gemv_seq_kernel<3,4,true>"
+        kernel_name = "gemv_chain_kernel<3,4,1>"
         launch_desc = "one CUDA graph holding one goq_gemv_sequence call (%d linears, each waits for all earlier ones)" % n_lin
         ratio, ratio_src = NCU_TRAFFIC_RATIO_SEQ, "ncu dram bytes of a 14-linear sequence launch scaled by algorithmic bytes"
         if int(goq.workspace_status(ws_seq)) != 0:
             raise RuntimeError("sequence kernel reported a device-side timeout")
     else:
-        kernel_name = {4: "gemv_tc_kernel<3,1,16>", 2: "linear_mma_kernel<3,1>", 1: "gemv_scalar_kernel"}.get(
+        kernel_name = {2: "linear_mma_kernel<3,1>", 1: "gemv_scalar_kernel"}.get(
             args.gemv_variant, "gemv_stream_kernel<3,1,4,true>")
         launch_desc = "one CUDA graph of %d goq_gemv nodes per step" % n_lin
         # one ncu capture of the 4096x4096 launch read 8.96 MB of DRAM for 8.39 MB of algorithmic bytes;

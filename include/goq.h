@@ -88,7 +88,8 @@ size_t goq_workspace_bytes(const goq_desc* desc, int op, int m);
 goq_status goq_workspace_init(void* ws, size_t ws_bytes, void* stream);
 
 /* Read the device-side status word of a scratch buffer after synchronising `stream`:
- * GOQ_OK, or GOQ_ERR_TIMEOUT if a kernel gave up on a bounded wait (its outputs are then undefined). */
+ * GOQ_OK, or GOQ_ERR_TIMEOUT if a kernel gave up on a bounded wait. Its outputs are then undefined and counters in
+ * the buffer may be left non-zero: zero-fill it again (goq_workspace_init) before the next call that uses it. */
 goq_status goq_workspace_status(const void* ws, void* stream, int* status_out);
 
 /* goq_pack - re-tile quantizer output into the layout the kernels stream (Sections 3.2-3.4 give
@@ -120,9 +121,13 @@ goq_status goq_unpack(const goq_desc* desc, const void* packed, uint8_t* codes_b
  *   ws       scratch of goq_workspace_bytes(desc, GOQ_OP_GEMV, batch) bytes, 256-byte aligned,
  *            initialised once with goq_workspace_init (may be NULL if the size is 0)
  * Each PoT term is applied to the activation as an exponent shift; sums are fp32. Up to 4 tokens
- * whose activations fit the sequence kernel's staging buffer run as a one-linear goq_gemv_sequence
- * in its integer-operand form (same rounding and saturation of non-finite activations as stated
- * there); the other cases take the bf16-operand streaming kernel. */
+ * whose activations fit the chain kernel's staging buffer run as a one-linear goq_gemv_sequence
+ * (integer operands: same rounding and saturation of non-finite activations as stated there);
+ * the other cases take the bf16-operand streaming kernel.
+ * Stream order: the streaming kernel starts fetching `packed` before earlier work on the stream has
+ * finished (programmatic dependent launch), so the packed weights must not be written by work that
+ * is still in flight on the stream when the call is issued (synchronise after goq_pack, or put
+ * other work in between). x and y follow plain stream order. */
 goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16, int batch, void* y,
                     int y_dtype, void* ws, size_t ws_bytes, void* stream);
 
@@ -162,10 +167,13 @@ goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x
  * the process exits); nothing is allocated or freed by this call, by any CUDA call it makes, or through torch.
  *   Arguments as goq_gemv; always the bf16-operand streaming kernel (goq_gemv takes the integer-operand form for
  *   up to 4 tokens, so the two can differ in the last bits, both far inside the stated tolerance).
- *   Limits: the streaming kernel's scratch (status word, tile counters, 1 MiB of parked partial sums) must fit
- *   GOQ_STATIC_SCRATCH_BYTES (it does for every layer that kernel takes: n_out up to 262 144), otherwise
- *   GOQ_ERR_WORKSPACE is returned and nothing is launched; configurations goq_gemv serves with its
- *   scratch-free kernels (group < 32, wbits = 4) return GOQ_ERR_UNSUPPORTED here - use goq_gemv for them.
+ *   Limits: configurations goq_gemv serves with its scratch-free kernels (group < 32, wbits = 4, more than
+ *   16384 row tiles) return GOQ_ERR_UNSUPPORTED here and nothing is launched - use goq_gemv for them. Every layer
+ *   the streaming kernel does take fits the array (status word, tile counters, 1 MiB of parked partial sums);
+ *   GOQ_ERR_WORKSPACE is reserved for a build whose array is smaller than that.
+ *   Status: a kernel that gave up on a bounded wait writes GOQ_ERR_TIMEOUT into the array's first word; read it
+ *   with goq_gemv_static_status (which synchronises the stream) BEFORE the next goq_gemv_static call on the
+ *   device, because every call clears the word.
  *   First call on each device: looks up the array's device address (once per device, with that device
  *   current). Make that first call outside any stream capture.
  *   Sharing: every call on a device uses the same array. The call clears the part that must start at zero
@@ -176,14 +184,18 @@ goq_status goq_gemv_host(const goq_desc* desc, const void* packed, const void* x
 #define GOQ_STATIC_SCRATCH_BYTES (2u * 1024u * 1024u)
 goq_status goq_gemv_static(const goq_desc* desc, const void* packed, const void* x_bf16, int batch, void* y,
                            int y_dtype, void* stream);
+/* Device-side status word of the built-in scratch array of the current device, read after synchronising `stream`
+ * (the paper has no counterpart; allocates nothing: the word is copied through the array's cached address). */
+goq_status goq_gemv_static_status(void* stream, int* status_out);
 
 /* goq_gemv_sequence: a chain of decode GEMVs (Eq. 4, one call of goq_gemv each) executed by ONE persistent
  * cooperative kernel, in order. Results are those of calling goq_gemv item by item on one stream; what changes
  * is the cost: no launch, prologue or first-byte latency per linear, and the weight stream never stops at a
- * boundary between linears. When every item has batch <= 4 the kernel computes with integer operands: the
- * activations of each token and 128-wide k-block become 16-bit fixed point (exact for every element within 2^-7 of
- * the block's largest magnitude, rounded at 2^-15 of it below; measured normwise error ~1e-5 or less), and
- * non-finite activations are not propagated (they saturate). Otherwise bf16 operands, exact products.
+ * boundary between linears. The kernel computes with integer operands: the activations of each token and
+ * 128-wide k-block become 16-bit fixed point (exact for every element within 2^-7 of the block's largest
+ * magnitude, rounded at 2^-15 of it below; measured normwise error ~1e-5 or less), the PoT weights times 2^emax
+ * are small integers, sums are exact in int32 and the coefficient multiply is fp32. Non-finite activations are
+ * not propagated (they saturate).
  *   items    HOST array of n_items entries (read during the call, not kept):
  *            desc, packed, x_bf16 [batch][k_in], y [batch][n_out], y_dtype as in goq_gemv, all device pointers;
  *            depends != 0 : this item's x (or y) may alias outputs of EARLIER items of the sequence - the kernel
@@ -191,12 +203,14 @@ goq_status goq_gemv_static(const goq_desc* desc, const void* packed, const void*
  *            depends == 0 : x and y are independent of every earlier item (their buffers must not overlap the
  *                           outputs of earlier items).
  *   Constraints (else GOQ_ERR_UNSUPPORTED): every item has the same wbits (2 or 3) and group (32, 64, 128),
- *   batch <= 8, and batch * round_up(k_in, 128) * 2 bytes <= 139264 (the activations are staged in shared memory;
- *   up to 23040 bytes two CTAs share an SM, above that the launch takes one CTA per SM), k_in <= 12288.
- *   ws       goq_sequence_workspace_bytes(n_items) bytes, 256-byte aligned, zeroed once with goq_workspace_init;
- *            the call leaves it zero. One status word as for goq_gemv (goq_workspace_status).
+ *   batch <= 8, k_in <= 12288, and the staged activations (2 * batch * (round_up(k_in, 128) + 32) bytes) fit in
+ *   shared memory beside two 16-record stages of the weight stream (about 180 KB: batch 8 up to k_in = 11008).
+ *   ws       goq_sequence_workspace_bytes(n_items) bytes, 256-byte aligned, zero-filled once with
+ *            goq_workspace_init; every call leaves it ready for the next one. Its first word is the status word
+ *            (goq_workspace_status): after GOQ_ERR_TIMEOUT the outputs are undefined and the buffer must be
+ *            zero-filled again before it is reused.
  * Sequences longer than GOQ_SEQUENCE_MAX_ITEMS are split into several launches. The device must support
- * cooperative launches (every sm_100 device does); the grid is sized so that all CTAs are resident. */
+ * cooperative launches (every sm_100 device does); the grid is one CTA per SM, all resident. */
 typedef struct {
     goq_desc desc;
     const void* packed;
@@ -226,11 +240,14 @@ goq_status goq_gemv_sequence_host(const goq_gemv_item* items, int n_items, const
 int goq_last_cuda_error(void);
 
 /* Force a kernel variant (benchmarks and tests only): 0 = automatic, 1 = scalar exponent-add
- * kernel, 2 = tensor-core fragment kernel, 3 = streaming tensor-core kernel, 4 = tcgen05 kernel with
- * the FP8 weight operand in tensor memory, 5 = goq_gemv_sequence always with bf16 operands (it uses integer
- * operands when every item has batch <= 4). Process-wide.
- * Returns the previous value. */
+ * kernel, 2 = tensor-core fragment kernel, 3 = streaming tensor-core kernel. Process-wide. Returns the
+ * previous value. */
 int goq_set_gemv_variant(int variant);
+
+/* Bound, in polls, of every device-side wait of goq_gemv_sequence (tests only; 0 restores the kernel's own bound).
+ * With a bound of a few polls a dependent chain gives up at once: the call returns GOQ_OK (it only enqueues), the
+ * status word then reads GOQ_ERR_TIMEOUT, the context stays usable. Process-wide. Returns the previous value. */
+int goq_set_wait_limit(int polls);
 
 #ifdef __cplusplus
 }

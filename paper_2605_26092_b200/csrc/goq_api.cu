@@ -10,6 +10,7 @@ using goq::Geometry;
 namespace {
 
 std::atomic<int> g_gemv_variant{0};
+std::atomic<int> g_wait_limit{0};   // 0: the kernels' own bound on device-side waits
 constexpr int kGemmViaGemvMaxTokens = 48;
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -32,14 +33,18 @@ goq_status check_arch() {
 }
 
 std::atomic<int> g_last_cuda_error{0};
-goq_status from_cuda(cudaError_t e) {
+goq_status from_cuda(cudaError_t e) { return goq::status_from_cuda(e); }
+
+}  // namespace
+
+namespace goq {
+goq_status status_from_cuda(cudaError_t e) {
     if (e == cudaSuccess) return GOQ_OK;
     (void)cudaGetLastError();  // do not leave a non-sticky error behind for the next call to trip over
     g_last_cuda_error.store((int)e, std::memory_order_relaxed);
     return GOQ_ERR_CUDA;
 }
-
-}  // namespace
+}  // namespace goq
 
 extern "C" {
 
@@ -76,7 +81,7 @@ size_t goq_workspace_bytes(const goq_desc* desc, int op, int m) {
     if (op == GOQ_OP_GEMV && m <= 16) {
         size_t need = 0;
         if (goq::gemv_stream_supported(g)) need = goq::gemv_stream_workspace(g);
-        if (goq::gemv_tc_supported(g, m) && goq::gemv_tc_workspace(g) > need) need = goq::gemv_tc_workspace(g);
+        if (m <= 4 && goq::gemv_seq_supported(g, m) && goq::gemv_seq_workspace(1) > need) need = goq::gemv_seq_workspace(1);
         return need;
     }
     if (op == GOQ_OP_GEMM) {
@@ -119,29 +124,18 @@ goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16
         return GOQ_ERR_ALIGNMENT;
     if (goq_status s = check_arch()) return s;
     const int variant = g_gemv_variant.load(std::memory_order_relaxed);
-    // the tensor-memory kernel is selectable but not the default: its tcgen05 A-operand feed caps it below the
-    // streaming kernel's rate on this part
-    const bool use_tc = goq::gemv_tc_supported(g, batch) && variant == 4;
-    if (variant == 4 && !use_tc) return GOQ_ERR_UNSUPPORTED;
-    if (use_tc) {
-        if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
-        if (ws_bytes < goq::gemv_tc_workspace(g)) return GOQ_ERR_WORKSPACE;
-        if (!goq::stream_hash_is_bijective()) return GOQ_ERR_UNSUPPORTED;
-        return from_cuda(goq::launch_gemv_tc(g, packed, x_bf16, batch, y, y_dtype, ws, (cudaStream_t)stream));
-    }
     bool use_stream = goq::gemv_stream_supported(g) && (variant == 0 || variant == 3);
     if (variant == 3 && !use_stream) return GOQ_ERR_UNSUPPORTED;
     if (use_stream) {
         if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
         if (ws_bytes < goq::gemv_stream_workspace(g)) return GOQ_ERR_WORKSPACE;
         if (!goq::stream_hash_is_bijective()) return GOQ_ERR_UNSUPPORTED;
-        // Up to 4 tokens whose activations fit the sequence kernel's staging buffer: its integer-operand form as a
-        // one-linear sequence is the faster kernel (13.6 against 15.3 us per linear over the Llama-2-7B shapes at
-        // batch 1). A refused cooperative launch falls through to the streaming kernel.
+        // Up to 4 tokens whose activations fit the chain kernel's staging buffer: that kernel as a one-linear chain
+        // is the faster one. A refused cooperative launch falls through to the streaming kernel.
         if (variant == 0 && batch <= 4 && goq::gemv_seq_supported(g, batch) && ws_bytes >= goq::gemv_seq_workspace(1)) {
             goq::SeqCall c{g, packed, x_bf16, y, batch, y_dtype, 0};
-            goq::g_seq_int8 = true;
-            if (goq::launch_gemv_seq(&c, 1, g.wbits, g.group, g.unit_bytes, ws, (cudaStream_t)stream) == cudaSuccess)
+            if (goq::launch_gemv_seq(&c, 1, g.wbits, g.group, g.unit_bytes, ws, g_wait_limit.load(std::memory_order_relaxed),
+                                     (cudaStream_t)stream) == cudaSuccess)
                 return GOQ_OK;
             (void)cudaGetLastError();
         }
@@ -240,12 +234,11 @@ goq_status goq_gemv_sequence(const goq_gemv_item* items, int n_items, void* ws, 
     if (ws_bytes < goq::gemv_seq_workspace(n_items)) return GOQ_ERR_WORKSPACE;
     if (goq_status s = check_arch()) return s;
     if (!goq::stream_hash_is_bijective()) return GOQ_ERR_UNSUPPORTED;
-    goq::g_seq_int8 = g_gemv_variant.load(std::memory_order_relaxed) != 5;
     for (int i0 = 0; i0 < n_items; i0 += goq::kSeqMaxItems) {
         const int n = (n_items - i0 < goq::kSeqMaxItems) ? (n_items - i0) : goq::kSeqMaxItems;
         // a chunk boundary is a kernel boundary on the stream: the first item of a chunk needs no counter wait
         cudaError_t e = goq::launch_gemv_seq(&calls[(size_t)i0], n, calls[0].g.wbits, calls[0].g.group, calls[0].g.unit_bytes, ws,
-                                             (cudaStream_t)stream);
+                                             g_wait_limit.load(std::memory_order_relaxed), (cudaStream_t)stream);
         if (e != cudaSuccess) return from_cuda(e);
     }
     return GOQ_OK;
@@ -306,5 +299,7 @@ goq_status goq_workspace_status(const void* ws, void* stream, int* status_out) {
 int goq_last_cuda_error(void) { return g_last_cuda_error.load(std::memory_order_relaxed); }
 
 int goq_set_gemv_variant(int variant) { return g_gemv_variant.exchange(variant); }
+
+int goq_set_wait_limit(int polls) { return g_wait_limit.exchange(polls > 0 ? polls : 0); }
 
 }  // extern "C"

@@ -7,7 +7,8 @@
 //     128 k) and loads the 512 x 64 bf16 activation tile with two 2-D TMA copies (128-byte swizzle);
 //   - eight expander warps decode the records (same byte-table decode and record lookup as the GEMV:
 //     b1 from the code bytes, b2 = byte-permuted b1 with pair signs, Section 3.3), form
-//     w_hat = c1*b1 + c2*b2 in fp32, round once to fp16 and store the 128 x 64 operand tile to shared
+//     w_hat = c1*b1 + c2*b2 with one half2 multiply and one half2 fma (a single rounding to fp16: the products
+//     c*b are exact scalings of c) and store the 128 x 64 operand tile to shared
 //     memory in the K-major, 128-byte-swizzled layout the tensor core reads;
 //   - one thread issues tcgen05.mma (M=128, N=256, K=16, fp16 x fp16 -> fp32) into a 128 x 512 fp32
 //     accumulator that fills the SM's tensor memory, and commits each stage back to the producers.

@@ -1,0 +1,757 @@
+// A chain of decode GEMVs (batch <= 8) in ONE persistent kernel: one CTA per SM, resident for the whole chain.
+//
+// Work split. The unit records of a linear (16 rows x 128 k each, Section 3.1's macro-blocks tiled 16 rows high)
+// are numbered tile by tile, k-block by k-block, which is also their order in the packed buffer. CTA c of G takes
+// the contiguous range [U c / G, U (c+1) / G) of the U records of every linear: equal bytes per SM whatever the
+// shape. A range is consumed 16 records at a time (one ring stage = one bulk copy), record w of a stage by
+// consumer warp w; a last stage of n < 16 records is split at the granularity of a 32-wide k-chunk so that the
+// 4n chunks are spread evenly over the 16 warps.
+//
+// Roles. 16 consumer warps do the arithmetic and touch global memory only to read activations. One producer
+// thread keeps the weight stream going, across the boundaries between linears too (weights do not depend on
+// results). One control warp does everything else that waits on global memory: per 16-row tile part it adds the
+// 16 partial sums the consumer warps parked in shared memory (warp order) and stores the outputs; a tile whose
+// records fall into several CTAs is finished by the CTA that holds its end, the others post their part in scratch
+// (each value in one 64-bit word together with a per-launch tag: no fence, no counter), and the finisher adds the
+// parts in CTA order - deterministic. A range that ends inside a tile is walked starting with that open tile, so
+// the posted parts are early and a finisher waits only on lower-numbered CTAs. The control warp then reports the
+// linear finished on a device-wide counter and, before a linear flagged `depends`, waits until every CTA has.
+//
+// Math per record (Eq. 4 of the paper, integer operands): every PoT state times 2^emax is a small integer, so b1
+// is one byte-table lookup per four weights; b2 = the same bytes routed by "partner i XOR s" (Section 3.3) with
+// the pair signs applied as  sum_k q_k x_k - 2 sum_{k flipped} q_k x_k : the second operand is the first one
+// masked, which costs one AND per register (a flipped zero contributes 0 - 0). The activations of a token and a
+// 128-wide k-block are 16-bit fixed point Q = 256 q0 + q1 (two int8 columns of the MMA's B operand), the sums are
+// exact in int32, and the coefficient multiply happens once per macro-block in fp32, outside the inner product.
+//
+// Every wait is bounded; on expiry an abort flag is raised, every role leaves its loops (all waits watch the flag),
+// copies in flight are drained and GOQ_ERR_TIMEOUT is written to the status word.
+#include "goq_stream_core.cuh"
+#include "goq_internal.h"
+
+namespace goq {
+namespace chain {
+
+constexpr int kNW = 16;                      // consumer warps
+constexpr int kCtrlWarp = kNW;               // polls the completion counters
+constexpr int kProdWarp = kNW + 1;           // issues the bulk copies
+constexpr int kThreads = (kNW + 2) * 32;
+constexpr int kStageRecs = kNW;
+constexpr int kTileSlots = 4;                // in-CTA reduction slots (tile parts in flight)
+constexpr int kXPad = 32;                    // bytes between activation planes beyond k_pad: keeps the B-fragment loads conflict-free
+constexpr int kMaxKBlocks = 96;              // activation scales kept per k-block: k_in <= 12288
+constexpr int kGlobalSpin = 1 << 20;
+constexpr int kMaxStages = 8;
+
+struct Item {
+    const uint8_t* packed;
+    const uint16_t* x;
+    void* y;
+    unsigned long long kb_magic;             // ceil(2^32 / k_blocks): record number -> tile by multiply and shift (exact while units * k_blocks < 2^32)
+    unsigned int units;                      // n_tiles * k_blocks
+    int n_tiles, k_blocks, k_in, n_out, m, y_dtype, depends;
+};
+struct Params {
+    Item item[kSeqMaxItems];
+    int n_items, unit_bytes, n_stages, x_double, xbuf_bytes, spin_limit;
+    int* status;
+    int* done;       // [n_items] CTAs that have finished each linear; zero on entry, left zero
+    unsigned* epoch; // launches this scratch buffer has seen: tags the posted parts (zero-filled scratch carries no valid tag)
+    uint2* parts;    // [n_items][G][2][32 lanes x 2 NG] posted partial sums, each value in one 64-bit word with its tag
+};
+
+constexpr int kPartWords = 128;              // 64-bit (value, tag) words of one posted part: 16 rows x 8 tokens
+
+// ---- small helpers ---------------------------------------------------------------------------------
+template <int WB> struct IntTables;
+template <> struct IntTables<3> { static constexpr uint32_t P0 = 0x00020408u, P1 = 0xFFFEFCF8u; };  // 8 4 2 0 -8 -4 -2 -1
+template <> struct IntTables<2> { static constexpr uint32_t P0 = 0xFFFE0002u, P1 = 0u; };           // 2 0 -2 -1
+
+// volatile: stays behind the waits (also volatile) that make the activation planes valid
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ float ld_cg_f32(const float* p) {
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+    return v;
+}
+// mbarrier operations by 32-bit shared-window address (no generic-to-shared conversion in the hot loop)
+__device__ __forceinline__ bool try_wait_a(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void arrive_a(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// slow path of a wait whose first probe failed: bounded, gives up when another thread has
+__device__ __noinline__ bool wait_slow_a(uint32_t bar, uint32_t parity, volatile int* abort_flag, int limit) {
+    for (int it = 0; it < limit; ++it) {
+        if (try_wait_a(bar, parity)) return true;
+        if ((it & 63) == 63 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int limit) {
+    for (int it = 0; it < limit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63) == 63 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+// One micro-block word -> int8 operands (value * 2^emax): b1 (pa: weights 0..3, pb: 4..7), the routed bytes of
+// b2 (qa, qb) and the same bytes at the sign-flipped positions only (fa, fb).
+template <int WB>
+__device__ __forceinline__ void decode_word(uint32_t w, uint32_t lut_lane, uint32_t& pa, uint32_t& pb, uint32_t& qa,
+                                            uint32_t& qb, uint32_t& fa, uint32_t& fb) {
+    const uint32_t m = w & 0x77777777u, mh = m >> 16;
+    pa = prmt_b32(IntTables<WB>::P0, IntTables<WB>::P1, m);
+    pb = prmt_b32(IntTables<WB>::P0, IntTables<WB>::P1, mh);
+    const uint32_t h = (w & 0x88888888u) * kHashMul;
+    const uint4 e = lds128(((h >> 19) & 0x1F80u) | lut_lane);   // selectors x, y; 0xFF at the flipped bytes z, w
+    qa = prmt_b32(pa, pb, e.x);
+    qb = prmt_b32(pa, pb, e.y);
+    fa = qa & e.z;
+    fb = qb & e.w;
+}
+
+// The range of CTA `cta` of `G` over `units` records, and the order it is walked in.
+struct Walk {
+    unsigned a, b, L;        // range [a, b), length
+    unsigned L1, s1;         // the first L1 positions are records s1, s1+1, ... (the open tile at the end of the range); then a, a+1, ...
+    int Ta, Tb, P;           // first and last tile touched, number of tile parts
+    bool rot;
+};
+__device__ __forceinline__ Walk make_walk(const Item& it, int cta, int G) {
+    Walk w;
+    w.a = (unsigned)((unsigned long long)it.units * (unsigned)cta / (unsigned)G);
+    w.b = (unsigned)((unsigned long long)it.units * (unsigned)(cta + 1) / (unsigned)G);
+    w.L = w.b - w.a;
+    w.L1 = 0; w.s1 = 0; w.Ta = 0; w.Tb = 0; w.P = 0; w.rot = false;
+    if (w.L) {
+        const unsigned kb = (unsigned)it.k_blocks;
+        w.Ta = (int)(w.a / kb);
+        w.Tb = (int)((w.b - 1) / kb);
+        w.P = w.Tb - w.Ta + 1;
+        w.rot = w.Tb > w.Ta && (w.b % kb) != 0;
+        if (w.rot) { w.s1 = (unsigned)w.Tb * kb; w.L1 = w.b - w.s1; }
+    }
+    return w;
+}
+__device__ __forceinline__ unsigned walk_record(const Walk& w, unsigned j) { return j < w.L1 ? w.s1 + j : w.a + (j - w.L1); }
+__device__ __forceinline__ int walk_part_of_tile(const Walk& w, int T) { return w.rot ? (T == w.Tb ? 0 : 1 + T - w.Ta) : T - w.Ta; }
+__device__ __forceinline__ int walk_tile_of_part(const Walk& w, int q) { return w.rot ? (q == 0 ? w.Tb : w.Ta + q - 1) : w.Ta + q; }
+
+// CTA that owns record r of a linear with `units` records split over G CTAs
+__device__ __forceinline__ int owner_of(unsigned long long r, unsigned units, int G) {
+    return (int)(((r + 1) * (unsigned)G - 1) / units);
+}
+
+// ---- hand-over of one tile part (kept out of line) ------------------------------------------------------
+// A consumer warp parks its sums of part number sq (counted per CTA over the whole chain) in reduction slot sq % kTileSlots
+// and arrives on the slot's mbarrier; the control warp adds the 16 partials, stores or passes on the result and then
+// frees the slot. Returns false after a give-up.
+struct FlushCtx {
+    float* red;
+    uint64_t* part_bar;
+    volatile int* done_gen;
+    volatile int* abort_flag;
+    int spin;
+};
+struct Sums4 { float v[4]; };   // by value: the accumulators never have their address taken, so they stay in registers
+template <int NG>
+__device__ __noinline__ bool flush_part(const FlushCtx& c, unsigned sq, Sums4 sums) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
+    const int rs = (int)(sq % kTileSlots);
+    if (*c.abort_flag) return false;
+    if (sq >= (unsigned)kTileSlots) {   // the slot's previous part must have been taken over
+        int spins = 0;
+        while (c.done_gen[rs] != (int)(sq - kTileSlots + 1)) {
+            if (*c.abort_flag || ++spins > c.spin) { *c.abort_flag = 1; return false; }
+            __nanosleep(20);
+        }
+    }
+    float* rb = c.red + ((size_t)rs * kNW + warp) * (NG * 64);
+#pragma unroll
+    for (int cg = 0; cg < NG; ++cg) {
+        rb[cg * 64 + g * 4 + t] = sums.v[2 * cg];
+        rb[cg * 64 + (g + 8) * 4 + t] = sums.v[2 * cg + 1];
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&c.part_bar[rs]);   // releases the warp's stores (ordered before it by the barrier above)
+    return true;
+}
+
+// sums of one macro-block -> fp32, times the coefficients (outside the inner product, Eq. 4)
+template <int NG>
+__device__ __forceinline__ void group_end(int (&s1)[NG][4], int (&s2)[NG][4], int (&s3)[NG][4], uint32_t cfa, uint32_t cfb, float (&rec)[NG][2]) {
+    const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
+    const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
+    const float c1b = __half2float(__ushort_as_half((unsigned short)(cfb & 0xFFFFu)));
+    const float c2b = __half2float(__ushort_as_half((unsigned short)(cfb >> 16)));
+#pragma unroll
+    for (int cg = 0; cg < NG; ++cg) {
+        // columns 2t, 2t+1 hold the high and low activation slices of one token: S = 256 S_hi + S_lo, exact in int32
+        rec[cg][0] += c1a * (float)(s1[cg][0] * 256 + s1[cg][1]) + c2a * (float)((s2[cg][0] - 2 * s3[cg][0]) * 256 + (s2[cg][1] - 2 * s3[cg][1]));
+        rec[cg][1] += c1b * (float)(s1[cg][2] * 256 + s1[cg][3]) + c2b * (float)((s2[cg][2] - 2 * s3[cg][2]) * 256 + (s2[cg][3] - 2 * s3[cg][3]));
+#pragma unroll
+        for (int r = 0; r < 4; ++r) s1[cg][r] = s2[cg][r] = s3[cg][r] = 0;
+    }
+}
+
+template <int WB, int CPG, int NG>
+__global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_constant__ Params p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* lut = smem + ((8192u - (smem_u32(smem) & 8191u)) & 8191u);   // 8 KiB boundary: slot offsets are OR-ed in
+    const int stage_bytes = kStageRecs * p.unit_bytes;
+    unsigned char* ring = lut + kLutBytes;
+    float* red = reinterpret_cast<float*>(ring + (size_t)p.n_stages * stage_bytes);     // [slot][warp][NG][64]
+    float* xscale = red + kTileSlots * kNW * NG * 64;                                   // [2][k-block][4 NG tokens]
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(xscale + 2 * kMaxKBlocks * 4 * NG);
+    uint64_t* empty_bar = full_bar + kMaxStages;
+    uint64_t* dep_bar = empty_bar + kMaxStages;
+    uint64_t* x_bar = dep_bar + 1;
+    uint64_t* free_bar = x_bar + 1;
+    uint64_t* part_bar = free_bar + 1;
+    unsigned char* xq = reinterpret_cast<unsigned char*>(part_bar + kTileSlots);                 // [2][2 m][k_pad + kXPad] int8 planes
+    __shared__ volatile int abort_flag;
+    __shared__ volatile int done_gen[kTileSlots];
+
+    // the broadcast tells the compiler that the warp index (and everything derived from it) is uniform across the warp
+    const int tid = threadIdx.x, warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0), lane = tid & 31;
+    const int G = (int)gridDim.x, cta = (int)blockIdx.x;
+    const int spin = p.spin_limit;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int i = 0; i < kTileSlots; ++i) { done_gen[i] = 0; mbar_init(&part_bar[i], kNW); }
+        for (int s = 0; s < p.n_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kNW); }
+        mbar_init(dep_bar, 1);
+        mbar_init(x_bar, kNW);
+        mbar_init(free_bar, kNW);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i < 64 * kLutCopies; i += kThreads) {
+        const uint32_t* e = c_exchange_lut.v[i / kLutCopies];
+        *reinterpret_cast<uint4*>(lut + (size_t)i * 16) = make_uint4(e[0], e[1], (e[2] >> 7) * 255u, (e[3] >> 7) * 255u);
+    }
+    __syncthreads();
+
+    // ================= producer: the weight stream of this CTA's ranges, linear after linear =================
+    if (warp == kProdWarp) {
+        if (lane == 0) {
+            int slot = 0, round = 0, issued = 0;
+            bool ok = true;
+            for (int i = 0; i < p.n_items && ok; ++i) {
+                const Item& it = p.item[i];
+                const Walk wk = make_walk(it, cta, G);
+                for (unsigned j0 = 0; j0 < wk.L; j0 += kStageRecs) {
+                    if (round > 0 && !wait_bar(&empty_bar[slot], (round - 1) & 1, &abort_flag, spin)) { ok = false; break; }
+                    const unsigned n = min((unsigned)kStageRecs, wk.L - j0);
+                    unsigned char* dst = ring + (size_t)slot * stage_bytes;
+                    mbar_arrive_expect_tx(&full_bar[slot], n * (unsigned)p.unit_bytes);
+                    // positions j0 .. j0+n-1 of the walk: one run of records, or two if the stage straddles the turn of the walk
+                    const unsigned n1 = (j0 < wk.L1) ? min(n, wk.L1 - j0) : 0u;
+                    if (n1) bulk_copy_g2s(dst, it.packed + (size_t)walk_record(wk, j0) * p.unit_bytes, n1 * (unsigned)p.unit_bytes, &full_bar[slot]);
+                    if (n > n1)
+                        bulk_copy_g2s(dst + (size_t)n1 * p.unit_bytes, it.packed + (size_t)walk_record(wk, j0 + n1) * p.unit_bytes,
+                                      (n - n1) * (unsigned)p.unit_bytes, &full_bar[slot]);
+                    if (++slot == p.n_stages) { slot = 0; ++round; }
+                    ++issued;
+                }
+            }
+            // after a give-up the copies this thread issued must still land before the CTA (and its shared memory) goes away
+            if (!ok || abort_flag) {
+                const int first = issued > p.n_stages ? issued - p.n_stages : 0;
+                for (int s = first; s < issued; ++s) {
+                    const int sl = s % p.n_stages;
+                    const uint32_t parity = (uint32_t)(s / p.n_stages) & 1u;
+                    for (int t = 0; t < kSpinLimit && !mbar_try_wait(&full_bar[sl], parity); ++t) { }
+                }
+                atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
+            }
+        }
+        return;
+    }
+
+    // ================= control: everything that touches global memory apart from the activations =================
+    // Per linear and tile part of this CTA: add the 16 parked partials in warp order; a part that covers its whole tile is
+    // stored, another one is parked in scratch, and the last CTA of the tile to arrive adds all parts in CTA order and
+    // stores. Then report the CTA finished; before a dependent linear, wait until every CTA has reported.
+    if (warp == kCtrlWarp) {
+        unsigned seq = 0;
+        bool ok = true;
+        // nobody changes the count before every CTA has finished the last linear; the tag is the count scrambled (and odd,
+        // hence non-zero), so that neither zero-filled scratch nor small integers left by other kernels pass for it
+        const unsigned epoch = *p.epoch, tag = ((epoch + 1u) * 0x9E3779B1u) | 1u;
+        for (int i = 0; i < p.n_items && ok; ++i) {
+            const Item& it = p.item[i];
+            const Walk wk = make_walk(it, cta, G);
+            if (wk.L) {
+                if (it.depends && i > 0) {
+                    if (lane == 0) {
+                        int spins = 0;
+                        while (abort_flag == 0 && ld_acquire_gpu(&p.done[i - 1]) < G)
+                            if (++spins > kGlobalSpin || spins > spin) { abort_flag = 1; break; }
+                        if (abort_flag == 0) mbar_arrive(dep_bar);
+                    }
+                    __syncwarp();
+                    if (abort_flag) { ok = false; break; }
+                }
+                const int kb = it.k_blocks;
+                for (int q = 0; q < wk.P; ++q) {
+                    const unsigned sq = seq + (unsigned)q;
+                    const int rs = (int)(sq % kTileSlots);
+                    if (!wait_bar(&part_bar[rs], (sq / kTileSlots) & 1u, &abort_flag, spin)) { ok = false; break; }
+                    const float* rall = red + (size_t)rs * kNW * (NG * 64);
+                    float out[NG][2];
+#pragma unroll
+                    for (int cg = 0; cg < NG; ++cg)
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            float v[kNW];
+#pragma unroll
+                            for (int w2 = 0; w2 < kNW; ++w2) v[w2] = rall[(size_t)w2 * (NG * 64) + cg * 64 + hh * 32 + lane];
+                            float sum = 0.f;
+#pragma unroll
+                            for (int w2 = 0; w2 < kNW; ++w2) sum += v[w2];   // warp order
+                            out[cg][hh] = sum;
+                        }
+                    __syncwarp();
+                    if (lane == 0) done_gen[rs] = (int)(sq + 1);   // the slot may be parked in again
+                    const int T = walk_tile_of_part(wk, q);
+                    const unsigned long long r_lo = (unsigned long long)T * (unsigned)kb, r_hi = r_lo + (unsigned)kb;
+                    bool store = r_lo >= wk.a && r_hi <= wk.b;
+                    if (!store) {
+                        const int c_first = owner_of(r_lo, it.units, G), c_last = owner_of(r_hi - 1, it.units, G);
+                        // The CTA that holds the end of the tile finishes it; the others post their part and go on. A posted
+                        // value travels in one 64-bit word with the launch's tag, so it needs no fence and no counter: the
+                        // finisher reads the words until the tag is there. Every CTA walks its range starting with the tile
+                        // that is open at the range's end, so the posted parts are early, and the finisher waits only on
+                        // lower-numbered CTAs (no cycle).
+                        if (cta != c_last) {
+                            uint2* mine = p.parts + (((size_t)i * G + cta) * 2 + (T == wk.Ta ? 0 : 1)) * kPartWords;
+#pragma unroll
+                            for (int cg = 0; cg < NG; ++cg)
+#pragma unroll
+                                for (int hh = 0; hh < 2; ++hh)
+                                    asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(mine + (cg * 2 + hh) * 32 + lane),
+                                                 "r"(__float_as_uint(out[cg][hh])), "r"(tag) : "memory");
+                        } else {
+                            float sum[NG][2];
+#pragma unroll
+                            for (int cg = 0; cg < NG; ++cg) sum[cg][0] = sum[cg][1] = 0.f;
+                            bool good = true;
+                            for (int cc = c_first; cc < c_last && good; ++cc) {   // CTA order; this CTA's own part comes last
+                                const unsigned ac = (unsigned)((unsigned long long)it.units * (unsigned)cc / (unsigned)G);
+                                if (ac == (unsigned)((unsigned long long)it.units * (unsigned)(cc + 1) / (unsigned)G)) continue;   // empty range
+                                const uint2* pc = p.parts + (((size_t)i * G + cc) * 2 + ((int)(ac / (unsigned)kb) == T ? 0 : 1)) * kPartWords;
+                                int spins = 0;
+                                for (;;) {
+                                    uint2 w[NG][2];
+                                    bool all = true;
+#pragma unroll
+                                    for (int cg = 0; cg < NG; ++cg)
+#pragma unroll
+                                        for (int hh = 0; hh < 2; ++hh) {
+                                            asm volatile("ld.relaxed.gpu.global.v2.u32 {%0, %1}, [%2];" : "=r"(w[cg][hh].x), "=r"(w[cg][hh].y)
+                                                         : "l"(pc + (cg * 2 + hh) * 32 + lane) : "memory");
+                                            all = all && w[cg][hh].y == tag;
+                                        }
+                                    if (__all_sync(0xFFFFFFFFu, all)) {
+#pragma unroll
+                                        for (int cg = 0; cg < NG; ++cg) { sum[cg][0] += __uint_as_float(w[cg][0].x); sum[cg][1] += __uint_as_float(w[cg][1].x); }
+                                        break;
+                                    }
+                                    if (abort_flag || ++spins > kGlobalSpin || spins > spin) { abort_flag = 1; good = false; break; }
+                                }
+                            }
+                            if (!good) { ok = false; break; }
+#pragma unroll
+                            for (int cg = 0; cg < NG; ++cg) { out[cg][0] += sum[cg][0]; out[cg][1] += sum[cg][1]; }
+                            store = true;
+                        }
+                    }
+                    if (store) {
+#pragma unroll
+                        for (int cg = 0; cg < NG; ++cg)
+#pragma unroll
+                            for (int hh = 0; hh < 2; ++hh) {
+                                const int row = T * 16 + hh * 8 + (lane >> 2), tok = cg * 4 + (lane & 3);
+                                if (row < it.n_out && tok < it.m) {
+                                    if (it.y_dtype == GOQ_F32) reinterpret_cast<float*>(it.y)[(size_t)tok * it.n_out + row] = out[cg][hh];
+                                    else reinterpret_cast<uint16_t*>(it.y)[(size_t)tok * it.n_out + row] = f32_to_bf16_rne(out[cg][hh]);
+                                }
+                            }
+                    }
+                }
+                if (!ok) break;
+                seq += (unsigned)wk.P;
+            }
+            // this CTA has finished linear i: the warp's stores are ordered before lane 0's fetch-add, which releases them
+            __syncwarp();
+            if (lane == 0) {
+                if (i < p.n_items - 1) {
+                    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(&p.done[i]) : "memory");
+                } else {   // the CTA that completes the last linear last leaves the counters zero for the next call
+                    const int prev = atomic_add_acq_rel_gpu(&p.done[i], 1);
+                    if (prev == G - 1) {
+                        for (int j = 0; j < p.n_items; ++j) p.done[j] = 0;
+                        *p.epoch = epoch + 1u;
+                    }
+                }
+            }
+        }
+        if (lane == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
+        return;
+    }
+
+    // ================= consumers =================
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t lut_lane = smem_u32(lut) + (lane & (kLutCopies - 1)) * 16;
+    const uint32_t ring_addr = smem_u32(ring), unit_bytes = (uint32_t)p.unit_bytes;
+    const uint32_t full_addr = smem_u32(full_bar), empty_addr = smem_u32(empty_bar);
+    int slot = 0, phase = 0;          // position in the stage ring
+    uint32_t dep_phase = 0, x_phase = 0, free_phase = 0;
+    int x_sel = 0;                    // activation buffer of the current linear
+    unsigned seq = 0;                 // tile parts this CTA has opened so far (same in every warp): indexes the reduction slots
+    bool alive = true;
+
+    for (int i = 0; i < p.n_items && alive; ++i) {
+        const Item& it = p.item[i];
+        const Walk wk = make_walk(it, cta, G);
+        if (wk.L == 0) continue;   // nothing of this linear belongs to this CTA (the control warp reports it finished)
+        const int kb = it.k_blocks, k_pad = kb * kBlockK, plane = k_pad + kXPad, m = it.m;
+        if (p.x_double) x_sel ^= 1;
+        unsigned char* xb = xq + (size_t)x_sel * p.xbuf_bytes;
+        float* xsc = xscale + x_sel * (kMaxKBlocks * 4 * NG);
+
+        // ---- start of the linear: wait for the dependency, then every warp converts its slice of the activations ----
+        if (it.depends && i > 0) {
+            if (!wait_bar(dep_bar, dep_phase, &abort_flag, spin)) { alive = false; break; }
+            dep_phase ^= 1u;
+        } else if (!p.x_double) {   // one buffer: every warp must have left the previous linear
+            __syncwarp();
+            if (lane == 0) mbar_arrive(free_bar);
+            if (!wait_bar(free_bar, free_phase, &abort_flag, spin)) { alive = false; break; }
+            free_phase ^= 1u;
+        }
+        {
+            // 16-byte chunks of 8 bf16; 16 chunks = one k-block of one token: Q = rne(x 2^s), the block's largest magnitude in [2^14, 2^15)
+            const int cpt = k_pad / 8, total = cpt * m;
+            for (int c0 = warp * 32; c0 < total; c0 += kNW * 32) {
+                const int c = c0 + lane;
+                const bool in = c < total;
+                const int r = in ? c / cpt : 0, k0 = in ? (c - r * cpt) * 8 : 0;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (in && k0 < it.k_in) v = __ldcg(reinterpret_cast<const uint4*>(it.x + (size_t)r * it.k_in + k0));   // L2: written by other SMs
+                const uint32_t in32[4] = {v.x, v.y, v.z, v.w};
+                uint32_t amax = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) amax = max(amax, max(in32[j] & 0x7FFFu, (in32[j] >> 16) & 0x7FFFu));
+#pragma unroll
+                for (int o = 1; o < 16; o <<= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+                int sfield = 268 - (int)(amax >> 7);
+                sfield = sfield < 1 ? 1 : (sfield > 253 ? 253 : sfield);
+                const float mult = __uint_as_float((uint32_t)sfield << 23);
+                uint32_t q0[2] = {0u, 0u}, q1[2] = {0u, 0u};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t bits = (j & 1) ? (in32[j >> 1] & 0xFFFF0000u) : (in32[j >> 1] << 16);
+                    // rne to an integer without a convert: adding 1.5 * 2^23 leaves it in the low mantissa bits
+                    int Q = __float_as_int(fmaf(__uint_as_float(bits), mult, 12582912.0f)) - 0x4B400000;
+                    Q = max(-32639, min(32639, Q));
+                    const int lo = ((Q + 128) & 255) - 128, hi = (Q - lo) >> 8;   // Q = 256 hi + lo, both int8
+                    q0[j >> 2] |= (uint32_t)(hi & 255) << (8 * (j & 3));
+                    q1[j >> 2] |= (uint32_t)(lo & 255) << (8 * (j & 3));
+                }
+                if (in) {
+                    *reinterpret_cast<uint2*>(xb + (size_t)(2 * r) * plane + k0) = make_uint2(q0[0], q0[1]);
+                    *reinterpret_cast<uint2*>(xb + (size_t)(2 * r + 1) * plane + k0) = make_uint2(q1[0], q1[1]);
+                    // 2^-s, and 2^-emax for the integer weights
+                    if ((lane & 15) == 0) xsc[(k0 >> 7) * (4 * NG) + r] = __uint_as_float((uint32_t)(254 - sfield) << 23) * (1.0f / (float)(1 << ((1 << (WB - 1)) - 1)));
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(x_bar);
+            if (!wait_bar(x_bar, x_phase, &abort_flag, spin)) { alive = false; break; }
+            x_phase ^= 1u;
+        }
+        // B fragment of lane (g, t): column g of column group cg = plane 8 cg + g (token 4 cg + g/2, slice g&1), k bytes t*8..t*8+7 of a chunk.
+        // Planes of tokens that do not exist alias the last real plane: an output column depends on its own B column only.
+        uint32_t xrow[NG];
+        uint32_t xs_tok[NG];
+#pragma unroll
+        for (int cg = 0; cg < NG; ++cg) {
+            xrow[cg] = order_after_wait(smem_u32(xb) + (uint32_t)(min(8 * cg + g, 2 * m - 1) * plane + t * 8));
+            xs_tok[cg] = smem_u32(xsc + min(cg * 4 + t, m - 1));
+        }
+        FlushCtx fc;
+        fc.red = red; fc.part_bar = part_bar; fc.done_gen = done_gen; fc.abort_flag = &abort_flag; fc.spin = spin;
+
+        int cur_q = 0;                         // tile part this warp is accumulating
+        float acc[NG][2];
+#pragma unroll
+        for (int cg = 0; cg < NG; ++cg) acc[cg][0] = acc[cg][1] = 0.f;
+        const unsigned n_full = wk.L / kStageRecs, n_tail = wk.L - n_full * kStageRecs;
+        unsigned st = 0;                                                                     // next full stage
+        unsigned u = (unsigned)warp * 4u * n_tail / kNW;                                     // next chunk of the tail stage
+        const unsigned u1 = (unsigned)(warp + 1) * 4u * n_tail / kNW;
+        bool tail_open = false;
+        for (;;) {
+            // ---- the next piece of work of this warp: where it is in the walk, which tile part it belongs to ----
+            const bool in_full = st < n_full, in_tail = !in_full && u < u1;
+            unsigned rho = 0;
+            int T = 0, kbi = 0, qn = wk.P;
+            if (in_full || in_tail) {
+                rho = walk_record(wk, in_full ? st * kStageRecs + warp : n_full * kStageRecs + (u >> 2));
+                T = (int)(((unsigned long long)rho * it.kb_magic) >> 32);
+                kbi = (int)(rho - (unsigned)T * (unsigned)kb);
+                qn = walk_part_of_tile(wk, T);
+            }
+            for (; cur_q < qn; ++cur_q) {   // parts this warp has passed (or never touched: zeros) are handed over
+                Sums4 sums;
+#pragma unroll
+                for (int cg = 0; cg < 2; ++cg) { sums.v[2 * cg] = cg < NG ? acc[cg < NG ? cg : 0][0] : 0.f; sums.v[2 * cg + 1] = cg < NG ? acc[cg < NG ? cg : 0][1] : 0.f; }
+                if (!flush_part<NG>(fc, seq + (unsigned)cur_q, sums)) { alive = false; break; }
+#pragma unroll
+                for (int cg = 0; cg < NG; ++cg) acc[cg][0] = acc[cg][1] = 0.f;
+            }
+            if (!alive) break;
+            if (in_full) {
+                // stages in a row in which this warp's record stays inside tile T and on this side of the turn of the walk
+                const unsigned j = st * kStageRecs + warp;
+                unsigned run = ((unsigned)(kb - kbi) + kStageRecs - 1) / kStageRecs;
+                if (j < wk.L1) run = min(run, (wk.L1 - j + kStageRecs - 1) / kStageRecs);
+                run = min(run, n_full - st);
+                st += run;
+                // ================= the hot loop: one record per iteration =================
+                for (; run; --run, kbi += kStageRecs) {
+                    if (!try_wait_a(full_addr + slot * 8, phase) && !wait_slow_a(full_addr + slot * 8, phase, &abort_flag, spin)) { alive = false; break; }
+                    const uint32_t unit = order_after_wait(ring_addr + slot * stage_bytes + warp * unit_bytes + lane * 16);
+                    const uint4 wv0 = lds128(unit), wv1 = lds128(unit + 512);
+                    const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
+                    const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
+                    int s1[NG][4], s2[NG][4], s3[NG][4];
+                    float rec[NG][2];
+#pragma unroll
+                    for (int cg = 0; cg < NG; ++cg) {
+                        rec[cg][0] = rec[cg][1] = 0.f;
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) s1[cg][r] = s2[cg][r] = s3[cg][r] = 0;
+                    }
+                    const uint32_t koff = (uint32_t)kbi * kBlockK;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t pa0, pb0, qa0, qb0, fa0, fb0, pa1, pb1, qa1, qb1, fa1, fb1;
+                        decode_word<WB>(w0[c], lut_lane, pa0, pb0, qa0, qb0, fa0, fb0);
+                        decode_word<WB>(w1[c], lut_lane, pa1, pb1, qa1, qb1, fa1, fb1);
+#pragma unroll
+                        for (int cg = 0; cg < NG; ++cg) {
+                            const uint2 xf = lds64(xrow[cg] + koff + c * 32);
+                            mma_s8(s1[cg], pa0, pa1, pb0, pb1, xf.x, xf.y);
+                            mma_s8(s2[cg], qa0, qa1, qb0, qb1, xf.x, xf.y);
+                            mma_s8(s3[cg], fa0, fa1, fb0, fb1, xf.x, xf.y);
+                        }
+                        if (((c + 1) % CPG) == 0) group_end<NG>(s1, s2, s3, lds32(coef_addr + (c / CPG) * 64), lds32(coef_addr + (c / CPG) * 64 + 32), rec);
+                    }
+#pragma unroll
+                    for (int cg = 0; cg < NG; ++cg) {
+                        const float sv = lds_f32(xs_tok[cg] + kbi * (16 * NG));   // undo the activation scale of this k-block
+                        acc[cg][0] = fmaf(sv, rec[cg][0], acc[cg][0]);
+                        acc[cg][1] = fmaf(sv, rec[cg][1], acc[cg][1]);
+                    }
+                    __syncwarp();
+                    if (lane == 0) arrive_a(empty_addr + slot * 8);
+                    if (++slot == p.n_stages) { slot = 0; phase ^= 1; }
+                }
+                if (!alive) break;
+            } else if (in_tail) {
+                // ---- the last stage of the range: chunks cb..ce-1 of one record ----
+                if (!tail_open) {
+                    if (!wait_bar(&full_bar[slot], phase, &abort_flag, spin)) { alive = false; break; }
+                    tail_open = true;
+                }
+                const unsigned rloc = u >> 2, cb = u & 3u, ce = min(4u, cb + (u1 - u));
+                const uint32_t unit = order_after_wait(ring_addr + slot * stage_bytes + rloc * unit_bytes + lane * 16);
+                const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
+                int s1[NG][4], s2[NG][4], s3[NG][4];
+                float rec[NG][2];
+#pragma unroll
+                for (int cg = 0; cg < NG; ++cg) {
+                    rec[cg][0] = rec[cg][1] = 0.f;
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) s1[cg][r] = s2[cg][r] = s3[cg][r] = 0;
+                }
+                for (unsigned c = cb; c < ce; ++c) {
+                    uint32_t pa0, pb0, qa0, qb0, fa0, fb0, pa1, pb1, qa1, qb1, fa1, fb1;
+                    decode_word<WB>(lds32(unit + c * 4), lut_lane, pa0, pb0, qa0, qb0, fa0, fb0);
+                    decode_word<WB>(lds32(unit + 512 + c * 4), lut_lane, pa1, pb1, qa1, qb1, fa1, fb1);
+#pragma unroll
+                    for (int cg = 0; cg < NG; ++cg) {
+                        const uint2 xf = lds64(xrow[cg] + (uint32_t)kbi * kBlockK + c * 32);
+                        mma_s8(s1[cg], pa0, pa1, pb0, pb1, xf.x, xf.y);
+                        mma_s8(s2[cg], qa0, qa1, qb0, qb1, xf.x, xf.y);
+                        mma_s8(s3[cg], fa0, fa1, fb0, fb1, xf.x, xf.y);
+                    }
+                    if (((c + 1) % CPG) == 0 || c + 1 == ce)   // end of a macro-block, or of this warp's share of it (the sums are linear)
+                        group_end<NG>(s1, s2, s3, lds32(coef_addr + (c / CPG) * 64), lds32(coef_addr + (c / CPG) * 64 + 32), rec);
+                }
+#pragma unroll
+                for (int cg = 0; cg < NG; ++cg) {
+                    const float sv = lds_f32(xs_tok[cg] + kbi * (16 * NG));
+                    acc[cg][0] = fmaf(sv, rec[cg][0], acc[cg][0]);
+                    acc[cg][1] = fmaf(sv, rec[cg][1], acc[cg][1]);
+                }
+                u += ce - cb;
+            } else {
+                break;   // every part has been handed over
+            }
+        }
+        if (!alive) break;
+        if (n_tail) {   // every warp takes part in the tail stage's hand-shake, with or without chunks of its own
+            if (!tail_open && !wait_bar(&full_bar[slot], phase, &abort_flag, spin)) { alive = false; break; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[slot]);
+            if (++slot == p.n_stages) { slot = 0; phase ^= 1; }
+        }
+        seq += (unsigned)wk.P;
+    }
+    if (lane == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
+}
+
+}  // namespace chain
+}  // namespace goq
+
+// ---- host side -------------------------------------------------------------------------------------
+namespace goq {
+
+static int chain_sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 148;
+    return n > 0 ? n : 148;
+}
+
+static constexpr size_t kChainSmemMax = 226 * 1024;   // the opt-in limit is 227 KiB per CTA, static shared variables included
+
+static size_t chain_fixed_smem(int ng) {
+    return 8192 /* alignment slack */ + (size_t)kLutBytes + (size_t)chain::kTileSlots * chain::kNW * ng * 64 * sizeof(float) +
+           (size_t)2 * chain::kMaxKBlocks * 4 * ng * sizeof(float) + (size_t)(2 * chain::kMaxStages + 4 + chain::kTileSlots) * sizeof(uint64_t);
+}
+static size_t chain_xbuf_bytes(int m, int k_pad) { return ((size_t)2 * m * (k_pad + chain::kXPad) + 127) & ~(size_t)127; }
+
+bool gemv_seq_supported(const Geometry& g, int m) {
+    if (!(g.group >= 32 && g.wbits <= 3 && m >= 1 && m <= 8 && g.k_blocks <= chain::kMaxKBlocks)) return false;
+    if ((unsigned long long)g.n_units * (unsigned)g.k_blocks >= (1ull << 32)) return false;   // record -> tile by multiply and shift
+    // at least two ring stages beside one activation buffer
+    return chain_fixed_smem(m <= 4 ? 1 : 2) + chain_xbuf_bytes(m, g.k_pad) + (size_t)2 * chain::kStageRecs * g.unit_bytes <= kChainSmemMax;
+}
+// Scratch: [status word and, in its second word, the launch count, 256 B][done: n ints - zero on entry, left zero] then the
+// posted partial sums, placed behind the counter area every kernel of the library keeps zero, so that a buffer laid out
+// for goq_gemv can serve a one-linear chain. The whole buffer starts zero-filled (goq_workspace_init): a posted value is
+// valid when it carries the current launch's tag, and zero is never a tag.
+size_t gemv_seq_zeroed_prefix(int n_items) {
+    const size_t n = (size_t)(n_items > 0 ? n_items : 0);
+    const size_t z = kWsStatusBytes + align_up(n * sizeof(int), 256);
+    return z > kWsScratchOff ? z : kWsScratchOff;
+}
+size_t gemv_seq_workspace(int n_items) {
+    const size_t n = (size_t)(n_items > 0 ? n_items : 0), G = (size_t)chain_sm_count();
+    return gemv_seq_zeroed_prefix(n_items) + n * G * 2 * chain::kPartWords * sizeof(uint2);
+}
+
+template <int WB, int CPG, int NG>
+static cudaError_t launch_chain_cfg(chain::Params& p, size_t x_need, cudaStream_t st) {
+    auto kernel = chain::gemv_chain_kernel<WB, CPG, NG>;
+    const size_t stage_bytes = (size_t)chain::kStageRecs * p.unit_bytes;
+    const size_t fixed = chain_fixed_smem(NG);
+    // two activation buffers when they leave room for four ring stages, else one
+    p.x_double = (fixed + 2 * x_need + 4 * stage_bytes <= kChainSmemMax) ? 1 : 0;
+    p.xbuf_bytes = (int)x_need;
+    const size_t xtotal = (size_t)(p.x_double ? 2 : 1) * x_need;
+    if (fixed + xtotal + 2 * stage_bytes > kChainSmemMax) return cudaErrorInvalidConfiguration;
+    int n_stages = (int)((kChainSmemMax - fixed - xtotal) / stage_bytes);
+    if (n_stages > chain::kMaxStages) n_stages = chain::kMaxStages;
+    p.n_stages = n_stages;
+    const size_t smem = fixed + xtotal + (size_t)n_stages * stage_bytes;
+    static SmemAttrCache smem_attr;
+    if (cudaError_t e = ensure_dynamic_smem(kernel, smem, smem_attr)) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(chain_sm_count());   // every CTA must be resident: the completion counters are waited on
+    cfg.blockDim = dim3(chain::kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
+cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, int unit_bytes, void* ws, int spin_limit, cudaStream_t st) {
+    static thread_local chain::Params p;   // ~17 KB: kept off the stack
+    auto* wsb = (uint8_t*)ws;
+    p.n_items = n;
+    p.unit_bytes = unit_bytes;
+    p.spin_limit = spin_limit > 0 ? spin_limit : kSpinLimit;
+    p.status = (int*)wsb;
+    p.done = (int*)(wsb + 256);
+    p.epoch = (unsigned*)(wsb + 4);
+    p.parts = (uint2*)(wsb + gemv_seq_zeroed_prefix(n));
+    int m_max = 1;
+    size_t x_need = 0;
+    for (int i = 0; i < n; ++i) {
+        chain::Item& it = p.item[i];
+        const Geometry& g = calls[i].g;
+        it.packed = (const uint8_t*)calls[i].packed;
+        it.x = (const uint16_t*)calls[i].x;
+        it.y = calls[i].y;
+        it.kb_magic = ((1ull << 32) + (unsigned)g.k_blocks - 1) / (unsigned)g.k_blocks;
+        it.units = (unsigned)g.n_units;
+        it.n_tiles = g.n_tiles;
+        it.k_blocks = g.k_blocks;
+        it.k_in = g.k_in;
+        it.n_out = g.n_out;
+        it.m = calls[i].m;
+        it.y_dtype = calls[i].y_dtype;
+        it.depends = calls[i].depends;
+        if (calls[i].m > m_max) m_max = calls[i].m;
+        const size_t b = chain_xbuf_bytes(calls[i].m, g.k_pad);
+        if (b > x_need) x_need = b;
+    }
+    const int cpg = group / 32;
+    if (m_max <= 4) {
+        if (wbits == 3) return cpg == 1 ? launch_chain_cfg<3, 1, 1>(p, x_need, st) : cpg == 2 ? launch_chain_cfg<3, 2, 1>(p, x_need, st) : launch_chain_cfg<3, 4, 1>(p, x_need, st);
+        return cpg == 1 ? launch_chain_cfg<2, 1, 1>(p, x_need, st) : cpg == 2 ? launch_chain_cfg<2, 2, 1>(p, x_need, st) : launch_chain_cfg<2, 4, 1>(p, x_need, st);
+    }
+    if (wbits == 3) return cpg == 1 ? launch_chain_cfg<3, 1, 2>(p, x_need, st) : cpg == 2 ? launch_chain_cfg<3, 2, 2>(p, x_need, st) : launch_chain_cfg<3, 4, 2>(p, x_need, st);
+    return cpg == 1 ? launch_chain_cfg<2, 1, 2>(p, x_need, st) : cpg == 2 ? launch_chain_cfg<2, 2, 2>(p, x_need, st) : launch_chain_cfg<2, 4, 2>(p, x_need, st);
+}
+
+}  // namespace goq

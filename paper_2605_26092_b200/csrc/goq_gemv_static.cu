@@ -32,7 +32,8 @@ goq_status static_scratch_address(void** out) {
     std::lock_guard<std::mutex> lock(g_scratch_mutex);
     if (!g_scratch_addr[dev]) {
         void* ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return GOQ_ERR_CUDA;
+        if (cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch)) return goq::status_from_cuda(e);
+        if (!ptr) return GOQ_ERR_CUDA;
         g_scratch_addr[dev] = ptr;
     }
     *out = g_scratch_addr[dev];
@@ -55,9 +56,8 @@ extern "C" goq_status goq_gemv_static(const goq_desc* desc, const void* packed, 
     const size_t need = goq::gemv_stream_workspace(g);
     if (need > kStaticScratchBytes) return GOQ_ERR_WORKSPACE;  // layer has too many 16-row tiles for the fixed array
     int major = 0, dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
-        return GOQ_ERR_CUDA;
+    if (cudaError_t e = cudaGetDevice(&dev)) return goq::status_from_cuda(e);
+    if (cudaError_t e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) return goq::status_from_cuda(e);
     if (major != 10) return GOQ_ERR_ARCH;
     void* scratch = nullptr;
     if (goq_status s = static_scratch_address(&scratch)) return s;
@@ -65,8 +65,18 @@ extern "C" goq_status goq_gemv_static(const goq_desc* desc, const void* packed, 
     // The array keeps whatever the previous call left. The status word and the tile counters must start
     // at zero, so clear exactly that prefix; the parked partial sums behind it are always written before
     // they are read.
-    if (cudaMemsetAsync(scratch, 0, goq::gemv_stream_zeroed_prefix(g), st) != cudaSuccess)
-        return GOQ_ERR_CUDA;
-    return goq::launch_gemv_stream(g, packed, x_bf16, batch, y, y_dtype, scratch, st) == cudaSuccess ? GOQ_OK
-                                                                                                     : GOQ_ERR_CUDA;
+    if (cudaError_t e = cudaMemsetAsync(scratch, 0, goq::gemv_stream_zeroed_prefix(g), st)) return goq::status_from_cuda(e);
+    return goq::status_from_cuda(goq::launch_gemv_stream(g, packed, x_bf16, batch, y, y_dtype, scratch, st));
+}
+
+extern "C" goq_status goq_gemv_static_status(void* stream, int* status_out) {
+    if (!status_out) return GOQ_ERR_INVALID_ARG;
+    void* scratch = nullptr;
+    if (goq_status s = static_scratch_address(&scratch)) return s;
+    int v = 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaError_t e = cudaMemcpyAsync(&v, scratch, sizeof(int), cudaMemcpyDeviceToHost, st)) return goq::status_from_cuda(e);
+    if (cudaError_t e = cudaStreamSynchronize(st)) return goq::status_from_cuda(e);
+    *status_out = v;
+    return GOQ_OK;
 }

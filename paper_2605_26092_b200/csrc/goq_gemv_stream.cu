@@ -68,17 +68,6 @@ __device__ __forceinline__ int range_begin(int i, int n_units, int n_ctas) {
     return (int)((long long)n_units * i / n_ctas);
 }
 
-#ifdef GOQ_TRACE
-__device__ unsigned long long g_trace[512][17][12];
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%clock64;" : "=l"(t)); return t; }
-#define GOQ_TR(slot) do { if ((threadIdx.x & 31) == 0) g_trace[blockIdx.x][threadIdx.x >> 5][slot] = gtime(); } while (0)
-__device__ unsigned long long g_wall[2][512][4];
-__device__ __forceinline__ unsigned long long wtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define GOQ_WALL(slot) do { if (threadIdx.x == 0) g_wall[(p.m_total - 1) & 1][blockIdx.x][slot] = wtime(); } while (0)
-#else
-#define GOQ_TR(slot) do { } while (0)
-#define GOQ_WALL(slot) do { } while (0)
-#endif
 constexpr int kRedSlots = 2;  // ring of per-tile reduction buffers inside a CTA
 
 // WB: weight bits (2, 3); NT: 8-token column tiles (1, 2); CPG: 32-wide chunks per macro-block (1, 2, 4)
@@ -101,8 +90,6 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
     __shared__ int arrive_cnt[kRedSlots];  // warps that have parked their sums for the tile using the slot
     __shared__ int done_gen[kRedSlots];    // 1 + local index of the last tile fully reduced out of the slot
 
-    GOQ_TR(0);
-    GOQ_WALL(0);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_ctas = gridDim.x;
     const int u_begin = range_begin(blockIdx.x, p.n_units, n_ctas), u_end = range_begin(blockIdx.x + 1, p.n_units, n_ctas);
@@ -120,7 +107,6 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    GOQ_TR(1);
     // the next kernel in the stream may begin its own prologue and weight prefetch
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
@@ -141,7 +127,6 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
                 mbar_arrive_expect_tx(&full_bar[slot], bytes);
                 bulk_copy_g2s(ring + (size_t)slot * stage_bytes, src + (size_t)s * stage_bytes, bytes, &full_bar[slot]);
                 if (++slot == p.n_stages) { slot = 0; ++round; }
-                if (s == 0) GOQ_TR(2);
                 if (!x_issued && (s + 1 == my_stages || s + 1 == p.n_stages)) {
                     // the ring is primed: now the activations, which the preceding kernel may have produced
                     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -153,7 +138,6 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
                     x_issued = true;
                 }
             }
-            GOQ_TR(3);
             if (abort_flag) drain_issued_stages(full_bar, issued, p.n_stages);
         }
         return;
@@ -171,7 +155,6 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
         for (int i = tid; i < tail * p.m_total; i += kConsumerWarps * 32) xw[(size_t)(i / tail) * kp + p.k_in + (i % tail)] = 0;
     }
     consumer_bar_sync();
-    GOQ_TR(2);
 
     const int g = lane >> 2, t = lane & 3;
     const uint32_t lut_lane = smem_u32(lut) + (lane & (kLutCopies - 1)) * 16;
@@ -180,9 +163,6 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
 
     // everything below reads activations or writes outputs / scratch: wait for the preceding kernel
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    GOQ_TR(3);
-    GOQ_WALL(1);
-    int tr_n = 0;
 
     // per-lane activation row (token nt*8+g). Lanes whose token does not exist read the last token's
     // row instead of zeros: an MMA output column depends only on its own B column, and columns of
@@ -248,7 +228,7 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
 #pragma unroll
                         for (int q = 0; q < NT * 4; ++q) out[q] = 0.f;
                         for (int w = 0; w < kConsumerWarps; ++w) {
-                            // warp w holds a record of the segment iff some i in [a, b) has i % 8 == w
+                            // warp w holds a record of the segment iff some i in [a, b) has i % 16 == w
                             const int first = a + ((w - a) & (kStageUnits - 1));
                             if (first < b) {
 #pragma unroll
@@ -316,7 +296,6 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
         }
 
         if (mbar_wait_bounded(&full_bar[slot], phase, &abort_flag)) {
-            if (tr_n < 3) GOQ_TR(4 + 2 * tr_n);
             const uint32_t unit = order_after_wait(smem_u32(ring) + slot * stage_bytes + warp * p.unit_bytes + lane * 16);
             const int kb0 = (u - tile_u0) * kBlockK;
             const uint4 wv0 = lds128(unit), wv1 = lds128(unit + 512);
@@ -371,13 +350,9 @@ __global__ void __launch_bounds__(kStreamThreads, (NT == 1) ? 2 : 1) gemv_stream
             }
         }
         __syncwarp();
-        if (tr_n < 3) GOQ_TR(5 + 2 * tr_n);
-        ++tr_n;
         if (lane == 0) mbar_arrive(&empty_bar[slot]);
         if (++slot == p.n_stages) { slot = 0; phase ^= 1; }
     }
-    GOQ_TR(10);
-    GOQ_WALL(2);
     if (lane == 0 && abort_flag) atomicExch(p.status, (int)GOQ_ERR_TIMEOUT);
 }
 

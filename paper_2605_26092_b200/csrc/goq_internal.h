@@ -5,6 +5,9 @@
 
 namespace goq {
 
+// GOQ_OK, or GOQ_ERR_CUDA after remembering the error for goq_last_cuda_error and clearing a non-sticky one.
+goq_status status_from_cuda(cudaError_t e);
+
 // The dynamic shared memory limit of a kernel is a per-device attribute: remember, per device, the largest size it
 // has been raised to (one cache object per kernel instantiation, a function-local static at the call site).
 struct SmemAttrCache { size_t set[64] = {}; };
@@ -42,16 +45,10 @@ bool stream_hash_is_bijective();
 cudaError_t launch_gemv_stream(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y, int y_dtype,
                                void* ws, cudaStream_t st);
 
-// Decode GEMV on tcgen05 with the FP8 weight operand in tensor memory (group 64 or 128, wbits <= 3, m <= 16).
-// `ws` holds gemv_tc_workspace(g) bytes, zero on entry (goq_workspace_init), counters left zero on return.
-bool gemv_tc_supported(const Geometry& g, int m);
-size_t gemv_tc_workspace(const Geometry& g);
-cudaError_t launch_gemv_tc(const Geometry& g, const void* packed, const void* x_bf16, int m, void* y, int y_dtype,
-                           void* ws, cudaStream_t st);
-
-// A sequence of decode GEMVs in one persistent cooperative kernel (group >= 32, wbits <= 3, batch <= 8, the staged
+// A chain of decode GEMVs in one persistent cooperative kernel (group >= 32, wbits <= 3, batch <= 8, the staged
 // activations of each linear fit in shared memory; every linear has the same wbits and group). `ws` holds
-// gemv_seq_workspace(n) bytes, zero on entry, left zero on return.
+// gemv_seq_workspace(n) bytes whose first gemv_seq_zeroed_prefix(n) bytes are zero on entry and left zero on return.
+// spin_limit > 0 replaces the bound of every device-side wait (tests make waits run out with it).
 constexpr int kSeqMaxItems = 256;
 struct SeqCall {
     Geometry g;
@@ -60,10 +57,11 @@ struct SeqCall {
     void* y;
     int m, y_dtype, depends;
 };
-extern bool g_seq_int8;   // false: never use the integer-operand form (tests)
 bool gemv_seq_supported(const Geometry& g, int m);
 size_t gemv_seq_workspace(int n_items);
-cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, int unit_bytes, void* ws, cudaStream_t st);
+size_t gemv_seq_zeroed_prefix(int n_items);
+cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, int unit_bytes, void* ws, int spin_limit,
+                            cudaStream_t st);
 
 // Prefill GEMM on tcgen05 tensor cores (wbits <= 3). `ws` holds gemm_tc_workspace(g, m) bytes: status word and
 // (split-K) tile counters in the common areas, then the per-token scales, the fp16 copy of the m x k_in activations

@@ -23,7 +23,7 @@ EXPORTS = (
     "goq_status_string", "goq_packed_bytes", "goq_algorithmic_bytes", "goq_workspace_bytes", "goq_pack",
     "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant", "goq_workspace_init",
     "goq_workspace_status", "goq_gemv_static", "goq_last_cuda_error", "goq_sequence_workspace_bytes",
-    "goq_gemv_sequence", "goq_gemv_sequence_host",
+    "goq_gemv_sequence", "goq_gemv_sequence_host", "goq_set_wait_limit", "goq_gemv_static_status",
 )
 
 
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.goq_workspace_status.argtypes = [c_void_p, c_void_p, POINTER(c_int)]
         L.goq_gemv_static.restype = c_int
         L.goq_gemv_static.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p]
+        L.goq_gemv_static_status.restype = c_int
+        L.goq_gemv_static_status.argtypes = [c_void_p, POINTER(c_int)]
         L.goq_last_cuda_error.restype = c_int
         L.goq_last_cuda_error.argtypes = []
         L.goq_sequence_workspace_bytes.restype = ctypes.c_size_t
@@ -89,6 +91,8 @@ def lib() -> ctypes.CDLL:
                                              c_void_p, ctypes.c_size_t, c_void_p, ctypes.c_size_t, c_void_p]
         L.goq_set_gemv_variant.restype = c_int
         L.goq_set_gemv_variant.argtypes = [c_int]
+        L.goq_set_wait_limit.restype = c_int
+        L.goq_set_wait_limit.argtypes = [c_int]
         _lib = L
     return _lib
 
@@ -154,6 +158,11 @@ def set_gemv_variant(variant: int) -> int:
     return lib().goq_set_gemv_variant(variant)
 
 
+def set_wait_limit(polls: int) -> int:
+    """goq_set_wait_limit: bound of the device-side waits of goq_gemv_sequence (tests only; 0 = the kernel's own)."""
+    return lib().goq_set_wait_limit(polls)
+
+
 def pack(d: Desc, codes, meta, coef_f16, packed, stream=None):
     _check(lib().goq_pack(ctypes.byref(d), _ptr(codes), _ptr(meta), _ptr(coef_f16), _ptr(packed),
                           packed.numel() * packed.element_size(), _stream(stream)), "goq_pack")
@@ -175,6 +184,13 @@ def gemv_static(d: Desc, packed, x_bf16, batch: int, y, y_dtype: int, stream=Non
     For callers that cannot allocate device memory; calls that may overlap on the GPU must not share it."""
     _check(lib().goq_gemv_static(ctypes.byref(d), _ptr(packed), _ptr(x_bf16), batch, _ptr(y), y_dtype,
                                  _stream(stream)), "goq_gemv_static")
+
+
+def gemv_static_status(stream=None) -> int:
+    """goq_gemv_static_status: status word of the library's built-in scratch array (synchronises the stream)."""
+    out = c_int(0)
+    _check(lib().goq_gemv_static_status(_stream(stream), ctypes.byref(out)), "goq_gemv_static_status")
+    return out.value
 
 
 def sequence_workspace_bytes(n_items: int) -> int:

@@ -33,11 +33,11 @@ def _ws(goq, n_items):
     return ws
 
 
-@pytest.fixture(params=[0, 5], ids=["auto", "bf16-operands"])
-def form(goq, request):
-    """0: the kernel picks integer operands when every item has batch <= 4; 5: always bf16 operands."""
-    prev = goq.set_gemv_variant(request.param)
-    yield request.param
+@pytest.fixture
+def form(goq):
+    """Automatic kernel choice (the chain kernel has one arithmetic form: integer operands)."""
+    prev = goq.set_gemv_variant(0)
+    yield 0
     goq.set_gemv_variant(prev)
 
 
@@ -64,8 +64,11 @@ def test_chain_with_real_dependencies_matches_oracle_stage_by_stage(goq, form):
         for i, L in enumerate(layers):
             y_ref = O.linear_f64(L["codes"], L["meta"], L["coef"], si.bf16_bits_to_f64(x_bits), L["g"], L["b"])
             got = outs[i].float().cpu().numpy().astype(np.float64)
-            tol = TIGHT if i == 2 else 4e-3   # bf16 outputs carry one extra rounding
-            assert O.normwise_rel_err(got, y_ref) <= tol, (i, O.normwise_rel_err(got, y_ref))
+            if i == 2:
+                assert O.normwise_rel_err(got, y_ref) <= TIGHT, (i, O.normwise_rel_err(got, y_ref))
+            else:   # bf16 outputs carry one extra rounding: held to it element by element
+                from tests.gpu_util import check_bf16_output
+                check_bf16_output(got, y_ref, 1e-4, "stage %d" % i)
             if i < 2:
                 x_bits = outs[i].view(torch.int16).cpu().numpy().view(np.uint16)
 
@@ -91,8 +94,8 @@ def test_independent_items_of_mixed_shapes(goq, g, b, form):
     first = [y.clone() for y in ys]
     for L, xb, y in zip(layers, xs, ys):
         y_ref = O.linear_f64(L["codes"], L["meta"], L["coef"], si.bf16_bits_to_f64(xb), g, b)
-        err = O.normwise_rel_err(y.cpu().numpy().astype(np.float64), y_ref)
-        assert err <= TIGHT, err
+        from tests.gpu_util import check_parity
+        check_parity(y.cpu().numpy(), y_ref, TIGHT, 1e-4)
     goq.gemv_sequence(seq, ws)
     torch.cuda.synchronize()
     for a, y in zip(first, ys):
@@ -178,7 +181,8 @@ def test_one_7b_shaped_layer_sampled_rows(goq, form):
     assert goq.workspace_status(ws) == goq.OK
     for codes, meta, coef, xb, rows, y in checks:
         y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 128, 3, rows=rows)
-        assert O.normwise_rel_err(y.cpu().numpy().astype(np.float64)[:, rows], y_ref) <= TIGHT
+        from tests.gpu_util import check_parity
+        check_parity(y.cpu().numpy().astype(np.float64)[:, rows], y_ref, TIGHT, 1e-4)
 
 
 def test_unsupported_and_invalid_sequences_return_a_status(goq):
@@ -203,6 +207,35 @@ def test_unsupported_and_invalid_sequences_return_a_status(goq):
     assert e.value.status == goq.ERR_WORKSPACE
 
 
+def test_a_wait_that_runs_out_reports_timeout_and_the_context_stays_usable(goq):
+    """goq_set_wait_limit(1) bounds every device-side wait of the chain kernel to a single probe. In a dependent chain
+    the first CTA to finish the first linear probes the completion counter before the other CTAs have reported, finds
+    it short and gives up: the launch still ends by itself, the status word reads GOQ_ERR_TIMEOUT, nothing faults.
+    After the scratch buffer is zero-filled again the same chain runs correctly."""
+    from tests.gpu_util import dev
+    La, Lb = _layer(goq, 2048, 2048, 128, 3, seed=601), _layer(goq, 512, 2048, 128, 3, seed=602)
+    xa = si.bf16_activations(1, 2048, seed=31)
+    mid = torch.zeros((1, 2048), dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros((1, 512), dtype=torch.float32, device="cuda")
+    xd = dev(xa)
+    seq = goq.make_sequence([(La["d"], La["packed"], xd, 1, mid, goq.BF16, False), (Lb["d"], Lb["packed"], mid, 1, y, goq.F32, True)])
+    ws = _ws(goq, 2)
+    prev = goq.set_wait_limit(1)
+    try:
+        goq.gemv_sequence(seq, ws)
+        torch.cuda.synchronize()
+        assert goq.workspace_status(ws) == goq.ERR_TIMEOUT
+    finally:
+        goq.set_wait_limit(prev)
+    goq.workspace_init(ws)
+    goq.gemv_sequence(seq, ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    mid_bits = mid.view(torch.int16).cpu().numpy().view(np.uint16)
+    ref = O.linear_f64(Lb["codes"], Lb["meta"], Lb["coef"], si.bf16_bits_to_f64(mid_bits), 128, 3)
+    assert O.normwise_rel_err(y.cpu().numpy().astype(np.float64), ref) <= TIGHT
+
+
 def test_host_block_entry_point(goq):
     """goq_gemv_sequence_host: activations in one pinned host block, outputs in another; a two-linear chain whose
     second item reads the first one's bf16 output inside the output block."""
@@ -224,7 +257,8 @@ def test_host_block_entry_point(goq):
     assert goq.workspace_status(ws) == goq.OK
     mid_bits = y_host[:y0_bytes].numpy().view(np.uint16).reshape(m, n0)
     y0_ref = O.linear_f64(L0["codes"], L0["meta"], L0["coef"], si.bf16_bits_to_f64(xb), 64, 3)
-    assert O.normwise_rel_err(si.bf16_bits_to_f64(mid_bits), y0_ref) <= 4e-3
+    from tests.gpu_util import check_bf16_output
+    check_bf16_output(si.bf16_bits_to_f64(mid_bits), y0_ref, 1e-4)
     y1 = y_host[y0_bytes:].numpy().view(np.float32).reshape(m, n1).astype(np.float64)
     y1_ref = O.linear_f64(L1["codes"], L1["meta"], L1["coef"], si.bf16_bits_to_f64(mid_bits), 64, 3)
     assert O.normwise_rel_err(y1, y1_ref) <= TIGHT

@@ -59,6 +59,15 @@ def test_static_scratch_entry_matches_regular_entry_on_two_calls_in_a_row(goq):
         goq.gemv(d, packed, x, batch, y_regular, goq.F32, ws=ws)
         goq.gemv_static(d, packed, x, batch, y_static, goq.F32)
         torch.cuda.synchronize()
+        if call == 1:
+            # a warmed call allocates nothing: neither through torch nor behind its back (free device memory as the
+            # driver reports it is unchanged across the call)
+            torch_before, (free_before, _) = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()
+            goq.gemv_static(d, packed, x, batch, y_static, goq.F32)
+            torch.cuda.synchronize()
+            assert torch.cuda.memory_allocated() == torch_before
+            assert torch.cuda.mem_get_info()[0] == free_before
+        assert goq.gemv_static_status() == goq.OK   # the built-in array's status word: no wait gave up
         a = y_regular.cpu().numpy().astype(np.float64)
         b = y_static.cpu().numpy().astype(np.float64)
         assert np.all(np.isfinite(b))
@@ -83,7 +92,7 @@ def test_static_scratch_entry_rejects_what_it_cannot_serve(goq):
     # more 16-row tiles than the scratch buffer's counter area holds: the streaming kernel does not take the layer
     # (goq_gemv serves it with a scratch-free kernel), refused here before anything is launched
     huge = goq.desc(8_000_000, 128, 128, 3)
-    assert goq.workspace_bytes(huge, goq.OP_GEMV, 1) == 0
+    assert goq.workspace_bytes(huge, goq.OP_GEMV, 16) == 0
     assert status(huge) == goq.ERR_UNSUPPORTED
     # configurations the scratch-free kernels of goq_gemv serve
     assert status(goq.desc(16, 128, 16, 3)) == goq.ERR_UNSUPPORTED
