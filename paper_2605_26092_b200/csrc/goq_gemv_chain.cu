@@ -184,7 +184,7 @@ struct FlushCtx {
 };
 struct Sums4 { float v[4]; };   // by value: the accumulators never have their address taken, so they stay in registers
 template <int NG>
-__device__ __noinline__ bool flush_part(const FlushCtx& c, unsigned sq, Sums4 sums) {
+__device__ __forceinline__ bool flush_part(const FlushCtx& c, unsigned sq, Sums4 sums) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
     const int rs = (int)(sq % kTileSlots);
     if (*c.abort_flag) return false;
@@ -435,7 +435,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
     const uint32_t lut_lane = smem_u32(lut) + (lane & (kLutCopies - 1)) * 16;
     const uint32_t ring_addr = smem_u32(ring), unit_bytes = (uint32_t)p.unit_bytes;
     const uint32_t full_addr = smem_u32(full_bar), empty_addr = smem_u32(empty_bar);
-    int slot = 0, phase = 0;          // position in the stage ring
+    int slot = 0, phase = 0;          // position in the stage ring ...
+    uint32_t stage_off = 0, bar_off = 0;   // ... and the same as byte offsets of the stage and of its barriers
+    const uint32_t unit0 = ring_addr + (uint32_t)warp * unit_bytes + (uint32_t)lane * 16;
     uint32_t dep_phase = 0, x_phase = 0, free_phase = 0;
     int x_sel = 0;                    // activation buffer of the current linear
     unsigned seq = 0;                 // tile parts this CTA has opened so far (same in every warp): indexes the reduction slots
@@ -550,9 +552,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 run = min(run, n_full - st);
                 st += run;
                 // ================= the hot loop: one record per iteration =================
-                for (; run; --run, kbi += kStageRecs) {
-                    if (!try_wait_a(full_addr + slot * 8, phase) && !wait_slow_a(full_addr + slot * 8, phase, &abort_flag, spin)) { alive = false; break; }
-                    const uint32_t unit = order_after_wait(ring_addr + slot * stage_bytes + warp * unit_bytes + lane * 16);
+                uint32_t koff = (uint32_t)kbi * kBlockK, ksc = (uint32_t)kbi * (16 * NG);
+                kbi += (int)run * kStageRecs;
+                for (; run; --run, koff += kStageRecs * kBlockK, ksc += kStageRecs * 16 * NG) {
+                    if (!try_wait_a(full_addr + bar_off, phase) && !wait_slow_a(full_addr + bar_off, phase, &abort_flag, spin)) {
+                        alive = false;   // give up after this iteration (whatever it computes is never stored)
+                        run = 1;
+                    }
+                    const uint32_t unit = order_after_wait(unit0 + stage_off);
                     const uint4 wv0 = lds128(unit), wv1 = lds128(unit + 512);
                     const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
                     const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
@@ -564,7 +571,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
 #pragma unroll
                         for (int r = 0; r < 4; ++r) s1[cg][r] = s2[cg][r] = s3[cg][r] = 0;
                     }
-                    const uint32_t koff = (uint32_t)kbi * kBlockK;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint32_t pa0, pb0, qa0, qb0, fa0, fb0, pa1, pb1, qa1, qb1, fa1, fb1;
@@ -581,13 +587,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                     }
 #pragma unroll
                     for (int cg = 0; cg < NG; ++cg) {
-                        const float sv = lds_f32(xs_tok[cg] + kbi * (16 * NG));   // undo the activation scale of this k-block
+                        const float sv = lds_f32(xs_tok[cg] + ksc);   // undo the activation scale of this k-block
                         acc[cg][0] = fmaf(sv, rec[cg][0], acc[cg][0]);
                         acc[cg][1] = fmaf(sv, rec[cg][1], acc[cg][1]);
                     }
                     __syncwarp();
-                    if (lane == 0) arrive_a(empty_addr + slot * 8);
-                    if (++slot == p.n_stages) { slot = 0; phase ^= 1; }
+                    if (lane == 0) arrive_a(empty_addr + bar_off);
+                    stage_off += (uint32_t)stage_bytes; bar_off += 8;
+                    if (++slot == p.n_stages) { slot = 0; phase ^= 1; stage_off = 0; bar_off = 0; }
                 }
                 if (!alive) break;
             } else if (in_tail) {
@@ -637,7 +644,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
             if (!tail_open && !wait_bar(&full_bar[slot], phase, &abort_flag, spin)) { alive = false; break; }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[slot]);
-            if (++slot == p.n_stages) { slot = 0; phase ^= 1; }
+            stage_off += (uint32_t)stage_bytes; bar_off += 8;
+            if (++slot == p.n_stages) { slot = 0; phase ^= 1; stage_off = 0; bar_off = 0; }
         }
         seq += (unsigned)wk.P;
     }
