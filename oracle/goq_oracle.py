@@ -17,6 +17,10 @@ What is here, with the passage each part follows:
   decode_b1 / decode_b2 / reconstruct
                         Section 3.1: w_hat = c1 b1 + c2 b2; Section 3.3 on carrying the PoT
                         magnitude and the sign separately (a flipped zero stays zero; +2^-emax may appear in b2).
+  quantize_k1           Section 3.1, the single-basis form w_hat = c1 b1 (the K = 1 row of the basis-dimension
+                        ablation): b1 as in Section 3.2, c1 the least-squares scale, no second basis.
+  solve_ref             Section 3.4, REF mode (Eq. 3): c* = (A^T A + lambda I)^-1 A^T Y per macro-block with
+                        A = [X_q b1, X_q b2], Y = X_q w, lambda = 1e-4.
   linear_f64            Section 3.5, Eq. 4, float activations: per-group dot products against
                         b1 and b2, coefficients applied to the group sums.
   quantize_activations_int8 / quantize_coefficients_int8 / linear_i32
@@ -229,6 +233,52 @@ def _quantize_rows(w: np.ndarray, group: int, wbits: int):
 
     c = np.stack([c1, c2], axis=-1)
     return (codes.reshape(n, k), meta.reshape(n, k // MICRO), c, a_star.reshape(n, k // MICRO))
+
+
+# ----------------------------------------------------------------------------------------
+# Single-basis form (Section 3.1: w_hat = c1 b1) and REF-mode coefficients (Section 3.4, Eq. 3)
+# ----------------------------------------------------------------------------------------
+def quantize_k1(w: np.ndarray, group: int, wbits: int):
+    """K = 1: b1 = Q(w / ||w||_inf) (Section 3.2) and c1 = <w, b1> / ||b1||^2, the least-squares scale of
+    w_hat = c1 b1 (Section 3.1). Returned in the dual-basis format with an empty second basis:
+    record bytes 0 and c2 = 0, so every consumer of (codes, meta, coef) evaluates c1 b1."""
+    w = np.asarray(w, dtype=np.float64)
+    if not np.all(np.isfinite(w)):
+        raise ValueError("weights must be finite")
+    n, k = w.shape
+    if k % group or group % MICRO:
+        raise ValueError("K must be a multiple of group and group a multiple of 8")
+    wg = w.reshape(n, k // group, group)
+    s_norm = np.max(np.abs(wg), axis=-1, keepdims=True)
+    v = wg / np.where(s_norm == 0.0, 1.0, s_norm)
+    codes = rtn_codes(v, wbits)
+    codes[s_norm[..., 0] == 0.0] = emax_of(wbits)
+    b1 = lattice_values(wbits)[codes]
+    nb1 = np.sum(b1 * b1, axis=-1)
+    c1 = np.where(nb1 == 0.0, 0.0, np.sum(wg * b1, axis=-1) / np.where(nb1 == 0.0, 1.0, nb1))
+    coef = np.stack([c1, np.zeros_like(c1)], axis=-1).astype(np.float16)
+    return codes.reshape(n, k), np.zeros((n, k // MICRO), dtype=np.uint8), coef
+
+
+def solve_ref(w: np.ndarray, codes, meta, x_calib: np.ndarray, group: int, wbits: int, lam: float = 1e-4) -> np.ndarray:
+    """REF mode (Eq. 3). For every row n and macro-block j, with X_q = x_calib[:, j*g:(j+1)*g] (M observations),
+    A = [X_q b1, X_q b2] (M x 2), Y = X_q w:  c* = (A^T A + lam I)^-1 A^T Y.  Returns float64 [N][K/g][2]."""
+    w = np.asarray(w, dtype=np.float64)
+    x = np.asarray(x_calib, dtype=np.float64)
+    n, k = w.shape
+    nj = k // group
+    b1 = decode_b1(codes, wbits)
+    b2 = decode_b2(codes, meta, wbits)
+    out = np.empty((n, nj, 2), dtype=np.float64)
+    for j in range(nj):
+        xq = x[:, j * group:(j + 1) * group]                      # M x g
+        y = xq @ w[:, j * group:(j + 1) * group].T                # M x N : column n is X_q w_n
+        a1 = xq @ b1[:, j * group:(j + 1) * group].T              # M x N : X_q b1
+        a2 = xq @ b2[:, j * group:(j + 1) * group].T
+        for r in range(n):
+            a = np.stack([a1[:, r], a2[:, r]], axis=1)            # M x 2
+            out[r, j] = np.linalg.solve(a.T @ a + lam * np.eye(2), a.T @ y[:, r])
+    return out
 
 
 # ----------------------------------------------------------------------------------------

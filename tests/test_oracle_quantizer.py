@@ -74,6 +74,19 @@ def test_rtn_thresholds_and_ties_3bit():
         assert tie == (lo if abs(lo) < abs(hi) else hi)  # exact tie -> smaller magnitude
 
 
+@pytest.mark.parametrize("b", [2, 4])
+def test_rtn_ties_go_to_the_smaller_magnitude_at_other_widths(b):
+    """The midpoint between any two neighbouring states of the b-bit lattice maps to the one of smaller magnitude,
+    and a hair to either side maps to that side (the 3-bit case is spelt out threshold by threshold above)."""
+    vals = np.sort(O.lattice_values(b))
+    for lo, hi in zip(vals[:-1], vals[1:]):
+        mid = 0.5 * (lo + hi)   # dyadic: exact in float64
+        got = O.lattice_values(b)[O.rtn_codes(np.array([mid]), b)[0]]
+        assert got == (lo if abs(lo) < abs(hi) else hi)
+        assert O.lattice_values(b)[O.rtn_codes(np.array([mid - 1e-9]), b)[0]] == lo
+        assert O.lattice_values(b)[O.rtn_codes(np.array([mid + 1e-9]), b)[0]] == hi
+
+
 def test_largest_element_maps_to_unit():
     w = si.gaussian_weights(16, 256, seed=5)
     codes, _, _ = O.quantize_geo(w, 64, 3)
@@ -143,16 +156,17 @@ def test_residual_orthogonal_to_b1():
     assert np.all(dots <= bound)
 
 
-def test_alignment_is_optimal_over_all_64_candidates():
+@pytest.mark.parametrize("wb", [2, 3, 4])
+def test_alignment_is_optimal_over_all_64_candidates(wb):
     """Per micro-block exhaustive search over (s, eta) gives the same best alignment."""
     w = si.gaussian_weights(4, 128, seed=13)
-    codes, meta, _, aux = O.quantize_geo(w, 64, 3, return_aux=True)
-    b1 = O.decode_b1(codes, 3).reshape(4, 2, 64)
+    codes, meta, _, aux = O.quantize_geo(w, 64, wb, return_aux=True)
+    b1 = O.decode_b1(codes, wb).reshape(4, 2, 64)
     wg = _blocks(w, 64)
     r = wg - aux["c"][..., 0:1] * b1
     x = b1.reshape(4, 2, 8, 8)
     rho = r.reshape(4, 2, 8, 8)
-    b2 = O.decode_b2(codes, meta, 3).reshape(4, 2, 8, 8)
+    b2 = O.decode_b2(codes, meta, wb).reshape(4, 2, 8, 8)
     for idx in np.ndindex(4, 2, 8):
         best = -np.inf
         for s in (1, 2, 3, 4):
@@ -163,16 +177,16 @@ def test_alignment_is_optimal_over_all_64_candidates():
         assert got == pytest.approx(aux["alignment"].reshape(4, 2, 8)[idx], rel=1e-12, abs=1e-15)
 
 
-@pytest.mark.parametrize("g", [8, 16])
-def test_joint_brute_force_over_dual_lattice_on_tiny_groups(g):
+@pytest.mark.parametrize("g,wb", [(8, 3), (16, 3), (8, 2), (8, 4), (16, 2)])
+def test_joint_brute_force_over_dual_lattice_on_tiny_groups(g, wb):
     """Minimum reconstruction error over every (s, eta) assignment of every micro-block,
     with least-squares coefficients, equals what the analytical solver reaches."""
     rng = np.random.default_rng(17)
     for trial in range(6 if g == 8 else 2):
         w = rng.standard_normal((1, g)) * 0.02
-        codes, meta, _, aux = O.quantize_geo(w, g, 3, return_aux=True)
-        b1 = O.decode_b1(codes, 3)[0]
-        b2 = O.decode_b2(codes, meta, 3)[0]
+        codes, meta, _, aux = O.quantize_geo(w, g, wb, return_aux=True)
+        b1 = O.decode_b1(codes, wb)[0]
+        b2 = O.decode_b2(codes, meta, wb)[0]
         c1, c2 = aux["c"][0, 0]
         err = float(np.sum((w[0] - c1 * b1 - c2 * b2) ** 2))
         configs = [(s, eta) for s in (1, 2, 3, 4) for eta in itertools.product((1.0, -1.0), repeat=4)]
@@ -282,3 +296,59 @@ def test_reconstruction_is_the_sum_of_two_signed_pot_terms_exactly():
         # two bases never lose to one
         c1_only = c[..., 0].repeat(64, axis=1) * b1
         assert np.sum((w_hat - w) ** 2) <= np.sum((c1_only - w) ** 2) * (1 + 1e-3)
+
+
+# ---------------------------------------------------------------------------------------------
+# K = 1 (Section 3.1) and REF-mode coefficients (Section 3.4, Eq. 3)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("b", [2, 3, 4])
+def test_k1_is_the_first_basis_of_the_dual_form_and_never_better(b):
+    """Eq. 2 decouples, so the K = 1 scale is the dual form's c1; by Pythagoras the K = 2 error is the K = 1 error
+    minus c2^2 ||b2||^2 (the K = 1 / K = 2 comparison of the basis-dimension ablation, here per block)."""
+    w = si.gaussian_weights(24, 256, seed=70 + b).astype(np.float64)
+    c1k, m1k, cf1 = O.quantize_k1(w, 64, b)
+    c2k, m2k, cf2, aux = O.quantize_geo(w, 64, b, return_aux=True)
+    assert np.array_equal(c1k, c2k) and not m1k.any()
+    assert np.array_equal(cf1[..., 0], cf2[..., 0]) and not cf1[..., 1].any()
+    wg = w.reshape(24, 4, 64)
+    b1 = O.decode_b1(c2k, b).reshape(24, 4, 64)
+    b2 = O.decode_b2(c2k, m2k, b).reshape(24, 4, 64)
+    e1 = np.sum((wg - aux["c"][..., :1] * b1) ** 2, axis=-1)
+    e2 = np.sum((wg - aux["c"][..., :1] * b1 - aux["c"][..., 1:] * b2) ** 2, axis=-1)
+    assert np.all(e2 <= e1 + 1e-15)
+    assert np.allclose(e1 - e2, aux["c"][..., 1] ** 2 * np.sum(b2 * b2, axis=-1), rtol=1e-9, atol=1e-18)
+    # the K = 1 record evaluates to c1 b1 in the reference layer: the second term is multiplied by c2 = 0
+    x = si.bf16_bits_to_f64(si.bf16_activations(3, 256, seed=1))
+    y = O.linear_f64(c1k, m1k, cf1, x, 64, b)
+    ref = x @ (O.coef_to_f64(cf1)[..., :1].repeat(64, axis=1).reshape(24, 256) * O.decode_b1(c1k, b)).T
+    assert np.allclose(y, ref, rtol=1e-12, atol=1e-15)
+
+
+def test_ref_solve_against_library_least_squares_and_its_limits():
+    """Eq. 3 pinned three ways: (1) ridge = ordinary least squares on the augmented system [A; sqrt(lam) I] c = [Y; 0]
+    (library lstsq); (2) with orthonormal calibration rows spanning the block (X_q^T X_q = I) and lam -> 0 the
+    activation-space problem is the weight-space one, so REF returns the GEO coefficients of Eq. 2; (3) the
+    regulariser only shrinks: ||c(lam)|| decreases in lam."""
+    rng = np.random.default_rng(5)
+    n, k, g, b = 6, 128, 64, 3
+    w = si.gaussian_weights(n, k, seed=91).astype(np.float64)
+    codes, meta, coef, aux = O.quantize_geo(w, g, b, return_aux=True)
+    x = rng.standard_normal((40, k))
+    c = O.solve_ref(w, codes, meta, x, g, b, lam=1e-4)
+    b1, b2 = O.decode_b1(codes, b), O.decode_b2(codes, meta, b)
+    for r in range(n):
+        for j in range(k // g):
+            sl = slice(j * g, (j + 1) * g)
+            a = np.stack([x[:, sl] @ b1[r, sl], x[:, sl] @ b2[r, sl]], axis=1)
+            aug = np.vstack([a, np.sqrt(1e-4) * np.eye(2)])
+            rhs = np.concatenate([x[:, sl] @ w[r, sl], np.zeros(2)])
+            ref = np.linalg.lstsq(aug, rhs, rcond=None)[0]
+            assert np.allclose(c[r, j], ref, rtol=1e-9, atol=1e-12)
+    q, _ = np.linalg.qr(rng.standard_normal((g, g)))
+    xo = np.zeros((g, k))
+    xo[:, :g] = q
+    xo[:, g:] = q[::-1]
+    c0 = O.solve_ref(w, codes, meta, xo, g, b, lam=1e-13)
+    assert np.allclose(c0, aux["c"], rtol=1e-8, atol=1e-11)
+    norms = [np.linalg.norm(O.solve_ref(w, codes, meta, x, g, b, lam=l)) for l in (1e-6, 1e-2, 1e2)]
+    assert norms[0] > norms[1] > norms[2]
