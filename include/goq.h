@@ -55,14 +55,18 @@ typedef enum {
 typedef enum { GOQ_BF16 = 0, GOQ_F32 = 1, GOQ_I8 = 2 } goq_dtype;
 typedef enum { GOQ_OP_GEMV = 0, GOQ_OP_GEMM = 1 } goq_op;
 
-#define GOQ_LAYOUT_TILE16 1 /* the only packed layout so far; see goq_pack */
+#define GOQ_LAYOUT_TILE16 1 /* dual-basis weights w_hat = c1 b1 + c2 b2; see goq_pack */
+/* Single-basis weights w_hat = c1 b1 (Section 3.1, the K = 1 row of the basis-dimension ablation) in the same packed
+ * format: goq_pack and goq_quantize_geo store zero records and c2 = 0, so every kernel evaluates c1 b1, and the decode
+ * GEMV skips the second basis altogether (algorithmic bits per weight: wbits + 16/group). */
+#define GOQ_LAYOUT_TILE16_K1 2
 
 typedef struct {
     int32_t n_out;  /* output channels N */
     int32_t k_in;   /* input channels K */
     int32_t group;  /* macro-block size g: multiple of 8 that divides 128, or 128 (8,16,32,64,128) */
     int32_t wbits;  /* 2, 3 or 4 */
-    int32_t layout; /* GOQ_LAYOUT_TILE16 */
+    int32_t layout; /* GOQ_LAYOUT_TILE16 or GOQ_LAYOUT_TILE16_K1 */
 } goq_desc;
 
 /* Text for a status code (static string, never NULL). */
@@ -147,6 +151,41 @@ goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16
 goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int m, int x_dtype,
                     const float* sx, const int8_t* cq, const float* sc, void* y, int y_dtype,
                     int32_t* acc, void* ws, size_t ws_bytes, void* stream);
+
+/* goq_quantize_activations - the activation quantizer of Section 3.5 (X~ and s_x of Eq. 4): per-token symmetric 8-bit
+ * integers, s_x[m] = max_k |x[m,k]| / 127 (1 for an all-zero token), x~ = clamp(rne(x / s_x), +-127), evaluated in
+ * float64 (round half to even).
+ *   x      [m][k] GOQ_F32 or GOQ_BF16        xq  out [m][k] int8        sx  out [m] fp32
+ *   amax   optional [m] fp32: the tokens' largest magnitudes if the caller already has them (goq_gemm_i8_requant records
+ *          them in its epilogue); the kernel then reads x once instead of twice. NULL: computed here. */
+goq_status goq_quantize_activations(const void* x, int x_dtype, int m, int k, const float* amax, int8_t* xq, float* sx,
+                                    void* stream);
+
+/* goq_gemm_i8_requant - the integer layer of goq_gemm (x_dtype GOQ_I8) followed by the "global rescaling or
+ * requantization" of Section 3.5, after Eq. 4: y = sx * 2^-emax * (sc1 ACC_1 + sc2 ACC_2) as fp32, the per-token
+ * largest |y| recorded by the GEMM's epilogue, and - when yq, sy are given - y requantised to the next layer's int8
+ * activations with goq_quantize_activations' arithmetic (one more kernel that reads y once).
+ *   x, sx, cq, sc as in goq_gemm;  y out [m][n_out] fp32;  amax out [m] fp32 (cleared by the call);
+ *   yq out [m][n_out] int8 and sy out [m] fp32, both or neither. */
+goq_status goq_gemm_i8_requant(const goq_desc* desc, const void* packed, const int8_t* x, int m, const float* sx,
+                               const int8_t* cq, const float* sc, float* y, float* amax, int8_t* yq, float* sy, void* stream);
+
+/* goq_quantize_geo - the GEO-mode quantizer on the device (Sections 3.2-3.4): b1 = Q(w / ||w||_inf) on the asymmetric
+ * lattice (nearest state, ties to the smaller magnitude), residual r = w - c1 b1 (Eq. 1), per micro-block
+ * d = x_i r_j - x_j r_i, eta* = sgn d (+1 at 0), A_s = sum |d|, s* = first maximiser (Section 3.3, steps 1-3),
+ * c1 = <w,b1>/||b1||^2, c2 = <w,b2>/||b2||^2 (Eq. 2), rounded to fp16. float64 arithmetic; one warp per macro-block.
+ * With layout GOQ_LAYOUT_TILE16_K1 only b1 and c1 are computed (records 0, c2 = 0).
+ *   w      [n_out][k_in] fp32, 16-byte aligned (finite values)
+ *   codes, meta, coef_f16   out, in goq_pack's input format (codes 4-byte aligned) */
+goq_status goq_quantize_geo(const goq_desc* desc, const float* w, uint8_t* codes, uint8_t* meta, uint16_t* coef_f16,
+                            void* stream);
+
+/* goq_solve_ref - REF-mode coefficients (Section 3.4, Eq. 3): per row and macro-block, with X_q the calibration inputs
+ * restricted to the macro-block's channels, A = [X_q b1, X_q b2], Y = X_q w:  c* = (A^T A + lambda I)^-1 A^T Y.
+ *   w [n_out][k_in] fp32; codes, meta as produced by goq_quantize_geo; x_calib [m][k_in] fp32 (m observations);
+ *   lambda >= 0 (the paper uses 1e-4);  coef_f16 out [n_out][k_in/group][2];  c_f64 optional out, the unrounded pairs. */
+goq_status goq_solve_ref(const goq_desc* desc, const float* w, const uint8_t* codes, const uint8_t* meta,
+                         const float* x_calib, int m, double lambda, uint16_t* coef_f16, double* c_f64, void* stream);
 
 /* goq_gemv_host - goq_gemv for callers whose activations live in host memory (Eq. 4, as goq_gemv).
  *   x_host   HOST [batch][k_in] bf16 (pinned memory makes the copy asynchronous)

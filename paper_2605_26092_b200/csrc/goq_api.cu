@@ -71,6 +71,7 @@ size_t goq_packed_bytes(const goq_desc* desc) {
 size_t goq_algorithmic_bytes(const goq_desc* desc) {
     Geometry g;
     if (!goq::make_geometry(desc, &g)) return 0;
+    if (g.k1) return (size_t)g.n_out * g.k_in * g.wbits / 8 + (size_t)g.n_out * (g.k_in / g.group) * 2;   // codes + one fp16 scale
     // (wbits + 0.75) bits per weight = (4*wbits + 3) / 32 bytes
     return (size_t)g.n_out * g.k_in * (4 * g.wbits + 3) / 32 + (size_t)g.n_out * (g.k_in / g.group) * 4;
 }
@@ -206,10 +207,58 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
         const long long bound = (long long)g.k_in * 127 * 127 * (1ll << ((1 << (g.wbits - 1)) - 1));
         if (bound >= (1ll << 31)) return GOQ_ERR_OVERFLOW_BOUND;
         if (goq_status s = check_arch()) return s;
-        return from_cuda(goq::launch_gemm_a8(g, packed, (const int8_t*)x, m, sx, cq, sc, y, y_dtype, acc,
+        return from_cuda(goq::launch_gemm_a8(g, packed, (const int8_t*)x, m, sx, cq, sc, y, y_dtype, acc, nullptr,
                                              (cudaStream_t)stream));
     }
     return GOQ_ERR_INVALID_ARG;
+}
+
+goq_status goq_gemm_i8_requant(const goq_desc* desc, const void* packed, const int8_t* x, int m, const float* sx,
+                               const int8_t* cq, const float* sc, float* y, float* amax, int8_t* yq, float* sy, void* stream) {
+    Geometry g;
+    if (!goq::make_geometry(desc, &g) || !packed || !x || m < 1 || !sx || !cq || !sc || !y || !amax) return GOQ_ERR_INVALID_ARG;
+    if ((yq == nullptr) != (sy == nullptr)) return GOQ_ERR_INVALID_ARG;
+    if (!aligned(packed, 128) || !aligned(x, 16) || !aligned(y, 4) || !aligned(amax, 4) || !aligned(sx, 4) || !aligned(sc, 4) ||
+        !aligned(cq, 2) || !aligned(sy, 4))
+        return GOQ_ERR_ALIGNMENT;
+    if (g.wbits > 3 || g.group < 16 || (g.k_in % 16)) return GOQ_ERR_UNSUPPORTED;
+    const long long bound = (long long)g.k_in * 127 * 127 * (1ll << ((1 << (g.wbits - 1)) - 1));
+    if (bound >= (1ll << 31)) return GOQ_ERR_OVERFLOW_BOUND;
+    if (goq_status s = check_arch()) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaError_t e = cudaMemsetAsync(amax, 0, (size_t)m * sizeof(float), st)) return from_cuda(e);
+    if (cudaError_t e = goq::launch_gemm_a8(g, packed, x, m, sx, cq, sc, y, GOQ_F32, nullptr, amax, st)) return from_cuda(e);
+    if (yq) return from_cuda(goq::launch_quantize_act(y, GOQ_F32, m, g.n_out, amax, yq, sy, st));
+    return GOQ_OK;
+}
+
+goq_status goq_quantize_activations(const void* x, int x_dtype, int m, int k, const float* amax, int8_t* xq, float* sx,
+                                    void* stream) {
+    if (!x || !xq || !sx || m < 1 || k < 1) return GOQ_ERR_INVALID_ARG;
+    if (x_dtype != GOQ_F32 && x_dtype != GOQ_BF16) return GOQ_ERR_INVALID_ARG;
+    if (!aligned(x, x_dtype == GOQ_F32 ? 4 : 2) || !aligned(sx, 4) || !aligned(amax, 4)) return GOQ_ERR_ALIGNMENT;
+    if (goq_status s = check_arch()) return s;
+    return from_cuda(goq::launch_quantize_act(x, x_dtype, m, k, amax, xq, sx, (cudaStream_t)stream));
+}
+
+goq_status goq_quantize_geo(const goq_desc* desc, const float* w, uint8_t* codes, uint8_t* meta, uint16_t* coef_f16,
+                            void* stream) {
+    Geometry g;
+    if (!goq::make_geometry(desc, &g) || !w || !codes || !meta || !coef_f16) return GOQ_ERR_INVALID_ARG;
+    if (!aligned(w, 16) || !aligned(codes, 4) || !aligned(coef_f16, 2)) return GOQ_ERR_ALIGNMENT;
+    if (goq_status s = check_arch()) return s;
+    return from_cuda(goq::launch_quantize_geo(g, w, codes, meta, coef_f16, (cudaStream_t)stream));
+}
+
+goq_status goq_solve_ref(const goq_desc* desc, const float* w, const uint8_t* codes, const uint8_t* meta,
+                         const float* x_calib, int m, double lambda, uint16_t* coef_f16, double* c_f64, void* stream) {
+    Geometry g;
+    if (!goq::make_geometry(desc, &g) || !w || !codes || !meta || !x_calib || !coef_f16 || m < 1 || !(lambda >= 0.0))
+        return GOQ_ERR_INVALID_ARG;
+    if (g.k1) return GOQ_ERR_UNSUPPORTED;
+    if (!aligned(w, 4) || !aligned(x_calib, 4) || !aligned(coef_f16, 2) || !aligned(c_f64, 8)) return GOQ_ERR_ALIGNMENT;
+    if (goq_status s = check_arch()) return s;
+    return from_cuda(goq::launch_solve_ref(g, w, codes, meta, x_calib, m, lambda, coef_f16, c_f64, (cudaStream_t)stream));
 }
 
 size_t goq_sequence_workspace_bytes(int n_items) { return n_items > 0 ? goq::gemv_seq_workspace(n_items) : 0; }

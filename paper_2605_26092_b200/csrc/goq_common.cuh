@@ -40,6 +40,7 @@ struct Geometry {
     int n_tiles, k_blocks, n_groups;  // n_groups counts padded groups: k_pad / group
     int groups_per_block;             // 128 / group
     int unit_bytes;                   // bytes of one unit record
+    int k1;                           // 1: single-basis weights (layout GOQ_LAYOUT_TILE16_K1): records and c2 are zero
     int meta_off;                     // offset of the record-byte plane inside a unit (wbits = 4 only)
     size_t n_units;
     size_t total_bytes;
@@ -49,13 +50,14 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 
 __host__ inline bool make_geometry(const goq_desc* d, Geometry* g) {
     if (!d) return false;
-    if (d->layout != GOQ_LAYOUT_TILE16) return false;
+    if (d->layout != GOQ_LAYOUT_TILE16 && d->layout != GOQ_LAYOUT_TILE16_K1) return false;
     if (d->n_out <= 0 || d->k_in <= 0) return false;
     if (d->wbits < 2 || d->wbits > 4) return false;
     int gr = d->group;
     if (!(gr == 8 || gr == 16 || gr == 32 || gr == 64 || gr == 128)) return false;
     if (d->k_in % gr) return false;
     g->n_out = d->n_out; g->k_in = d->k_in; g->group = gr; g->wbits = d->wbits;
+    g->k1 = d->layout == GOQ_LAYOUT_TILE16_K1 ? 1 : 0;
     g->n_pad = (d->n_out + kTileRows - 1) / kTileRows * kTileRows;
     g->k_pad = (d->k_in + kBlockK - 1) / kBlockK * kBlockK;
     g->n_tiles = g->n_pad / kTileRows;

@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(kA8Tokens)
 gemm_a8_dp4a_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int8_t* __restrict__ x,
                     const float* __restrict__ sx,
                     const int8_t* __restrict__ cq, const float* __restrict__ sc, void* __restrict__ y, int y_dtype,
-                    int32_t* __restrict__ acc_out, int n_out, int k_in, int k_blocks, int group, int m_total) {
+                    int32_t* __restrict__ acc_out, float* __restrict__ amax, int n_out, int k_in, int k_blocks, int group, int m_total) {
     __shared__ __align__(16) int8_t b1s[16][kBlockK];
     __shared__ __align__(16) int8_t b2s[16][kBlockK];
     __shared__ int8_t cqs[16][16][2];  // [row][group inside the k-block][basis]
@@ -110,6 +110,7 @@ gemm_a8_dp4a_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const in
     if (!tok_ok) return;
     constexpr float kInvScale = 1.0f / (float)(1u << ((1u << (WB - 1)) - 1u));
     const float sxm = sx ? sx[tok] : 1.f;
+    float vmax = 0.f;
 #pragma unroll
     for (int r = 0; r < 16; ++r) {
         const int n = T * 16 + r;
@@ -122,8 +123,12 @@ gemm_a8_dp4a_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const in
             const float v = sxm * kInvScale * (sc[n * 2] * (float)acc1[r] + sc[n * 2 + 1] * (float)acc2[r]);
             if (y_dtype == GOQ_F32) reinterpret_cast<float*>(y)[(size_t)tok * n_out + n] = v;
             else reinterpret_cast<uint16_t*>(y)[(size_t)tok * n_out + n] = f32_to_bf16_rne(v);
+            vmax = fmaxf(vmax, fabsf(v));
         }
     }
+    // requantising epilogue (Section 3.5): the token's largest output magnitude, which the next layer's activation
+    // quantizer needs before it can write a single integer; non-negative floats order like their bit patterns
+    if (amax && y) atomicMax(reinterpret_cast<int*>(amax) + tok, __float_as_int(vmax));
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -188,8 +193,8 @@ template <int WB, int CPG>
 __global__ void __launch_bounds__(kA8Warps * 32, 2)
 gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int8_t* __restrict__ x,
                    const float* __restrict__ sx, const int8_t* __restrict__ cq, const float* __restrict__ sc,
-                   void* __restrict__ y, int y_dtype, int32_t* __restrict__ acc_out, int n_out, int n_tiles, int k_in,
-                   int k_blocks, int group, int m_total) {
+                   void* __restrict__ y, int y_dtype, int32_t* __restrict__ acc_out, float* __restrict__ amax, int n_out,
+                   int n_tiles, int k_in, int k_blocks, int group, int m_total) {
     // record table: byte selectors for positions 0..3 / 4..7 and byte masks of the flipped positions, indexed by the
     // hash of the record bits, eight bank-disjoint copies (entry e, copy c at e*128 + c*16)
     __shared__ __align__(16) unsigned char lut[64 * 8 * 16];
@@ -319,7 +324,8 @@ gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int
     if (!have_tile) return;
     constexpr float kInvScale = 1.0f / (float)(1u << ((1u << (WB - 1)) - 1u));
 #pragma unroll
-    for (int nt = 0; nt < kA8NT; ++nt)
+    for (int nt = 0; nt < kA8NT; ++nt) {
+        float vmax[2] = {0.f, 0.f};   // largest output magnitude of tokens nt*8 + 2t, + 2t+1 over this lane's two rows
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             const int row = (r & 2) ? row_b : row_a;
@@ -333,18 +339,34 @@ gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int
                     const float v = sx[tok] * kInvScale * (sc[row * 2] * (float)acc1[nt][r] + sc[row * 2 + 1] * (float)acc2[nt][r]);
                     if (y_dtype == GOQ_F32) reinterpret_cast<float*>(y)[(size_t)tok * n_out + row] = v;
                     else reinterpret_cast<uint16_t*>(y)[(size_t)tok * n_out + row] = f32_to_bf16_rne(v);
+                    vmax[r & 1] = fmaxf(vmax[r & 1], fabsf(v));
                 }
             }
         }
+        if (amax && y) {   // requantising epilogue (Section 3.5): per-token largest magnitude for the next layer's quantizer
+#pragma unroll
+            for (int o = 4; o < 32; o <<= 1) {   // over the eight lanes that share these two tokens
+                vmax[0] = fmaxf(vmax[0], __shfl_xor_sync(0xFFFFFFFFu, vmax[0], o));
+                vmax[1] = fmaxf(vmax[1], __shfl_xor_sync(0xFFFFFFFFu, vmax[1], o));
+            }
+            if (g == 0) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int tok = tok0 + nt * 8 + t * 2 + e;
+                    if (tok < m_total) atomicMax(reinterpret_cast<int*>(amax) + tok, __float_as_int(vmax[e]));
+                }
+            }
+        }
+    }
 }
 
 cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* x, int m, const float* sx,
-                           const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, cudaStream_t st) {
+                           const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, float* amax, cudaStream_t st) {
     auto* words = (const uint8_t*)packed;
     if (g.group >= 32) {
         dim3 grid2((g.n_tiles + kA8Warps - 1) / kA8Warps, (m + kA8Tok - 1) / kA8Tok), block2(kA8Warps * 32);
 #define GOQ_A8_LAUNCH(WB_, CPG_)                                                                                          \
-    gemm_a8_mma_kernel<WB_, CPG_><<<grid2, block2, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, g.n_out, \
+    gemm_a8_mma_kernel<WB_, CPG_><<<grid2, block2, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, amax, g.n_out, \
                                                            g.n_tiles, g.k_in, g.k_blocks, g.group, m)
         const int cpg = g.group >> 5;   // 1, 2 or 4
         if (g.wbits == 3) { if (cpg == 1) GOQ_A8_LAUNCH(3, 1); else if (cpg == 2) GOQ_A8_LAUNCH(3, 2); else GOQ_A8_LAUNCH(3, 4); }
@@ -354,10 +376,10 @@ cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* 
     }
     dim3 grid(g.n_tiles, (m + kA8Tokens - 1) / kA8Tokens), block(kA8Tokens);
     if (g.wbits == 3)
-        gemm_a8_dp4a_kernel<3><<<grid, block, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, g.n_out, g.k_in,
+        gemm_a8_dp4a_kernel<3><<<grid, block, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, amax, g.n_out, g.k_in,
                                                        g.k_blocks, g.group, m);
     else
-        gemm_a8_dp4a_kernel<2><<<grid, block, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, g.n_out, g.k_in,
+        gemm_a8_dp4a_kernel<2><<<grid, block, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, amax, g.n_out, g.k_in,
                                                        g.k_blocks, g.group, m);
     return cudaGetLastError();
 }

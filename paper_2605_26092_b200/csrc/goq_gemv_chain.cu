@@ -125,18 +125,22 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
 
 // One micro-block word -> int8 operands (value * 2^emax): b1 (pa: weights 0..3, pb: 4..7), the routed bytes of
 // b2 (qa, qb) and the same bytes at the sign-flipped positions only (fa, fb).
-template <int WB>
+template <int WB, bool K1>
 __device__ __forceinline__ void decode_word(uint32_t w, uint32_t lut_lane, uint32_t& pa, uint32_t& pb, uint32_t& qa,
                                             uint32_t& qb, uint32_t& fa, uint32_t& fb) {
     const uint32_t m = w & 0x77777777u, mh = m >> 16;
     pa = prmt_b32(IntTables<WB>::P0, IntTables<WB>::P1, m);
     pb = prmt_b32(IntTables<WB>::P0, IntTables<WB>::P1, mh);
-    const uint32_t h = (w & 0x88888888u) * kHashMul;
-    const uint4 e = lds128(((h >> 19) & 0x1F80u) | lut_lane);   // selectors x, y; 0xFF at the flipped bytes z, w
-    qa = prmt_b32(pa, pb, e.x);
-    qb = prmt_b32(pa, pb, e.y);
-    fa = qa & e.z;
-    fb = qb & e.w;
+    if constexpr (K1) {   // single-basis weights (Section 3.1, w_hat = c1 b1): no second operand
+        qa = qb = fa = fb = 0u;
+    } else {
+        const uint32_t h = (w & 0x88888888u) * kHashMul;
+        const uint4 e = lds128(((h >> 19) & 0x1F80u) | lut_lane);   // selectors x, y; 0xFF at the flipped bytes z, w
+        qa = prmt_b32(pa, pb, e.x);
+        qb = prmt_b32(pa, pb, e.y);
+        fa = qa & e.z;
+        fb = qb & e.w;
+    }
 }
 
 // The range of CTA `cta` of `G` over `units` records, and the order it is walked in.
@@ -207,7 +211,7 @@ __device__ __forceinline__ bool flush_part(const FlushCtx& c, unsigned sq, Sums4
 }
 
 // sums of one macro-block -> fp32, times the coefficients (outside the inner product, Eq. 4)
-template <int NG>
+template <int NG, bool K1>
 __device__ __forceinline__ void group_end(int (&s1)[NG][4], int (&s2)[NG][4], int (&s3)[NG][4], uint32_t cfa, uint32_t cfb, float (&rec)[NG][2]) {
     const float c1a = __half2float(__ushort_as_half((unsigned short)(cfa & 0xFFFFu)));
     const float c2a = __half2float(__ushort_as_half((unsigned short)(cfa >> 16)));
@@ -216,14 +220,19 @@ __device__ __forceinline__ void group_end(int (&s1)[NG][4], int (&s2)[NG][4], in
 #pragma unroll
     for (int cg = 0; cg < NG; ++cg) {
         // columns 2t, 2t+1 hold the high and low activation slices of one token: S = 256 S_hi + S_lo, exact in int32
-        rec[cg][0] += c1a * (float)(s1[cg][0] * 256 + s1[cg][1]) + c2a * (float)((s2[cg][0] - 2 * s3[cg][0]) * 256 + (s2[cg][1] - 2 * s3[cg][1]));
-        rec[cg][1] += c1b * (float)(s1[cg][2] * 256 + s1[cg][3]) + c2b * (float)((s2[cg][2] - 2 * s3[cg][2]) * 256 + (s2[cg][3] - 2 * s3[cg][3]));
+        if constexpr (K1) {
+            rec[cg][0] += c1a * (float)(s1[cg][0] * 256 + s1[cg][1]);
+            rec[cg][1] += c1b * (float)(s1[cg][2] * 256 + s1[cg][3]);
+        } else {
+            rec[cg][0] += c1a * (float)(s1[cg][0] * 256 + s1[cg][1]) + c2a * (float)((s2[cg][0] - 2 * s3[cg][0]) * 256 + (s2[cg][1] - 2 * s3[cg][1]));
+            rec[cg][1] += c1b * (float)(s1[cg][2] * 256 + s1[cg][3]) + c2b * (float)((s2[cg][2] - 2 * s3[cg][2]) * 256 + (s2[cg][3] - 2 * s3[cg][3]));
+        }
 #pragma unroll
         for (int r = 0; r < 4; ++r) s1[cg][r] = s2[cg][r] = s3[cg][r] = 0;
     }
 }
 
-template <int WB, int CPG, int NG>
+template <int WB, int CPG, int NG, bool K1>
 __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_constant__ Params p) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* lut = smem + ((8192u - (smem_u32(smem) & 8191u)) & 8191u);   // 8 KiB boundary: slot offsets are OR-ed in
@@ -574,16 +583,18 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint32_t pa0, pb0, qa0, qb0, fa0, fb0, pa1, pb1, qa1, qb1, fa1, fb1;
-                        decode_word<WB>(w0[c], lut_lane, pa0, pb0, qa0, qb0, fa0, fb0);
-                        decode_word<WB>(w1[c], lut_lane, pa1, pb1, qa1, qb1, fa1, fb1);
+                        decode_word<WB, K1>(w0[c], lut_lane, pa0, pb0, qa0, qb0, fa0, fb0);
+                        decode_word<WB, K1>(w1[c], lut_lane, pa1, pb1, qa1, qb1, fa1, fb1);
 #pragma unroll
                         for (int cg = 0; cg < NG; ++cg) {
                             const uint2 xf = lds64(xrow[cg] + koff + c * 32);
                             mma_s8(s1[cg], pa0, pa1, pb0, pb1, xf.x, xf.y);
-                            mma_s8(s2[cg], qa0, qa1, qb0, qb1, xf.x, xf.y);
-                            mma_s8(s3[cg], fa0, fa1, fb0, fb1, xf.x, xf.y);
+                            if constexpr (!K1) {
+                                mma_s8(s2[cg], qa0, qa1, qb0, qb1, xf.x, xf.y);
+                                mma_s8(s3[cg], fa0, fa1, fb0, fb1, xf.x, xf.y);
+                            }
                         }
-                        if (((c + 1) % CPG) == 0) group_end<NG>(s1, s2, s3, lds32(coef_addr + (c / CPG) * 64), lds32(coef_addr + (c / CPG) * 64 + 32), rec);
+                        if (((c + 1) % CPG) == 0) group_end<NG, K1>(s1, s2, s3, lds32(coef_addr + (c / CPG) * 64), lds32(coef_addr + (c / CPG) * 64 + 32), rec);
                     }
 #pragma unroll
                     for (int cg = 0; cg < NG; ++cg) {
@@ -616,17 +627,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 }
                 for (unsigned c = cb; c < ce; ++c) {
                     uint32_t pa0, pb0, qa0, qb0, fa0, fb0, pa1, pb1, qa1, qb1, fa1, fb1;
-                    decode_word<WB>(lds32(unit + c * 4), lut_lane, pa0, pb0, qa0, qb0, fa0, fb0);
-                    decode_word<WB>(lds32(unit + 512 + c * 4), lut_lane, pa1, pb1, qa1, qb1, fa1, fb1);
+                    decode_word<WB, K1>(lds32(unit + c * 4), lut_lane, pa0, pb0, qa0, qb0, fa0, fb0);
+                    decode_word<WB, K1>(lds32(unit + 512 + c * 4), lut_lane, pa1, pb1, qa1, qb1, fa1, fb1);
 #pragma unroll
                     for (int cg = 0; cg < NG; ++cg) {
                         const uint2 xf = lds64(xrow[cg] + (uint32_t)kbi * kBlockK + c * 32);
                         mma_s8(s1[cg], pa0, pa1, pb0, pb1, xf.x, xf.y);
-                        mma_s8(s2[cg], qa0, qa1, qb0, qb1, xf.x, xf.y);
-                        mma_s8(s3[cg], fa0, fa1, fb0, fb1, xf.x, xf.y);
+                        if constexpr (!K1) {
+                            mma_s8(s2[cg], qa0, qa1, qb0, qb1, xf.x, xf.y);
+                            mma_s8(s3[cg], fa0, fa1, fb0, fb1, xf.x, xf.y);
+                        }
                     }
                     if (((c + 1) % CPG) == 0 || c + 1 == ce)   // end of a macro-block, or of this warp's share of it (the sums are linear)
-                        group_end<NG>(s1, s2, s3, lds32(coef_addr + (c / CPG) * 64), lds32(coef_addr + (c / CPG) * 64 + 32), rec);
+                        group_end<NG, K1>(s1, s2, s3, lds32(coef_addr + (c / CPG) * 64), lds32(coef_addr + (c / CPG) * 64 + 32), rec);
                 }
 #pragma unroll
                 for (int cg = 0; cg < NG; ++cg) {
@@ -693,9 +706,9 @@ size_t gemv_seq_workspace(int n_items) {
     return gemv_seq_zeroed_prefix(n_items) + n * G * 2 * chain::kPartWords * sizeof(uint2);
 }
 
-template <int WB, int CPG, int NG>
+template <int WB, int CPG, int NG, bool K1>
 static cudaError_t launch_chain_cfg(chain::Params& p, size_t x_need, cudaStream_t st) {
-    auto kernel = chain::gemv_chain_kernel<WB, CPG, NG>;
+    auto kernel = chain::gemv_chain_kernel<WB, CPG, NG, K1>;
     const size_t stage_bytes = (size_t)chain::kStageRecs * p.unit_bytes;
     const size_t fixed = chain_fixed_smem(NG);
     // two activation buffers when they leave room for four ring stages, else one
@@ -733,6 +746,7 @@ cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, i
     p.epoch = (unsigned*)(wsb + 4);
     p.parts = (uint2*)(wsb + gemv_seq_zeroed_prefix(n));
     int m_max = 1;
+    bool k1 = true;
     size_t x_need = 0;
     for (int i = 0; i < n; ++i) {
         chain::Item& it = p.item[i];
@@ -750,16 +764,20 @@ cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, i
         it.y_dtype = calls[i].y_dtype;
         it.depends = calls[i].depends;
         if (calls[i].m > m_max) m_max = calls[i].m;
+        k1 = k1 && g.k1;
         const size_t b = chain_xbuf_bytes(calls[i].m, g.k_pad);
         if (b > x_need) x_need = b;
     }
     const int cpg = group / 32;
+#define GOQ_CHAIN(WB_, NG_, K1_)                                                                             \
+    (cpg == 1 ? launch_chain_cfg<WB_, 1, NG_, K1_>(p, x_need, st) : cpg == 2 ? launch_chain_cfg<WB_, 2, NG_, K1_>(p, x_need, st) \
+                                                                             : launch_chain_cfg<WB_, 4, NG_, K1_>(p, x_need, st))
     if (m_max <= 4) {
-        if (wbits == 3) return cpg == 1 ? launch_chain_cfg<3, 1, 1>(p, x_need, st) : cpg == 2 ? launch_chain_cfg<3, 2, 1>(p, x_need, st) : launch_chain_cfg<3, 4, 1>(p, x_need, st);
-        return cpg == 1 ? launch_chain_cfg<2, 1, 1>(p, x_need, st) : cpg == 2 ? launch_chain_cfg<2, 2, 1>(p, x_need, st) : launch_chain_cfg<2, 4, 1>(p, x_need, st);
+        if (k1) return wbits == 3 ? GOQ_CHAIN(3, 1, true) : GOQ_CHAIN(2, 1, true);   // every linear single-basis: the second operand is skipped
+        return wbits == 3 ? GOQ_CHAIN(3, 1, false) : GOQ_CHAIN(2, 1, false);
     }
-    if (wbits == 3) return cpg == 1 ? launch_chain_cfg<3, 1, 2>(p, x_need, st) : cpg == 2 ? launch_chain_cfg<3, 2, 2>(p, x_need, st) : launch_chain_cfg<3, 4, 2>(p, x_need, st);
-    return cpg == 1 ? launch_chain_cfg<2, 1, 2>(p, x_need, st) : cpg == 2 ? launch_chain_cfg<2, 2, 2>(p, x_need, st) : launch_chain_cfg<2, 4, 2>(p, x_need, st);
+    return wbits == 3 ? GOQ_CHAIN(3, 2, false) : GOQ_CHAIN(2, 2, false);
+#undef GOQ_CHAIN
 }
 
 }  // namespace goq

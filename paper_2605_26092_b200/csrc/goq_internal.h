@@ -72,7 +72,14 @@ cudaError_t launch_gemm_tc(const Geometry& g, const void* packed, const void* x_
                            void* ws, cudaStream_t st);
 
 // Integer-activation layer.
+// amax (optional, with y): per-token largest |y|, combined into the array with an integer max (zero it before the launch).
 cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* x, int m, const float* sx,
-                           const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, cudaStream_t st);
+                           const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, float* amax, cudaStream_t st);
+
+// The steps before the inner product (goq_quant.cu).
+cudaError_t launch_quantize_geo(const Geometry& g, const float* w, uint8_t* codes, uint8_t* meta, uint16_t* coef, cudaStream_t st);
+cudaError_t launch_solve_ref(const Geometry& g, const float* w, const uint8_t* codes, const uint8_t* meta, const float* x_calib,
+                             int m, double lambda, uint16_t* coef, double* c_out, cudaStream_t st);
+cudaError_t launch_quantize_act(const void* x, int x_dtype, int m, int k, const float* amax, int8_t* xq, float* sx, cudaStream_t st);
 
 }  // namespace goq

@@ -9,7 +9,7 @@ namespace goq {
 
 __global__ void pack_words_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ meta,
                                   uint8_t* __restrict__ packed, int n_out, int k_in, int n_pad, int k_pad,
-                                  int wbits, int unit_bytes, int meta_off) {
+                                  int wbits, int unit_bytes, int meta_off, int k1) {
     const int mbs = k_pad / 8;
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)n_pad * mbs) return;
@@ -20,7 +20,7 @@ __global__ void pack_words_kernel(const uint8_t* __restrict__ codes, const uint8
         const uint8_t* c = codes + (size_t)row * k_in + (size_t)mb * 8;
 #pragma unroll
         for (int i = 0; i < 8; ++i) w |= ((uint32_t)c[i] & ((1u << wbits) - 1u)) << (4 * i);
-        m = meta[(size_t)row * (k_in / 8) + mb] & 63u;
+        m = k1 ? 0u : (meta[(size_t)row * (k_in / 8) + mb] & 63u);   // single-basis weights carry no exchange record
     } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i) w |= zero_code << (4 * i);
@@ -36,14 +36,14 @@ __global__ void pack_words_kernel(const uint8_t* __restrict__ codes, const uint8
 }
 
 __global__ void pack_coef_kernel(const uint16_t* __restrict__ coef, uint8_t* __restrict__ packed, int n_out,
-                                 int n_pad, int groups_in, int groups_pad, int gpb, int k_blocks, int unit_bytes) {
+                                 int n_pad, int groups_in, int groups_pad, int gpb, int k_blocks, int unit_bytes, int k1) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)n_pad * groups_pad) return;
     int row = (int)(idx / groups_pad), j = (int)(idx % groups_pad);
     uint32_t v = 0;
     if (row < n_out && j < groups_in) {
         const uint16_t* c = coef + ((size_t)row * groups_in + j) * 2;
-        v = (uint32_t)c[0] | ((uint32_t)c[1] << 16);
+        v = (uint32_t)c[0] | (k1 ? 0u : ((uint32_t)c[1] << 16));   // single-basis weights: c2 = 0
     }
     uint8_t* unit = packed + unit_offset(row >> 4, j / gpb, k_blocks, unit_bytes);
     reinterpret_cast<uint32_t*>(unit + kCodeBytesPerUnit)[(j % gpb) * 16 + (row & 15)] = v;
@@ -100,11 +100,11 @@ cudaError_t launch_pack(const Geometry& g, const uint8_t* codes, const uint8_t* 
     auto* base = (uint8_t*)packed;
     size_t nw = (size_t)g.n_pad * (g.k_pad / 8);
     pack_words_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(codes, meta, base, g.n_out, g.k_in, g.n_pad,
-                                                                   g.k_pad, g.wbits, g.unit_bytes, g.meta_off);
+                                                                   g.k_pad, g.wbits, g.unit_bytes, g.meta_off, g.k1);
     size_t nc = (size_t)g.n_pad * g.n_groups;
     pack_coef_kernel<<<(unsigned)((nc + 255) / 256), 256, 0, st>>>(coef, base, g.n_out, g.n_pad, g.k_in / g.group,
                                                                   g.n_groups, g.groups_per_block, g.k_blocks,
-                                                                  g.unit_bytes);
+                                                                  g.unit_bytes, g.k1);
     return cudaGetLastError();
 }
 

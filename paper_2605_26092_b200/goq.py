@@ -18,12 +18,14 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_OVERFLOW
 BF16, F32, I8 = 0, 1, 2
 OP_GEMV, OP_GEMM = 0, 1
 LAYOUT_TILE16 = 1
+LAYOUT_TILE16_K1 = 2
 
 EXPORTS = (
     "goq_status_string", "goq_packed_bytes", "goq_algorithmic_bytes", "goq_workspace_bytes", "goq_pack",
     "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant", "goq_workspace_init",
     "goq_workspace_status", "goq_gemv_static", "goq_last_cuda_error", "goq_sequence_workspace_bytes",
-    "goq_gemv_sequence", "goq_gemv_sequence_host", "goq_set_wait_limit", "goq_gemv_static_status",
+    "goq_gemv_sequence", "goq_gemv_sequence_host", "goq_set_wait_limit", "goq_gemv_static_status", "goq_quantize_activations", "goq_gemm_i8_requant",
+    "goq_quantize_geo", "goq_solve_ref",
 )
 
 
@@ -78,6 +80,16 @@ def lib() -> ctypes.CDLL:
         L.goq_workspace_status.argtypes = [c_void_p, c_void_p, POINTER(c_int)]
         L.goq_gemv_static.restype = c_int
         L.goq_gemv_static.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p]
+        L.goq_quantize_activations.restype = c_int
+        L.goq_quantize_activations.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.goq_gemm_i8_requant.restype = c_int
+        L.goq_gemm_i8_requant.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p,
+                                          c_void_p, c_void_p, c_void_p, c_void_p]
+        L.goq_quantize_geo.restype = c_int
+        L.goq_quantize_geo.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.goq_solve_ref.restype = c_int
+        L.goq_solve_ref.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_int, ctypes.c_double, c_void_p,
+                                    c_void_p, c_void_p]
         L.goq_gemv_static_status.restype = c_int
         L.goq_gemv_static_status.argtypes = [c_void_p, POINTER(c_int)]
         L.goq_last_cuda_error.restype = c_int
@@ -184,6 +196,26 @@ def gemv_static(d: Desc, packed, x_bf16, batch: int, y, y_dtype: int, stream=Non
     For callers that cannot allocate device memory; calls that may overlap on the GPU must not share it."""
     _check(lib().goq_gemv_static(ctypes.byref(d), _ptr(packed), _ptr(x_bf16), batch, _ptr(y), y_dtype,
                                  _stream(stream)), "goq_gemv_static")
+
+
+def quantize_activations(x, x_dtype: int, m: int, k: int, xq, sx, amax=None, stream=None):
+    _check(lib().goq_quantize_activations(_ptr(x), x_dtype, m, k, _ptr(amax), _ptr(xq), _ptr(sx), _stream(stream)),
+           "goq_quantize_activations")
+
+
+def gemm_i8_requant(d: Desc, packed, x, m: int, sx, cq, sc, y, amax, yq=None, sy=None, stream=None):
+    _check(lib().goq_gemm_i8_requant(ctypes.byref(d), _ptr(packed), _ptr(x), m, _ptr(sx), _ptr(cq), _ptr(sc), _ptr(y),
+                                     _ptr(amax), _ptr(yq), _ptr(sy), _stream(stream)), "goq_gemm_i8_requant")
+
+
+def quantize_geo(d: Desc, w, codes, meta, coef_f16, stream=None):
+    _check(lib().goq_quantize_geo(ctypes.byref(d), _ptr(w), _ptr(codes), _ptr(meta), _ptr(coef_f16), _stream(stream)),
+           "goq_quantize_geo")
+
+
+def solve_ref(d: Desc, w, codes, meta, x_calib, m: int, lam: float, coef_f16, c_f64=None, stream=None):
+    _check(lib().goq_solve_ref(ctypes.byref(d), _ptr(w), _ptr(codes), _ptr(meta), _ptr(x_calib), m, float(lam),
+                               _ptr(coef_f16), _ptr(c_f64), _stream(stream)), "goq_solve_ref")
 
 
 def gemv_static_status(stream=None) -> int:
