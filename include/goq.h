@@ -147,19 +147,22 @@ goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16
  *      cq   [n_out][k_in/group][2] int8 integer coefficients,  sc [n_out][2] fp32 their per-channel scales
  *      acc  out, optional: [2][m][n_out] int32, ACC_b[m][n] = sum_j cq[n][j][b] * sum_{k in j} x[m][k] * (2^emax b_b[n][k])
  *      y    out, optional: [m][n_out] = sx[m] * 2^-emax * (sc[n][0]*ACC_1 + sc[n][1]*ACC_2)
- *    At least one of acc, y must be given. Returns GOQ_ERR_OVERFLOW_BOUND if k_in*127*127*2^emax >= 2^31. */
+ *    At least one of acc, y must be given. Returns GOQ_ERR_OVERFLOW_BOUND if k_in*127*127*2^emax >= 2^31 (W3: k_in up
+ *    to 16642; W4, emax = 7: k_in up to 1040). wbits = 4 and groups of 16 run on the packed-dot-product kernel, wbits <= 3
+ *    with groups of 32 or more on the int8 tensor-core kernel. */
 goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int m, int x_dtype,
                     const float* sx, const int8_t* cq, const float* sc, void* y, int y_dtype,
                     int32_t* acc, void* ws, size_t ws_bytes, void* stream);
 
-/* goq_quantize_activations - the activation quantizer of Section 3.5 (X~ and s_x of Eq. 4): per-token symmetric 8-bit
- * integers, s_x[m] = max_k |x[m,k]| / 127 (1 for an all-zero token), x~ = clamp(rne(x / s_x), +-127), evaluated in
- * float64 (round half to even).
- *   x      [m][k] GOQ_F32 or GOQ_BF16        xq  out [m][k] int8        sx  out [m] fp32
+/* goq_quantize_activations - the activation quantizer of Section 3.5 (X~ and s_x of Eq. 4): per-token symmetric
+ * b_a-bit integers in int8 containers, q_max = 2^(abits-1) - 1, s_x[m] = max_k |x[m,k]| / q_max (1 for an all-zero
+ * token), x~ = clamp(rne(x / s_x), +-q_max), evaluated in float64 (round half to even). abits = 8 is the W/A8 setting,
+ * 6 and 4 the A6 / A4 settings of the accuracy tables; the integer layer (goq_gemm with GOQ_I8) takes any of them.
+ *   x      [m][k] GOQ_F32 or GOQ_BF16        xq  out [m][k] int8        sx  out [m] fp32        abits in 2..8
  *   amax   optional [m] fp32: the tokens' largest magnitudes if the caller already has them (goq_gemm_i8_requant records
  *          them in its epilogue); the kernel then reads x once instead of twice. NULL: computed here. */
-goq_status goq_quantize_activations(const void* x, int x_dtype, int m, int k, const float* amax, int8_t* xq, float* sx,
-                                    void* stream);
+goq_status goq_quantize_activations(const void* x, int x_dtype, int m, int k, int abits, const float* amax, int8_t* xq,
+                                    float* sx, void* stream);
 
 /* goq_gemm_i8_requant - the integer layer of goq_gemm (x_dtype GOQ_I8) followed by the "global rescaling or
  * requantization" of Section 3.5, after Eq. 4: y = sx * 2^-emax * (sc1 ACC_1 + sc2 ACC_2) as fp32, the per-token

@@ -23,7 +23,7 @@ What is here, with the passage each part follows:
                         A = [X_q b1, X_q b2], Y = X_q w, lambda = 1e-4.
   linear_f64            Section 3.5, Eq. 4, float activations: per-group dot products against
                         b1 and b2, coefficients applied to the group sums.
-  quantize_activations_int8 / quantize_coefficients_int8 / linear_i32
+  quantize_activations_int8 / quantize_activations_int / quantize_coefficients_int8 / linear_i32
                         Section 3.5, Eq. 4 with integer X~ and c~: exact integer S1, S2, ACC1, ACC2.
 
 Readings taken where the paper is silent (each is also listed in the design notes):
@@ -340,6 +340,19 @@ def quantize_activations_int8(x: np.ndarray):
     amax = np.max(np.abs(x), axis=1)
     sx = np.where(amax == 0.0, 1.0, amax / 127.0)
     xq = np.clip(_rne(x / sx[:, None]), -127, 127).astype(np.int8)
+    return xq, sx.astype(np.float32)
+
+
+def quantize_activations_int(x: np.ndarray, bits: int):
+    """Per-token symmetric b_a-bit integers in int8 containers (Section 3.5's b_a; the A4 / A6 settings of the accuracy
+    tables): q_max = 2^(bits-1) - 1, s_x[m] = max_k |x[m,k]| / q_max, x~ = clamp(rne(x / s_x), +-q_max)."""
+    if not 2 <= bits <= 8:
+        raise ValueError("bits must be in 2..8")
+    qmax = float((1 << (bits - 1)) - 1)
+    x = np.asarray(x, dtype=np.float64)
+    amax = np.max(np.abs(x), axis=1)
+    sx = np.where(amax == 0.0, 1.0, amax / qmax)
+    xq = np.clip(_rne(x / sx[:, None]), -qmax, qmax).astype(np.int8)
     return xq, sx.astype(np.float32)
 
 

@@ -202,7 +202,7 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
         if (!cq || (!y && !acc)) return GOQ_ERR_INVALID_ARG;
         if (y && (!sx || !sc)) return GOQ_ERR_INVALID_ARG;
         if (!aligned(acc, 4) || !aligned(sx, 4) || !aligned(sc, 4) || !aligned(cq, 2)) return GOQ_ERR_ALIGNMENT;
-        if (g.wbits > 3 || g.group < 16 || (g.k_in % 16)) return GOQ_ERR_UNSUPPORTED;
+        if (g.group < 16 || (g.k_in % 16)) return GOQ_ERR_UNSUPPORTED;
         // |ACC| <= k_in * 127 (x~) * 127 (c~) * 2^emax must stay below 2^31
         const long long bound = (long long)g.k_in * 127 * 127 * (1ll << ((1 << (g.wbits - 1)) - 1));
         if (bound >= (1ll << 31)) return GOQ_ERR_OVERFLOW_BOUND;
@@ -221,24 +221,24 @@ goq_status goq_gemm_i8_requant(const goq_desc* desc, const void* packed, const i
     if (!aligned(packed, 128) || !aligned(x, 16) || !aligned(y, 4) || !aligned(amax, 4) || !aligned(sx, 4) || !aligned(sc, 4) ||
         !aligned(cq, 2) || !aligned(sy, 4))
         return GOQ_ERR_ALIGNMENT;
-    if (g.wbits > 3 || g.group < 16 || (g.k_in % 16)) return GOQ_ERR_UNSUPPORTED;
+    if (g.group < 16 || (g.k_in % 16)) return GOQ_ERR_UNSUPPORTED;
     const long long bound = (long long)g.k_in * 127 * 127 * (1ll << ((1 << (g.wbits - 1)) - 1));
     if (bound >= (1ll << 31)) return GOQ_ERR_OVERFLOW_BOUND;
     if (goq_status s = check_arch()) return s;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaError_t e = cudaMemsetAsync(amax, 0, (size_t)m * sizeof(float), st)) return from_cuda(e);
     if (cudaError_t e = goq::launch_gemm_a8(g, packed, x, m, sx, cq, sc, y, GOQ_F32, nullptr, amax, st)) return from_cuda(e);
-    if (yq) return from_cuda(goq::launch_quantize_act(y, GOQ_F32, m, g.n_out, amax, yq, sy, st));
+    if (yq) return from_cuda(goq::launch_quantize_act(y, GOQ_F32, m, g.n_out, 8, amax, yq, sy, st));
     return GOQ_OK;
 }
 
-goq_status goq_quantize_activations(const void* x, int x_dtype, int m, int k, const float* amax, int8_t* xq, float* sx,
-                                    void* stream) {
-    if (!x || !xq || !sx || m < 1 || k < 1) return GOQ_ERR_INVALID_ARG;
+goq_status goq_quantize_activations(const void* x, int x_dtype, int m, int k, int abits, const float* amax, int8_t* xq,
+                                    float* sx, void* stream) {
+    if (!x || !xq || !sx || m < 1 || k < 1 || abits < 2 || abits > 8) return GOQ_ERR_INVALID_ARG;
     if (x_dtype != GOQ_F32 && x_dtype != GOQ_BF16) return GOQ_ERR_INVALID_ARG;
     if (!aligned(x, x_dtype == GOQ_F32 ? 4 : 2) || !aligned(sx, 4) || !aligned(amax, 4)) return GOQ_ERR_ALIGNMENT;
     if (goq_status s = check_arch()) return s;
-    return from_cuda(goq::launch_quantize_act(x, x_dtype, m, k, amax, xq, sx, (cudaStream_t)stream));
+    return from_cuda(goq::launch_quantize_act(x, x_dtype, m, k, abits, amax, xq, sx, (cudaStream_t)stream));
 }
 
 goq_status goq_quantize_geo(const goq_desc* desc, const float* w, uint8_t* codes, uint8_t* meta, uint16_t* coef_f16,

@@ -29,9 +29,14 @@ __global__ void __launch_bounds__(kA8Tokens)
 gemm_a8_dp4a_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int8_t* __restrict__ x,
                     const float* __restrict__ sx,
                     const int8_t* __restrict__ cq, const float* __restrict__ sc, void* __restrict__ y, int y_dtype,
-                    int32_t* __restrict__ acc_out, float* __restrict__ amax, int n_out, int k_in, int k_blocks, int group, int m_total) {
+                    int32_t* __restrict__ acc_out, float* __restrict__ amax, int n_out, int k_in, int k_blocks, int group, int m_total,
+                    int meta_off) {
     __shared__ __align__(16) int8_t b1s[16][kBlockK];
     __shared__ __align__(16) int8_t b2s[16][kBlockK];
+    // W4: 2^emax = 128 does not fit a signed byte, so an integer weight v = +-2^(7-e) is held as v = 2 h + l with
+    // h = v / 2 for e <= 6 (|h| <= 64) and l = +-1 for e = 7: S = 2 (x . h) + (x . l), still exact integer arithmetic
+    __shared__ __align__(16) int8_t b1l[WB == 4 ? 16 : 1][kBlockK];
+    __shared__ __align__(16) int8_t b2l[WB == 4 ? 16 : 1][kBlockK];
     __shared__ int8_t cqs[16][16][2];  // [row][group inside the k-block][basis]
 
     const int T = blockIdx.x;
@@ -52,15 +57,22 @@ gemm_a8_dp4a_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const in
                 reinterpret_cast<const uint32_t*>(packed + unit_offset(T, bk, k_blocks, unit_bytes))[wi];
             const int v = wi >> 7, ln = (wi >> 2) & 31, c = wi & 3;
             const int row = v * 8 + (ln >> 2), kk = c * 32 + (ln & 3) * 8;
-            const uint32_t meta = gather_meta(w);
-            const uint32_t cw = w & 0x77777777u;
+            const uint32_t meta = WB == 4 ? (uint32_t)(packed + unit_offset(T, bk, k_blocks, unit_bytes))[meta_off + wi] : gather_meta(w);
+            const uint32_t cw = WB == 4 ? w : (w & 0x77777777u);
             const uint32_t src = xor_permute_nibbles(cw, (int)(meta & 3u) + 1);
             const uint32_t flips = flip_mask(meta);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                b1s[row][kk + i] = (int8_t)pot_int<WB>((cw >> (4 * i)) & 15u);
-                const int v2 = pot_int<WB>((src >> (4 * i)) & 15u);
-                b2s[row][kk + i] = (int8_t)(((flips >> i) & 1u) ? -v2 : v2);
+                const int v1 = pot_int<WB>((cw >> (4 * i)) & 15u);
+                const int u2 = pot_int<WB>((src >> (4 * i)) & 15u);
+                const int v2 = ((flips >> i) & 1u) ? -u2 : u2;
+                if constexpr (WB == 4) {
+                    b1s[row][kk + i] = (int8_t)(v1 / 2); b1l[row][kk + i] = (int8_t)(v1 % 2);
+                    b2s[row][kk + i] = (int8_t)(v2 / 2); b2l[row][kk + i] = (int8_t)(v2 % 2);
+                } else {
+                    b1s[row][kk + i] = (int8_t)v1;
+                    b2s[row][kk + i] = (int8_t)v2;
+                }
             }
         }
         for (int i = threadIdx.x; i < 16 * gpb * 2; i += kA8Tokens) {
@@ -96,6 +108,22 @@ gemm_a8_dp4a_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const in
                         s2 = __dp4a((int)xr[q].z, (int)b.z, s2);
                         s2 = __dp4a((int)xr[q].w, (int)b.w, s2);
                     }
+                }
+                if constexpr (WB == 4) {
+                    int l1 = 0, l2 = 0;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (q >= q0 && q < q1) {
+                            const uint4 a = *reinterpret_cast<const uint4*>(&b1l[row][q * 16]);
+                            const uint4 b = *reinterpret_cast<const uint4*>(&b2l[row][q * 16]);
+                            l1 = __dp4a((int)xr[q].x, (int)a.x, l1); l1 = __dp4a((int)xr[q].y, (int)a.y, l1);
+                            l1 = __dp4a((int)xr[q].z, (int)a.z, l1); l1 = __dp4a((int)xr[q].w, (int)a.w, l1);
+                            l2 = __dp4a((int)xr[q].x, (int)b.x, l2); l2 = __dp4a((int)xr[q].y, (int)b.y, l2);
+                            l2 = __dp4a((int)xr[q].z, (int)b.z, l2); l2 = __dp4a((int)xr[q].w, (int)b.w, l2);
+                        }
+                    }
+                    s1 = 2 * s1 + l1;
+                    s2 = 2 * s2 + l2;
                 }
                 // acc[row] with a compile-time index
 #pragma unroll
@@ -363,7 +391,7 @@ gemm_a8_mma_kernel(const uint8_t* __restrict__ packed, int unit_bytes, const int
 cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* x, int m, const float* sx,
                            const int8_t* cq, const float* sc, void* y, int y_dtype, int32_t* acc, float* amax, cudaStream_t st) {
     auto* words = (const uint8_t*)packed;
-    if (g.group >= 32) {
+    if (g.group >= 32 && g.wbits <= 3) {
         dim3 grid2((g.n_tiles + kA8Warps - 1) / kA8Warps, (m + kA8Tok - 1) / kA8Tok), block2(kA8Warps * 32);
 #define GOQ_A8_LAUNCH(WB_, CPG_)                                                                                          \
     gemm_a8_mma_kernel<WB_, CPG_><<<grid2, block2, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, amax, g.n_out, \
@@ -375,12 +403,13 @@ cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* 
         return cudaGetLastError();
     }
     dim3 grid(g.n_tiles, (m + kA8Tokens - 1) / kA8Tokens), block(kA8Tokens);
-    if (g.wbits == 3)
-        gemm_a8_dp4a_kernel<3><<<grid, block, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, amax, g.n_out, g.k_in,
-                                                       g.k_blocks, g.group, m);
-    else
-        gemm_a8_dp4a_kernel<2><<<grid, block, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, amax, g.n_out, g.k_in,
-                                                       g.k_blocks, g.group, m);
+#define GOQ_A8_DP4A(WB_)                                                                                                    \
+    gemm_a8_dp4a_kernel<WB_><<<grid, block, 0, st>>>(words, g.unit_bytes, x, sx, cq, sc, y, y_dtype, acc, amax, g.n_out, g.k_in, \
+                                                     g.k_blocks, g.group, m, g.meta_off)
+    if (g.wbits == 4) GOQ_A8_DP4A(4);
+    else if (g.wbits == 3) GOQ_A8_DP4A(3);
+    else GOQ_A8_DP4A(2);
+#undef GOQ_A8_DP4A
     return cudaGetLastError();
 }
 

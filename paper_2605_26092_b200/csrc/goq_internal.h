@@ -80,6 +80,7 @@ cudaError_t launch_gemm_a8(const Geometry& g, const void* packed, const int8_t* 
 cudaError_t launch_quantize_geo(const Geometry& g, const float* w, uint8_t* codes, uint8_t* meta, uint16_t* coef, cudaStream_t st);
 cudaError_t launch_solve_ref(const Geometry& g, const float* w, const uint8_t* codes, const uint8_t* meta, const float* x_calib,
                              int m, double lambda, uint16_t* coef, double* c_out, cudaStream_t st);
-cudaError_t launch_quantize_act(const void* x, int x_dtype, int m, int k, const float* amax, int8_t* xq, float* sx, cudaStream_t st);
+cudaError_t launch_quantize_act(const void* x, int x_dtype, int m, int k, int abits, const float* amax, int8_t* xq, float* sx,
+                                cudaStream_t st);
 
 }  // namespace goq

@@ -234,7 +234,8 @@ solve_ref_kernel(const float* __restrict__ w, const uint8_t* __restrict__ codes,
 }
 
 // ---- activation quantizer (Section 3.5: X~, s_x) -----------------------------------------------------------
-// Per token: s_x = max |x| / 127 (1 for an all-zero token), x~ = clamp(rne(x / s_x), +-127). One CTA per token; when the
+// Per token: s_x = max |x| / q_max (1 for an all-zero token), x~ = clamp(rne(x / s_x), +-q_max), q_max = 2^(bits-1) - 1,
+// in int8 containers whatever the width. One CTA per token; when the
 // caller already has the token's largest magnitude (the integer GEMM's epilogue can record it) the first pass is skipped.
 template <typename T> __device__ __forceinline__ double load_act(const T* p);
 template <> __device__ __forceinline__ double load_act<float>(const float* p) { return (double)*p; }
@@ -242,7 +243,8 @@ template <> __device__ __forceinline__ double load_act<uint16_t>(const uint16_t*
 
 template <typename T>
 __global__ void __launch_bounds__(256)
-quantize_act_kernel(const T* __restrict__ x, int k, const float* __restrict__ amax_in, int8_t* __restrict__ xq, float* __restrict__ sx) {
+quantize_act_kernel(const T* __restrict__ x, int k, const float* __restrict__ amax_in, int8_t* __restrict__ xq, float* __restrict__ sx,
+                    double qmax) {
     __shared__ double red[8];
     __shared__ double s_amax;
     const int tok = blockIdx.x, tid = threadIdx.x;
@@ -262,10 +264,10 @@ quantize_act_kernel(const T* __restrict__ x, int k, const float* __restrict__ am
         }
     }
     __syncthreads();
-    const double s = s_amax == 0.0 ? 1.0 : s_amax / 127.0;
+    const double s = s_amax == 0.0 ? 1.0 : s_amax / qmax;
     for (int i = tid; i < k; i += 256) {
         double q = rint(load_act<T>(row + i) / s);   // round half to even
-        q = fmin(127.0, fmax(-127.0, q));
+        q = fmin(qmax, fmax(-qmax, q));
         xq[(size_t)tok * k + i] = (int8_t)(int)q;
     }
     if (tid == 0) sx[tok] = (float)s;
@@ -287,9 +289,11 @@ cudaError_t launch_solve_ref(const Geometry& g, const float* w, const uint8_t* c
                                                                  g.group, g.wbits);
     return cudaGetLastError();
 }
-cudaError_t launch_quantize_act(const void* x, int x_dtype, int m, int k, const float* amax, int8_t* xq, float* sx, cudaStream_t st) {
-    if (x_dtype == GOQ_F32) quant::quantize_act_kernel<float><<<m, 256, 0, st>>>((const float*)x, k, amax, xq, sx);
-    else quant::quantize_act_kernel<uint16_t><<<m, 256, 0, st>>>((const uint16_t*)x, k, amax, xq, sx);
+cudaError_t launch_quantize_act(const void* x, int x_dtype, int m, int k, int abits, const float* amax, int8_t* xq, float* sx,
+                                cudaStream_t st) {
+    const double qmax = (double)((1 << (abits - 1)) - 1);
+    if (x_dtype == GOQ_F32) quant::quantize_act_kernel<float><<<m, 256, 0, st>>>((const float*)x, k, amax, xq, sx, qmax);
+    else quant::quantize_act_kernel<uint16_t><<<m, 256, 0, st>>>((const uint16_t*)x, k, amax, xq, sx, qmax);
     return cudaGetLastError();
 }
 

@@ -81,7 +81,7 @@ def lib() -> ctypes.CDLL:
         L.goq_gemv_static.restype = c_int
         L.goq_gemv_static.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p]
         L.goq_quantize_activations.restype = c_int
-        L.goq_quantize_activations.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.goq_quantize_activations.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
         L.goq_gemm_i8_requant.restype = c_int
         L.goq_gemm_i8_requant.argtypes = [POINTER(Desc), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p,
                                           c_void_p, c_void_p, c_void_p, c_void_p]
@@ -198,8 +198,8 @@ def gemv_static(d: Desc, packed, x_bf16, batch: int, y, y_dtype: int, stream=Non
                                  _stream(stream)), "goq_gemv_static")
 
 
-def quantize_activations(x, x_dtype: int, m: int, k: int, xq, sx, amax=None, stream=None):
-    _check(lib().goq_quantize_activations(_ptr(x), x_dtype, m, k, _ptr(amax), _ptr(xq), _ptr(sx), _stream(stream)),
+def quantize_activations(x, x_dtype: int, m: int, k: int, xq, sx, amax=None, abits: int = 8, stream=None):
+    _check(lib().goq_quantize_activations(_ptr(x), x_dtype, m, k, abits, _ptr(amax), _ptr(xq), _ptr(sx), _stream(stream)),
            "goq_quantize_activations")
 
 

@@ -86,6 +86,28 @@ def test_activation_quantizer_bit_equal_to_oracle(goq, dtype):
         assert np.array_equal(sx.cpu().numpy(), sx_ref)
 
 
+@pytest.mark.parametrize("abits,b,g,k", [(4, 3, 64, 768), (6, 3, 128, 1024), (8, 4, 64, 768), (4, 4, 32, 512), (8, 4, 16, 256)])
+def test_narrow_activations_and_w4_on_the_integer_path(goq, abits, b, g, k):
+    """A4 / A6 activations in int8 containers (quantised on the device, bit-equal to the oracle) through the integer
+    layer, and W4 weights (2^emax = 128 split over two signed bytes): ACC_1, ACC_2 bit-exact against the oracle."""
+    from tests.gpu_util import pack_weights, run_gemm_i8
+    n, m = 72, 150
+    codes, meta, coef = O.quantize_geo(si.weights_with_outlier_channels(n, k, seed=abits + b), g, b)
+    cq, sc = O.quantize_coefficients_int8(coef)
+    x = si.f32_activations(m, k, seed=abits).astype(np.float32)
+    xq_ref, sx_ref = O.quantize_activations_int(x, abits)
+    xq = torch.empty((m, k), dtype=torch.int8, device="cuda")
+    sx = torch.empty((m,), dtype=torch.float32, device="cuda")
+    goq.quantize_activations(torch.from_numpy(x).cuda(), goq.F32, m, k, xq, sx, abits=abits)
+    torch.cuda.synchronize()
+    assert np.array_equal(xq.cpu().numpy(), xq_ref) and np.array_equal(sx.cpu().numpy(), sx_ref)
+    d, packed = pack_weights(n, k, g, b, codes, meta, coef)
+    acc, y = run_gemm_i8(d, packed, xq_ref, sx_ref, cq, sc)
+    a1, a2, y_ref = O.linear_i32(codes, meta, cq, sc, xq_ref, sx_ref, g, b)
+    assert np.array_equal(acc[0], a1) and np.array_equal(acc[1], a2)
+    assert O.normwise_rel_err(y, y_ref) <= TIGHT
+
+
 def test_integer_layer_with_requantising_epilogue(goq):
     """goq_gemm_i8_requant: y equals goq_gemm's y bit for bit, the recorded per-token maxima equal max |y| exactly, and
     the requantised output equals the oracle's quantizer applied to the y actually produced (Section 3.5)."""

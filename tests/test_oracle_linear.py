@@ -143,3 +143,19 @@ def test_bf16_helpers_roundtrip():
     assert np.array_equal(t.view(torch.int16).numpy().view(np.uint16), bits)
     y = np.array([1.00390625, 1.01171875], dtype=np.float32)    # ties: round to even
     assert si.f32_to_bf16_bits(y).tolist() == [0x3F80, 0x3F82]
+
+
+@pytest.mark.parametrize("bits", [4, 6, 8])
+def test_narrow_activation_integers_in_byte_containers(bits):
+    """b_a-bit activations (Section 3.5): the 8-bit case is the int8 quantizer; every width reaches +-q_max, stays inside
+    it, and is off by at most half a step (the grid is uniform, so round-to-nearest means |x - s q| <= s / 2)."""
+    x = si.f32_activations(9, 300, seed=bits)
+    x[3] = 0.0
+    xq, sx = O.quantize_activations_int(x, bits)
+    qmax = (1 << (bits - 1)) - 1
+    if bits == 8:
+        xq8, sx8 = O.quantize_activations_int8(x)
+        assert np.array_equal(xq, xq8) and np.array_equal(sx, sx8)
+    assert xq.dtype == np.int8 and np.abs(xq.astype(int)).max() == qmax and not xq[3].any() and sx[3] == 1.0
+    s64 = np.where(np.max(np.abs(x), 1) == 0, 1.0, np.max(np.abs(x), 1) / qmax)
+    assert np.all(np.abs(x - s64[:, None] * xq) <= 0.5 * s64[:, None] * (1 + 1e-12))
