@@ -29,6 +29,9 @@ import synth_inputs as si  # noqa: E402
 
 GROUP = 128
 WBITS = 3
+# what the timed kernel computes in: bf16 activations become 16-bit block fixed point (two int8 slices per value), the PoT
+# weights small integers; sums are exact in int32, the coefficient multiply and the sum over macro-blocks are fp32
+DTYPE = "int8 x int8 -> int32 (bf16 activations as 16-bit block fixed point), f32 coefficient stage"
 METRIC = "w3a16_gemv_hbm_gbs"
 UNIT = "GB/s"
 WORKLOAD = "llama2-7b-shaped linear stack (32 layers x 7 linears), W3 dual-basis PoT, group 128, batch-1 decode GEMV"
@@ -39,7 +42,9 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
+        measured_peaks.sustained = float(p.get("bf16_tflops_sustained", 1400.0))
         return float(p["hbm_gbs"]), float(p.get("bf16_tflops", 1590.0)), "measured (MEASURED_PEAKS.json)"
+    measured_peaks.sustained = 1400.0
     return 6650.0, 1590.0, "fallback (earlier measurement on this pool)"
 
 
@@ -226,6 +231,37 @@ def time_graph(torch, graph, steps, warmup):
     return e0.elapsed_time(e1) / steps  # ms per step
 
 
+def time_loop_with_clocks(torch, fn, device_index, min_seconds=0.5, warmup=3):
+    """Run fn() back to back for at least min_seconds with the clock sampler around the timed region.
+    Returns (ms per call, clock summary)."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+    reps = max(3, int(min_seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3)) + 1)
+    sampler = ClockSampler(device_index)
+    with sampler:
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps, sampler.summary()
+
+
+def clock_fractions(value, clocks, peaks):
+    """value against each peak, as measured and rescaled to the maximum SM clock (value * max MHz / median MHz)."""
+    out = {"clocks": clocks}
+    mhz, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    scaled = value * mx / mhz if mhz and mx else None
+    out["at_max_clock"] = scaled
+    for name, pk in peaks.items():
+        out["frac_of_" + name] = value / pk
+    return out
+
+
 def replica_seed(rank):
     """Each rank is an independent replica of the decode step with its own weights and activations."""
     return 1000 * rank
@@ -379,7 +415,7 @@ def run_cuda(args):
     if args.launch == "sequence":
         kernel_name = "gemv_chain_kernel<3,4,1>"
         launch_desc = "one CUDA graph holding one goq_gemv_sequence call (%d linears, each waits for all earlier ones)" % n_lin
-        ratio, ratio_src = NCU_TRAFFIC_RATIO_SEQ, "ncu dram bytes of a 14-linear sequence launch scaled by algorithmic bytes"
+        ratio, ratio_src = NCU_TRAFFIC_RATIO_SEQ, "ncu dram bytes of a 14-linear chain launch (profiles/gemv_chain_llama7b_2layers_batch1.md) scaled by algorithmic bytes"
         if int(goq.workspace_status(ws_seq)) != 0:
             raise RuntimeError("sequence kernel reported a device-side timeout")
     else:
@@ -395,7 +431,7 @@ def run_cuda(args):
         traffic, traffic_src = (launch_bytes * ratio, ratio_src) if ratio else (None, "not captured")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": DTYPE,
         "data": "synthetic",
         "config": {"workload": WORKLOAD, "layers": layers, "linears_per_step": n_lin, "batch": 1,
                    "bytes_per_step": step_bytes, "l2": "weights per step %.2f GB >> 126 MB L2, no flush needed" % (step_bytes / 1e9),
@@ -507,48 +543,36 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
         shapes[(n, k)] = {"us": us, "gbs": algorithmic_bytes(n, k, 1) / (us * 1e-6) / 1e9}
         del g
     out["gemv_batch1_per_shape"] = {"%dx%d" % k: v for k, v in shapes.items()}
-    # prefill GEMM, M = 2048, one layer's seven linears
+    # prefill GEMM, M = 2048, over every linear of the stack (32 layers x 7: the packed weights are resident), repeated
+    # for at least half a second with the clock sampler around exactly that region. Inputs per shape are shared (a linear
+    # stack with independent inputs), outputs per shape are reused.
     m = 2048
-    layer0 = stack[:7]
-    xs = [torch.randn((m, s["k"]), device="cuda").to(torch.bfloat16) for s in layer0]
-    ys = [torch.empty((m, s["n"]), dtype=torch.float32, device="cuda") for s in layer0]
-
-    ws_gemm = torch.empty(max(goq.workspace_bytes(s["d"], goq.OP_GEMM, m) for s in layer0), dtype=torch.uint8, device="cuda")
+    dev_index = torch.cuda.current_device()
+    xs_k = {k: torch.randn((m, k), device="cuda").to(torch.bfloat16) for k in sorted({s["k"] for s in stack})}
+    ys_n = {n: torch.empty((m, n), dtype=torch.float32, device="cuda") for n in sorted({s["n"] for s in stack})}
+    ws_gemm = torch.empty(max(goq.workspace_bytes(s["d"], goq.OP_GEMM, m) for s in stack[:7]), dtype=torch.uint8, device="cuda")
     goq.workspace_init(ws_gemm)
 
-    def step_gemm():
-        for s, x, y in zip(layer0, xs, ys):
-            goq.gemm(s["d"], s["packed"], x, m, goq.BF16, y=y, y_dtype=goq.F32, ws=ws_gemm)
+    def step_gemm_stack():
+        for s in stack:
+            goq.gemm(s["d"], s["packed"], xs_k[s["k"]], m, goq.BF16, y=ys_n[s["n"]], y_dtype=goq.F32, ws=ws_gemm)
 
-    step_gemm()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(3):
-        step_gemm()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / 3
-    flops = sum(2.0 * m * s["n"] * s["k"] for s in layer0)
-    out["gemm_m2048_layer_tflops"] = flops / (ms * 1e-3) / 1e12
-    out["gemm_m2048_frac_of_bf16_peak"] = out["gemm_m2048_layer_tflops"] / tf_peak
-    # the same layer with bf16 outputs (half the bytes of the epilogue's store burst)
-    yb = [torch.empty((m, s["n"]), dtype=torch.bfloat16, device="cuda") for s in layer0]
+    ms, clk = time_loop_with_clocks(torch, step_gemm_stack, dev_index)
+    flops = sum(2.0 * m * s["n"] * s["k"] for s in stack)
+    tf = flops / (ms * 1e-3) / 1e12
+    out["gemm_m2048_stack_tflops"] = tf
+    out["gemm_m2048_stack_ms"] = ms
+    out["gemm_m2048_stack"] = clock_fractions(tf, clk, {"bf16_burst_peak": tf_peak, "bf16_sustained_peak": measured_peaks.sustained})
+    out["gemm_m2048_frac_of_bf16_peak"] = tf / tf_peak
+    yb_n = {n: torch.empty((m, n), dtype=torch.bfloat16, device="cuda") for n in ys_n}
 
     def step_gemm_bf16_out():
-        for s, x, y in zip(layer0, xs, yb):
-            goq.gemm(s["d"], s["packed"], x, m, goq.BF16, y=y, y_dtype=goq.BF16, ws=ws_gemm)
+        for s in stack[:7]:
+            goq.gemm(s["d"], s["packed"], xs_k[s["k"]], m, goq.BF16, y=yb_n[s["n"]], y_dtype=goq.BF16, ws=ws_gemm)
 
-    step_gemm_bf16_out()
-    torch.cuda.synchronize()
-    e0.record()
-    for _ in range(3):
-        step_gemm_bf16_out()
-    e1.record()
-    torch.cuda.synchronize()
-    out["gemm_m2048_layer_tflops_bf16_out"] = flops / (e0.elapsed_time(e1) / 3 * 1e-3) / 1e12
-    del yb
-    del xs, ys, ws_gemm
+    ms_l, _ = time_loop_with_clocks(torch, step_gemm_bf16_out, dev_index, min_seconds=0.1)
+    out["gemm_m2048_layer_tflops_bf16_out"] = sum(2.0 * m * s["n"] * s["k"] for s in stack[:7]) / (ms_l * 1e-3) / 1e12
+    del xs_k, ys_n, yb_n, ws_gemm
     # batch-size crossover on one 70B-shaped linear (8192 x 8192, g128) at W3, W2 and W4: goq_gemv up to batch 16,
     # goq_gemm from there on; eight copies of the weights are rotated so every call reads cold weights
     n = k = 8192
@@ -566,7 +590,7 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
             copies.append(pk)
             del codes, meta, coef
         cross = {}
-        for batch in (1, 4, 16, 48, 64, 256):
+        for batch in (1, 4, 16, 32, 33, 64, 256):
             x = torch.randn((batch, k), device="cuda").to(torch.bfloat16)
             y = torch.empty((batch, n), dtype=torch.float32, device="cuda")
             paths = (["gemv"] if batch <= 16 else []) + (["gemm"] if batch >= 16 else [])
@@ -611,17 +635,13 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
         for v in vit:
             goq.gemm(v["d"], v["packed"], v["x"], mt, goq.I8, sx=v["sx"], cq=v["cq"], sc=v["sc"], acc=v["acc"])
 
-    step_a8()
-    torch.cuda.synchronize()
-    e0.record()
-    for _ in range(3):
-        step_a8()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / 3
+    ms, clk = time_loop_with_clocks(torch, step_a8, dev_index)
     ops = sum(2.0 * 2.0 * mt * v["n"] * v["k"] for v in vit)  # two bases, multiply-add = 2 ops
-    out["w3a8_vit_b16_int_tops"] = ops / (ms * 1e-3) / 1e12
+    tops = ops / (ms * 1e-3) / 1e12
+    out["w3a8_vit_b16_int_tops"] = tops
     out["w3a8_vit_b16_ms"] = ms
+    # int8 peak taken as twice the measured bf16 figures (the nominal ratio of the dense rates)
+    out["w3a8_vit_b16"] = clock_fractions(tops, clk, {"int8_burst_peak_2x_bf16": 2 * tf_peak, "int8_sustained_peak_2x_bf16": 2 * measured_peaks.sustained})
     # the same linears with the scaled bf16 output instead of the two int32 accumulator planes (2 against 8 bytes per output)
     ys_a8 = [torch.empty((mt, v["n"]), dtype=torch.bfloat16, device="cuda") for v in vit]
 
@@ -629,20 +649,109 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
         for v, yv in zip(vit, ys_a8):
             goq.gemm(v["d"], v["packed"], v["x"], mt, goq.I8, sx=v["sx"], cq=v["cq"], sc=v["sc"], y=yv, y_dtype=goq.BF16)
 
-    step_a8_y()
-    torch.cuda.synchronize()
-    e0.record()
-    for _ in range(3):
-        step_a8_y()
-    e1.record()
-    torch.cuda.synchronize()
-    out["w3a8_vit_b16_int_tops_bf16_out"] = ops / (e0.elapsed_time(e1) / 3 * 1e-3) / 1e12
+    ms_y, _ = time_loop_with_clocks(torch, step_a8_y, dev_index, min_seconds=0.1)
+    out["w3a8_vit_b16_int_tops_bf16_out"] = ops / (ms_y * 1e-3) / 1e12
     del ys_a8
+    del vit
+    # steady state of the decode GEMV: one 70B-shaped 28672 x 8192 linear (117 MB of weights), eight copies rotated so
+    # that every call streams from HBM; as single goq_gemv calls and as one chain of eight independent linears
+    big = []
+    for c in range(8):
+        gen.manual_seed(8000 + c)
+        n, k = 28672, 8192
+        d = goq.desc(n, k, GROUP, WBITS)
+        codes = torch.randint(0, 1 << WBITS, (n, k), dtype=torch.uint8, device="cuda", generator=gen)
+        meta = torch.randint(0, 64, (n, k // 8), dtype=torch.uint8, device="cuda", generator=gen)
+        coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * 0.03).to(torch.float16)
+        pk = torch.empty(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
+        goq.pack(d, codes, meta, coef, pk)
+        big.append({"d": d, "packed": pk, "n": n, "k": k, "x": torch.randn((1, k), device="cuda", generator=gen).to(torch.bfloat16),
+                    "y": torch.empty((1, n), dtype=torch.float32, device="cuda")})
+        del codes, meta, coef
+    nbytes = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in big)
+    ws_big = goq.new_workspace(big[0]["d"], goq.OP_GEMV, 1)
+    g = capture(torch, lambda: [goq.gemv(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, ws=ws_big) for s in big])
+    out["gemv_batch1_steady_gbs"] = nbytes / (time_graph(torch, g, 10, 3) * 1e-3) / 1e9
+    del g
+    seq_big = goq.make_sequence([(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, False) for s in big])
+    ws_sb = torch.empty(goq.sequence_workspace_bytes(len(big)), dtype=torch.uint8, device="cuda")
+    goq.workspace_init(ws_sb)
+    g = capture(torch, lambda: goq.gemv_sequence(seq_big, ws_sb))
+    out["gemv_batch1_steady_chain_gbs"] = nbytes / (time_graph(torch, g, 10, 3) * 1e-3) / 1e9
+    del g, big, seq_big
+    # the same decode step with bf16 operands (exponent shift of the bf16 activation in the tensor core: the streaming kernel)
+    prev = goq.set_gemv_variant(3)
+    try:
+        g = capture(torch, step_graph)
+        out["gemv_bf16_operand_form_gbs"] = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack) / (time_graph(torch, g, 10, 3) * 1e-3) / 1e9
+        del g
+    finally:
+        goq.set_gemv_variant(prev)
+    # GEO quantizer on the device: the 7B stack's shapes, fp32 weights in, codes + records + fp16 pairs out
+    # (algorithmic bytes per weight: 4 read, 1 + 1/8 + 4/group written)
+    qt = {}
+    total_s = 0.0
+    for (n, k), count in (((4096, 4096), 4), ((11008, 4096), 2), ((4096, 11008), 1)):
+        d = goq.desc(n, k, GROUP, WBITS)
+        w = torch.randn((n, k), device="cuda") * 0.02
+        codes = torch.empty((n, k), dtype=torch.uint8, device="cuda")
+        meta = torch.empty((n, k // 8), dtype=torch.uint8, device="cuda")
+        coef = torch.empty((n, k // GROUP, 2), dtype=torch.float16, device="cuda")
+        ms_q, _ = time_loop_with_clocks(torch, lambda: goq.quantize_geo(d, w, codes, meta, coef), dev_index, min_seconds=0.05)
+        qbytes = n * k * (4 + 1 + 0.125) + n * (k // GROUP) * 4
+        qt["%dx%d" % (n, k)] = {"us": ms_q * 1e3, "gbs": qbytes / (ms_q * 1e-3) / 1e9}
+        total_s += ms_q * 1e-3 * count * layers
+        del w, codes, meta, coef
+    out["quantize_geo_per_shape"] = qt
+    out["quantize_geo_7b_stack_seconds"] = total_s   # context: the paper reports 0.47 min for LLaMA-2-7B on its own hardware
     return out
 
 
 NCU_TRAFFIC_RATIO = 8.96 / 8.39
-NCU_TRAFFIC_RATIO_SEQ = (215.2 + 3.9) / 202.9   # ncu: 215.2 MB read + 3.9 MB written for the 202.9 MB (algorithmic) of a 14-linear launch
+NCU_TRAFFIC_RATIO_SEQ = (215.2 + 4.2) / 202.9   # ncu: 215.2 MB read + 4.2 MB written for the 202.9 MB (algorithmic) of a 14-linear launch
+
+
+def run_probe_steady(args):
+    """`--probe steady`: only the steady-state case of the decode GEMV - a chain of `--copies` independent 28672 x 8192
+    linears (117 MB each) - a few times. Small enough for a profiler capture of one launch; prints one JSON line."""
+    import torch
+    from paper_2605_26092_b200 import build
+    build.build()
+    from paper_2605_26092_b200 import goq
+    gen = torch.Generator(device="cuda")
+    n, k = 28672, 8192
+    d = goq.desc(n, k, GROUP, WBITS)
+    items, keep = [], []
+    for c in range(args.copies):
+        gen.manual_seed(8000 + c)
+        codes = torch.randint(0, 1 << WBITS, (n, k), dtype=torch.uint8, device="cuda", generator=gen)
+        meta = torch.randint(0, 64, (n, k // 8), dtype=torch.uint8, device="cuda", generator=gen)
+        coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * 0.03).to(torch.float16)
+        pk = torch.empty(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
+        goq.pack(d, codes, meta, coef, pk)
+        x = torch.randn((1, k), device="cuda", generator=gen).to(torch.bfloat16)
+        y = torch.empty((1, n), dtype=torch.float32, device="cuda")
+        keep += [pk, x, y]
+        items.append((d, pk, x, 1, y, goq.F32, False))
+        del codes, meta, coef
+    seq = goq.make_sequence(items)
+    ws = torch.empty(goq.sequence_workspace_bytes(len(items)), dtype=torch.uint8, device="cuda")
+    goq.workspace_init(ws)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    best = float("inf")
+    for _ in range(max(args.steps, 1) + max(args.warmup, 1)):
+        e0.record(); goq.gemv_sequence(seq, ws); e1.record(); torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    nbytes = args.copies * algorithmic_bytes(n, k, 1)
+    print(json.dumps({"probe": "steady", "copies": args.copies, "algorithmic_bytes": nbytes, "best_ms": best,
+                      "gbs": nbytes / (best * 1e-3) / 1e9, "status": int(goq.workspace_status(ws))}))
+
+
+def launch_command(n_gpus, argv, port=None):
+    """The command that starts one rank per GPU on this node for `bench.py --gpus N` (N > 1) when no launcher has."""
+    port = port or (29500 + os.getpid() % 2000)
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n_gpus),
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
 
 
 def main():
@@ -660,7 +769,16 @@ def main():
                     help="force a kernel variant (goq_set_gemv_variant): 0 automatic, 3 streaming, 4 tcgen05 tensor-memory GEMV, ...")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="dram bytes per launch of the dominant kernel from an ncu capture (reported as-is)")
+    ap.add_argument("--probe", choices=("steady",), default=None, help="run one small case only (for profiler captures)")
+    ap.add_argument("--copies", type=int, default=2, help="--probe steady: number of 28672 x 8192 linears in the chain")
     args = ap.parse_args()
+    if args.probe == "steady":
+        if args.steps == 200:
+            args.steps = 3
+        return run_probe_steady(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # asked for N GPUs without a launcher: start the N ranks (replicas, one per GPU) ourselves
+        os.execv(sys.executable, launch_command(args.gpus, sys.argv[1:]))
     if args.impl == "reference":
         if args.steps == 200:
             args.steps = 5

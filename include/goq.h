@@ -138,7 +138,7 @@ goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16
 /* goq_gemm - the same layer for m activation rows.
  *  x_dtype GOQ_BF16: x [m][k_in] bf16; y out [m][n_out] (GOQ_BF16 or GOQ_F32); sx, cq, sc, acc unused (NULL).
  *      ws: goq_workspace_bytes(desc, GOQ_OP_GEMM, m) bytes, 256-byte aligned, initialised once with
- *      goq_workspace_init. From 49 rows on the tensor-core kernel runs: it keeps an fp16 copy of x
+ *      goq_workspace_init. From 33 rows on the tensor-core kernel runs: it keeps an fp16 copy of x
  *      (each row scaled by a power of two, undone in the output) in ws, so the size grows with m * k_in, and it
  *      rounds c1*b1 + c2*b2 once to fp16 (normwise output error about 1.5e-4; |c1*b1 + c2*b2| must stay below
  *      65504).

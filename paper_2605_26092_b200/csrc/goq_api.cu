@@ -11,7 +11,7 @@ namespace {
 
 std::atomic<int> g_gemv_variant{0};
 std::atomic<int> g_wait_limit{0};   // 0: the kernels' own bound on device-side waits
-constexpr int kGemmViaGemvMaxTokens = 48;
+constexpr int kGemmViaGemvMaxTokens = 32;   // above: the tcgen05 GEMM (split-K) is faster than 16-token GEMV launches
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -161,8 +161,8 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
         if (!y) return GOQ_ERR_INVALID_ARG;
         if (goq_status s = check_arch()) return s;
         const int variant = g_gemv_variant.load(std::memory_order_relaxed);
-        // Few tokens (17..48): the streaming GEMV kernel, 16 tokens per launch (36 us each on 8192 x 8192), against a
-        // tensor-core tile that is mostly padding (one 256-token half tile per CTA, measured below).
+        // Few tokens (17..32): the streaming GEMV kernel, 16 tokens per launch (36 us each on 8192 x 8192, so 72 us at
+        // 32 tokens), against ~89 us for the tensor-core kernel with split-K, which takes over from 33 tokens.
         if (m <= kGemmViaGemvMaxTokens && variant == 0 && goq::gemv_stream_supported(g)) {
             if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;
             if (ws_bytes < goq::gemv_stream_workspace(g)) return GOQ_ERR_WORKSPACE;
@@ -177,8 +177,8 @@ goq_status goq_gemm(const goq_desc* desc, const void* packed, const void* x, int
             }
             return GOQ_OK;
         }
-        // W4 has no streaming GEMV: up to 48 tokens its mma.sync kernel is the faster one (41 us at 16 tokens on
-        // 8192 x 8192 against ~105 us for a tensor-core half tile), so the tensor-core kernel takes W4 from 49 tokens on
+        // W4 has no streaming GEMV: up to 32 tokens its mma.sync kernel is the faster one (41 us at 16 tokens on
+        // 8192 x 8192 against ~92 us for the tensor-core kernel), so the tensor-core kernel takes W4 from 33 tokens on
         const bool w4_few = g.wbits == 4 && m <= kGemmViaGemvMaxTokens && variant == 0 && goq::linear_mma_supported(g);
         if (goq::gemm_tc_supported(g) && variant != 2 && !w4_few) {
             if (!ws || !aligned(ws, 256)) return ws ? GOQ_ERR_ALIGNMENT : GOQ_ERR_WORKSPACE;

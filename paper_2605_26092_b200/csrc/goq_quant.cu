@@ -34,15 +34,23 @@ __device__ __forceinline__ double lattice_value(int c, int wbits) {
     const double mag = __longlong_as_double((long long)(1023 - e) << 52);   // 2^-e
     return sg ? -mag : mag;
 }
-// nearest lattice state in linear distance; exact ties go to the state of smaller magnitude
+// Nearest lattice state in linear distance; exact ties go to the state of smaller magnitude. |v| <= 1. Between two
+// neighbouring magnitudes 2^E and 2^(E+1) the midpoint is 1.5 * 2^E, so the choice is read off the exponent field and the
+// top of the mantissa of |v|; below the smallest magnitude the neighbours are that state and zero. The positive side has
+// no +2^-emax (that bin is the zero): its smallest state is 2^-(emax-1), met by zero at the midpoint 2^-emax.
 __device__ __forceinline__ int rtn_code(double v, int wbits) {
-    int best = 0;
-    double bd = 1e300, bm = 1e300;
-    for (int c = 0; c < (1 << wbits); ++c) {
-        const double val = lattice_value(c, wbits), d = fabs(v - val), mg = fabs(val);
-        if (d < bd || (d == bd && mg < bm)) { bd = d; bm = mg; best = c; }
+    const int emax = (1 << (wbits - 1)) - 1;
+    const long long bits = __double_as_longlong(fabs(v));
+    const int E = (int)((bits >> 52) & 0x7FF) - 1023;                              // |v| = m 2^E, 1 <= m < 2
+    const bool upper = (bits & 0xFFFFFFFFFFFFFll) > (1ll << 51);                   // m > 1.5: the larger neighbour
+    const int e = -E - (upper ? 1 : 0);                                            // magnitude 2^-e
+    const double a = fabs(v);
+    if (v < 0.0) {
+        if (!(a > __longlong_as_double((long long)(1023 - emax - 1) << 52))) return emax;   // at or below 2^-(emax+1): zero
+        return (1 << (wbits - 1)) | min(e, emax);
     }
-    return best;
+    if (!(a > __longlong_as_double((long long)(1023 - emax) << 52))) return emax;           // at or below 2^-emax: zero
+    return min(e, emax - 1);
 }
 
 // b2 of the four elements a lane holds (elements 4*(lane&1) .. +3 of its micro-block) under record (s, flags):

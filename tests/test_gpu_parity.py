@@ -242,7 +242,7 @@ def test_gemm_bf16_small_full_parity(goq, n, k, g, b, m, variant):
     """Prefill GEMM, every output compared. variant 2: the two-operand mma.sync kernel, held to the tight bound.
     variant 0: from 65 tokens on the tcgen05 kernel, whose weight operand is w_hat rounded once to fp16: a relative
     error uniform in +-2^-12 per weight, rms 2^-12/sqrt(3) = 1.4e-4, independent between weights, so the normwise
-    output error is of that size; bound 5e-4. (Up to 48 tokens and group >= 32, variant 0 is the streaming GEMV: tight bound.)"""
+    output error is of that size; bound 5e-4. (Up to 32 tokens and group >= 32, variant 0 is the streaming GEMV: tight bound.)"""
     from tests.gpu_util import pack_weights, run_gemm_bf16
     codes, meta, coef = _quantized(n, k, g, b, seed=11 + n, outliers=True)
     d, packed = pack_weights(n, k, g, b, codes, meta, coef)
@@ -251,8 +251,8 @@ def test_gemm_bf16_small_full_parity(goq, n, k, g, b, m, variant):
     y = run_gemm_bf16(d, packed, xb, variant=variant)
     err = O.normwise_rel_err(y, y_ref)
     print("gemm variant %d: normwise error %.3e" % (variant, err))
-    # up to 48 tokens the streaming GEMV (W <= 3, group >= 32) or the exact mma.sync kernel (W4) takes the call
-    on_tc = variant == 0 and (m > 48 or (g < 32 and b <= 3))
+    # up to 32 tokens the streaming GEMV (W <= 3, group >= 32) or the exact mma.sync kernel (W4) takes the call
+    on_tc = variant == 0 and (m > 32 or (g < 32 and b <= 3))
     assert err <= TOL and err <= (GEMM_TC_TOL if on_tc else TIGHT), err
     from tests.gpu_util import elementwise_rel_err
     assert elementwise_rel_err(y, y_ref) <= (ELEM_TC if on_tc else ELEM_TIGHT)

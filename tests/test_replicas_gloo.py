@@ -49,3 +49,24 @@ def test_single_rank_needs_no_process_group():
     import bench
     ms_max, value = bench.aggregate_replicas(4.0, step_bytes=2 * 10 ** 9, world=1, device="cpu")
     assert ms_max == 4.0 and abs(value - 500.0) < 1e-9
+
+
+def test_gpus_flag_without_a_launcher_starts_one_rank_per_gpu():
+    """`bench.py --gpus N` with no WORLD_SIZE in the environment re-executes itself under torch.distributed.run with
+    N ranks on 127.0.0.1; the command keeps the caller's flags. The reference arm is used to run it for real on CPU:
+    rank 0 prints the line, the other rank exits 0 without work."""
+    import json
+    import subprocess
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.launch_command(4, ["--gpus", "4", "--steps", "7"], port=12345)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"]
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "4" and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[cmd.index("--master-port") + 1] == "12345" and cmd[-4:] == ["--gpus", "4", "--steps", "7"]
+    assert cmd[-5].endswith("bench.py")
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+                        "--warmup", "0"], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2
