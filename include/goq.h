@@ -138,10 +138,12 @@ goq_status goq_gemv(const goq_desc* desc, const void* packed, const void* x_bf16
 /* goq_gemm - the same layer for m activation rows.
  *  x_dtype GOQ_BF16: x [m][k_in] bf16; y out [m][n_out] (GOQ_BF16 or GOQ_F32); sx, cq, sc, acc unused (NULL).
  *      ws: goq_workspace_bytes(desc, GOQ_OP_GEMM, m) bytes, 256-byte aligned, initialised once with
- *      goq_workspace_init. From 33 rows on the tensor-core kernel runs: it keeps an fp16 copy of x
- *      (each row scaled by a power of two, undone in the output) in ws, so the size grows with m * k_in, and it
- *      rounds c1*b1 + c2*b2 once to fp16 (normwise output error about 1.5e-4; |c1*b1 + c2*b2| must stay below
- *      65504).
+ *      goq_workspace_init. From 33 rows on the tensor-core kernel runs: it keeps an fp16 copy of x (each row scaled by
+ *      a power of two, undone in the output) in ws, so the size grows with m * k_in, and it rounds c1*b1 + c2*b2 once
+ *      to fp16 (normwise output error about 1.5e-4 to 2.5e-4). The coefficients of every output channel are scaled by a
+ *      power of two taken from the channel's largest |c1|, |c2| before that rounding and the output is scaled back, so
+ *      the result does not depend on the magnitude of the weights; inside one channel, coefficients more than 2^13
+ *      below the channel's largest lose precision to fp16's range.
  *  x_dtype GOQ_I8 (Eq. 4 with integer X~ and c~; left shifts x~ << (emax-e), exact int32):
  *      x    [m][k_in] int8         sx [m] fp32 per-token scale
  *      cq   [n_out][k_in/group][2] int8 integer coefficients,  sc [n_out][2] fp32 their per-channel scales

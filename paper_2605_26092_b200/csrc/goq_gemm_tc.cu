@@ -20,7 +20,8 @@
 // the bf16 activations as fp16, each token scaled by the power of two that puts its largest magnitude in
 // [2^14, 2^15): bf16's 8 significant bits are kept exactly, and only elements more than 2^-28 below the
 // token's largest lose bits to fp16's range (they vanish below 2^-39 of it). The epilogue undoes the scale.
-// |w_hat| above 65504 overflows to infinity (coefficients that large do not occur: they scale fp16 weights).
+// The coefficients of every output channel are first multiplied by a power of two chosen from the channel's largest
+// coefficient (undone in the epilogue), so w_hat stays in fp16's normal range whatever the scale of the weights.
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, skips the remaining work,
 // still frees its tensor memory and records GOQ_ERR_TIMEOUT in the status word.
@@ -248,6 +249,8 @@ struct GemmParams {
     const uint8_t* packed;
     void* y;
     const float* inv_scale;   // [m_total] 2^-s of each token (the activations the tensor map covers are x * 2^s in fp16)
+    const uint32_t* row_scale;   // [n_pad] per-channel power of two for the coefficients, fp16 in both halves
+    const float* row_inv;        // [n_pad] its inverse
     int* status;
     int unit_bytes, meta_off, k_blocks, n_tiles, n_out, m_total, y_dtype, group_log2;
     // Tile schedule (1-D grid). CTAs [0, n_full) take 128 x 512 tiles, numbered channel-tile fastest; the remaining
@@ -284,6 +287,8 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
     uint64_t* epi_bar = bars + 11;      // [2] epilogue rendezvous of the four warps of a token half
     __shared__ uint32_t tmem_base_slot;
     __shared__ __align__(16) float inv_s[kTileM];   // 2^-s of this CTA's tokens (1 for tokens past the end)
+    __shared__ uint32_t row_s[kTileN];              // per-channel coefficient scale (fp16 x 2) of this CTA's 128 channels
+    __shared__ float row_i[kTileN];                 // ... and its inverse
     __shared__ volatile int abort_flag;
     __shared__ volatile int split_last;   // (split-K) this CTA completed its tile's counter
 
@@ -319,6 +324,11 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
         *reinterpret_cast<uint4*>(lut + (size_t)i * 16) = make_uint4(e[0], e[1], e[2], e[3]);
     }
     for (int i = tid; i < kTileM; i += kThreads) inv_s[i] = (tok0 + i < p.m_total) ? __ldg(&p.inv_scale[tok0 + i]) : 1.0f;
+    for (int i = tid; i < kTileN; i += kThreads) {
+        const bool in = T0 * kTileRows + i < p.n_tiles * kTileRows;
+        row_s[i] = in ? __ldg(&p.row_scale[T0 * kTileRows + i]) : 0x3C003C00u;   // 1.0
+        row_i[i] = in ? __ldg(&p.row_inv[T0 * kTileRows + i]) : 1.0f;
+    }
     if (warp == 1) tmem_alloc_512(&tmem_base_slot);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -388,6 +398,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
         const int e = warp - 2, g = lane >> 2, t = lane & 3;
         const uint32_t lut_lane = s32(lut) + (uint32_t)(lane & (kLutCopies - 1)) * 16;
         const bool valid = (T0 + e) < p.n_tiles;
+        const uint32_t rs_a = row_s[e * 16 + g], rs_b = row_s[e * 16 + 8 + g];   // scales of this lane's two channels
         constexpr uint32_t kZeroWord = (WB == 4) ? 0x77777777u : (WB == 3) ? 0x33333333u : 0x11111111u;  // every code = the zero state
         bool ok = true;
         for (int kb = 0; kb < nkb && ok; ++kb) {
@@ -419,8 +430,8 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                     const int jj = (c * 32 + t * 8) >> p.group_log2;  // macro-block of this micro-block inside the k-block
                     uint32_t cfa = 0u, cfb = 0u;   // {c1, c2} as stored: fp16 pairs
                     if (valid) {
-                        cfa = lds32(unit + kCodeBytesPerUnit + (jj * 16 + g) * 4);
-                        cfb = lds32(unit + kCodeBytesPerUnit + (jj * 16 + 8 + g) * 4);
+                        cfa = hmul2(lds32(unit + kCodeBytesPerUnit + (jj * 16 + g) * 4), rs_a);        // exact: a power of two
+                        cfb = hmul2(lds32(unit + kCodeBytesPerUnit + (jj * 16 + 8 + g) * 4), rs_b);
                     }
                     const uint32_t c1a = prmt(cfa, cfa, 0x1010u), c2a = prmt(cfa, cfa, 0x3232u);
                     const uint32_t c1b = prmt(cfb, cfb, 0x1010u), c2b = prmt(cfb, cfb, 0x3232u);
@@ -484,13 +495,14 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
                 const int col0 = col_half * 256 + cb * 32;
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)col0, v);
                 float* st = reinterpret_cast<float*>(b_tiles) + (col_half * 2 + (cb & 1)) * (32 * kTileN);
+                const float irs = row_i[q * 32 + lane];   // this lane's channel: undo the coefficient scale (a power of two)
 #pragma unroll
                 for (int j4 = 0; j4 < 8; ++j4) {   // the 32 tokens' inverse scales: eight broadcast 16-byte loads
                     const float4 f = *reinterpret_cast<const float4*>(&inv_s[col0 + 4 * j4]);
-                    st[(4 * j4 + 0) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 0]) * f.x;
-                    st[(4 * j4 + 1) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 1]) * f.y;
-                    st[(4 * j4 + 2) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 2]) * f.z;
-                    st[(4 * j4 + 3) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 3]) * f.w;
+                    st[(4 * j4 + 0) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 0]) * (f.x * irs);
+                    st[(4 * j4 + 1) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 1]) * (f.y * irs);
+                    st[(4 * j4 + 2) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 2]) * (f.z * irs);
+                    st[(4 * j4 + 3) * kTileN + q * 32 + lane] = __uint_as_float(v[4 * j4 + 3]) * (f.w * irs);
                 }
                 // bounded rendezvous of the half's four warps (a named barrier could not give up)
                 __syncwarp();
@@ -561,8 +573,40 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
 // xh[tok][k] = fp16(x[tok][k] * 2^s), inv_scale[tok] = 2^-s, s chosen from the exponent field of the token's largest
 // magnitude (an all-zero token gets the largest scale, harmlessly; inf / nan stay inf / nan).
 constexpr int kPrepThreads = 256;
+// Blocks beyond the tokens compute the per-channel scales of the weight operand, one 16-row tile each: w_hat is
+// formed in fp16, whose normal range ends at 2^-14, so every channel's coefficients are multiplied by the power of two
+// that puts the channel's largest |c1|, |c2| in [2^6, 2^7) (exact in fp16) and the epilogue divides it out again.
+// Coefficients down to 2^-13 of their channel's largest then keep full precision even times the smallest PoT state.
 __global__ void __launch_bounds__(kPrepThreads) x_to_f16_kernel(const uint16_t* __restrict__ x, int k_in, uint16_t* __restrict__ xh,
-                                                                float* __restrict__ inv_scale) {
+                                                                float* __restrict__ inv_scale, int m_total,
+                                                                const uint8_t* __restrict__ packed, int unit_bytes, int k_blocks,
+                                                                int groups_per_block, uint32_t* __restrict__ row_scale,
+                                                                float* __restrict__ row_inv) {
+    if ((int)blockIdx.x >= m_total) {
+        __shared__ uint32_t part_max[kPrepThreads / 16][16];
+        const int T = (int)blockIdx.x - m_total, r = threadIdx.x & 15, part = threadIdx.x >> 4;
+        uint32_t mx = 0;
+        for (int bk = part; bk < k_blocks; bk += kPrepThreads / 16) {
+            const uint32_t* cw = reinterpret_cast<const uint32_t*>(packed + ((size_t)T * k_blocks + bk) * unit_bytes + kCodeBytesPerUnit);
+            for (int jj = 0; jj < groups_per_block; ++jj) {
+                const uint32_t w = __ldg(&cw[jj * 16 + r]);
+                mx = max(mx, max(w & 0x7FFFu, (w >> 16) & 0x7FFFu));   // fp16 magnitudes order like their bit patterns
+            }
+        }
+        part_max[part][r] = mx;
+        __syncthreads();
+        if (threadIdx.x < 16) {
+            for (int q = 1; q < kPrepThreads / 16; ++q) mx = max(mx, part_max[q][r]);
+            int e = (int)(mx >> 10);                 // biased exponent of the largest coefficient (0: zero or subnormal)
+            if (e > 30) e = 30;                      // inf / nan coefficients: leave them alone
+            int shift = (mx == 0u) ? 0 : 21 - max(e, 1);   // 2^shift brings it to [2^6, 2^7)
+            shift = shift < -14 ? -14 : (shift > 15 ? 15 : shift);
+            const uint32_t h = (uint32_t)(15 + shift) << 10;
+            row_scale[T * 16 + r] = h | (h << 16);
+            row_inv[T * 16 + r] = __uint_as_float((uint32_t)(127 - shift) << 23);
+        }
+        return;
+    }
     const int tok = blockIdx.x, tid = threadIdx.x;
     const uint4* row = reinterpret_cast<const uint4*>(x + (size_t)tok * k_in);
     uint4* out = reinterpret_cast<uint4*>(xh + (size_t)tok * k_in);
@@ -641,11 +685,13 @@ static size_t smem_bytes(const Geometry& g) {
 
 template <int WB>
 static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* x, int m, void* y, int y_dtype, int* status,
-                             float* inv_scale, uint16_t* xh, int* tile_counter, float* partial, cudaStream_t st) {
+                             float* inv_scale, uint32_t* row_scale, float* row_inv, uint16_t* xh, int* tile_counter, float* partial,
+                             cudaStream_t st) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return cudaErrorNotSupported;
     if (g.k_in % 8 != 0) return cudaErrorInvalidValue;
-    x_to_f16_kernel<<<m, kPrepThreads, 0, st>>>((const uint16_t*)x, g.k_in, xh, inv_scale);
+    x_to_f16_kernel<<<m + g.n_tiles, kPrepThreads, 0, st>>>((const uint16_t*)x, g.k_in, xh, inv_scale, m, (const uint8_t*)packed,
+                                                           g.unit_bytes, g.k_blocks, g.groups_per_block, row_scale, row_inv);
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)g.k_in, (cuuint64_t)m};
     const cuuint64_t strides[1] = {(cuuint64_t)g.k_in * 2};
@@ -662,6 +708,8 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
     p.packed = (const uint8_t*)packed;
     p.y = y;
     p.inv_scale = inv_scale;
+    p.row_scale = row_scale;
+    p.row_inv = row_inv;
     p.status = status;
     p.unit_bytes = g.unit_bytes;
     p.meta_off = g.meta_off;
@@ -698,11 +746,13 @@ bool gemm_tc_supported(const Geometry& g) { return g.wbits <= 4 && g.k_in % 8 ==
 // copy of the activations and (split-K) the partial tiles.
 static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 namespace {
-struct TcScratch { size_t inv_off, xh_off, partial_off, total; };
+struct TcScratch { size_t inv_off, rs_off, ri_off, xh_off, partial_off, total; };
 TcScratch tc_scratch(const Geometry& g, int m) {
     TcScratch t;
     t.inv_off = kWsScratchOff;
-    t.xh_off = t.inv_off + align256((size_t)m * sizeof(float));
+    t.rs_off = t.inv_off + align256((size_t)m * sizeof(float));
+    t.ri_off = t.rs_off + align256((size_t)g.n_pad * sizeof(uint32_t));
+    t.xh_off = t.ri_off + align256((size_t)g.n_pad * sizeof(float));
     t.partial_off = align256(t.xh_off + (size_t)m * g.k_in * 2);
     const int split = tc::split_factor(g, m);
     const size_t tiles_x = (size_t)(g.n_pad + tc::kTileN - 1) / tc::kTileN;
@@ -717,11 +767,13 @@ cudaError_t launch_gemm_tc(const Geometry& g, const void* packed, const void* x,
     const TcScratch t = tc_scratch(g, m);
     uint8_t* b = (uint8_t*)ws;
     float* inv_scale = (float*)(b + t.inv_off);
+    uint32_t* rs = (uint32_t*)(b + t.rs_off);
+    float* ri = (float*)(b + t.ri_off);
     uint16_t* xh = (uint16_t*)(b + t.xh_off);
     int* counters = (int*)(b + kWsStatusBytes);   // at most sm_count / 2 tiles when the split is on
     float* partial = (float*)(b + t.partial_off);
-    if (g.wbits == 4) return tc::launch_wb<4>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, counters, partial, st);
-    return g.wbits == 3 ? tc::launch_wb<3>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, counters, partial, st)
-                        : tc::launch_wb<2>(g, packed, x, m, y, y_dtype, status, inv_scale, xh, counters, partial, st);
+    if (g.wbits == 4) return tc::launch_wb<4>(g, packed, x, m, y, y_dtype, status, inv_scale, rs, ri, xh, counters, partial, st);
+    return g.wbits == 3 ? tc::launch_wb<3>(g, packed, x, m, y, y_dtype, status, inv_scale, rs, ri, xh, counters, partial, st)
+                        : tc::launch_wb<2>(g, packed, x, m, y, y_dtype, status, inv_scale, rs, ri, xh, counters, partial, st);
 }
 }  // namespace goq

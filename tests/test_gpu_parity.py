@@ -276,6 +276,29 @@ def test_config4_prefill_2048_tokens_sampled_rows(goq, n, k):
     print("M=2048 %dx%d: normwise %.3e element-wise %.3e" % (n, k, nerr, eerr))
 
 
+@pytest.mark.parametrize("b", [3, 4])
+def test_gemm_small_and_mixed_weight_magnitudes(goq, b):
+    """The tcgen05 GEMM forms w_hat in fp16. Weights of standard deviation 2e-2 .. 1.2e-6 (coefficients down into fp16's
+    subnormal range) and a layer whose channels differ by 2^12 in scale must all come out at the kernel's usual accuracy:
+    every channel's coefficients are scaled by a power of two before w_hat is formed and the epilogue undoes it."""
+    from tests.gpu_util import pack_weights, run_gemm_bf16, check_parity
+    n, k, g, m = 256, 1024, 128, 200
+    xb = si.bf16_activations(m, k, seed=6)
+    for exp in (0, -8, -12, -14):
+        w = si.gaussian_weights(n, k, seed=5) * 2.0 ** exp
+        if exp == -8:
+            w[::3] *= 2.0 ** -12   # channels of very different scale inside one 128-channel tile
+        codes, meta, coef = O.quantize_geo(w, g, b)
+        d, packed = pack_weights(n, k, g, b, codes, meta, coef)
+        y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), g, b)
+        y = run_gemm_bf16(d, packed, xb)
+        # per channel: a channel 2^12 below its neighbours must be as accurate as they are
+        err = np.linalg.norm(y - y_ref, axis=0) / np.maximum(np.linalg.norm(y_ref, axis=0), 1e-300)
+        live = np.linalg.norm(y_ref, axis=0) > 0
+        assert np.max(err[live]) <= 4 * GEMM_TC_TOL, (exp, float(np.max(err[live])))
+        assert O.normwise_rel_err(y, y_ref) <= GEMM_TC_TOL, (exp, O.normwise_rel_err(y, y_ref))
+
+
 def test_gemm_token_scaling_extreme_activations(goq):
     """The tcgen05 GEMM feeds fp16 activations scaled per token by a power of two. Tokens of very different
     magnitude (2^100, 2^-100), an all-zero token, a token whose elements span 2^24 and one with many zeros must
