@@ -529,44 +529,58 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
 #pragma unroll
         for (int cg = 0; cg < NG; ++cg) acc[cg][0] = acc[cg][1] = 0.f;
         const unsigned n_full = wk.L / kStageRecs, n_tail = wk.L - n_full * kStageRecs;
-        unsigned st = 0;                                                                     // next full stage
-        unsigned u = (unsigned)warp * 4u * n_tail / kNW;                                     // next chunk of the tail stage
         const unsigned u1 = (unsigned)(warp + 1) * 4u * n_tail / kNW;
+        unsigned u = (unsigned)warp * 4u * n_tail / kNW;                                     // next chunk of the tail stage
         bool tail_open = false;
-        for (;;) {
-            // ---- the next piece of work of this warp: where it is in the walk, which tile part it belongs to ----
-            const bool in_full = st < n_full, in_tail = !in_full && u < u1;
-            unsigned rho = 0;
-            int T = 0, kbi = 0, qn = wk.P;
-            if (in_full || in_tail) {
-                rho = walk_record(wk, in_full ? st * kStageRecs + warp : n_full * kStageRecs + (u >> 2));
-                T = (int)(((unsigned long long)rho * it.kb_magic) >> 32);
-                kbi = (int)(rho - (unsigned)T * (unsigned)kb);
-                qn = walk_part_of_tile(wk, T);
-            }
-            for (; cur_q < qn; ++cur_q) {   // parts this warp has passed (or never touched: zeros) are handed over
+        // hand over the parts this warp has passed (or never touched: zeros) up to part qn
+        auto flush_to = [&](int qn) {
+            for (; cur_q < qn && alive; ++cur_q) {
                 Sums4 sums;
 #pragma unroll
                 for (int cg = 0; cg < 2; ++cg) { sums.v[2 * cg] = cg < NG ? acc[cg < NG ? cg : 0][0] : 0.f; sums.v[2 * cg + 1] = cg < NG ? acc[cg < NG ? cg : 0][1] : 0.f; }
-                if (!flush_part<NG>(fc, seq + (unsigned)cur_q, sums)) { alive = false; break; }
+                if (!flush_part<NG>(fc, seq + (unsigned)cur_q, sums)) alive = false;
 #pragma unroll
                 for (int cg = 0; cg < NG; ++cg) acc[cg][0] = acc[cg][1] = 0.f;
             }
-            if (!alive) break;
-            if (in_full) {
-                // stages in a row in which this warp's record stays inside tile T and on this side of the turn of the walk
-                const unsigned j = st * kStageRecs + warp;
+        };
+        // ---- full stages: record st*16 + warp of the walk. Its tile, k-block and part are found once and then carried
+        //      along (16 records further each stage); only the turn of the walk needs them found again ----
+        {
+            unsigned st = 0, j = (unsigned)warp;
+            int kbi = 0, q = 0;
+            bool locate = true;
+            while (st < n_full && alive) {
+                if (locate) {
+                    const unsigned rho = walk_record(wk, j);
+                    const int T = (int)(((unsigned long long)rho * it.kb_magic) >> 32);
+                    kbi = (int)(rho - (unsigned)T * (unsigned)kb);
+                    q = walk_part_of_tile(wk, T);
+                    locate = false;
+                }
+                if (cur_q < q) flush_to(q);
+                if (!alive) break;
+                // stages in a row in which this warp's record stays inside its tile and on this side of the turn of the walk
                 unsigned run = ((unsigned)(kb - kbi) + kStageRecs - 1) / kStageRecs;
-                if (j < wk.L1) run = min(run, (wk.L1 - j + kStageRecs - 1) / kStageRecs);
+                const bool before_turn = j < wk.L1;
+                if (before_turn) run = min(run, (wk.L1 - j + kStageRecs - 1) / kStageRecs);
                 run = min(run, n_full - st);
                 st += run;
+                j += run * kStageRecs;
+                if (before_turn && j >= wk.L1) locate = true;   // the next record lies beyond the turn
                 // ================= the hot loop: one record per iteration =================
                 uint32_t koff = (uint32_t)kbi * kBlockK, ksc = (uint32_t)kbi * (16 * NG);
                 kbi += (int)run * kStageRecs;
                 for (; run; --run, koff += kStageRecs * kBlockK, ksc += kStageRecs * 16 * NG) {
-                    if (!try_wait_a(full_addr + bar_off, phase) && !wait_slow_a(full_addr + bar_off, phase, &abort_flag, spin)) {
-                        alive = false;   // give up after this iteration (whatever it computes is never stored)
-                        run = 1;
+                    {   // bounded wait for the stage, written out so that the record loop contains no call
+                        int polls = 0;
+                        while (!try_wait_a(full_addr + bar_off, phase)) {
+                            if (++polls >= spin || ((polls & 255) == 0 && abort_flag)) {
+                                abort_flag = 1;
+                                alive = false;   // give up after this iteration (whatever it computes is never stored)
+                                run = 1;
+                                break;
+                            }
+                        }
                     }
                     const uint32_t unit = order_after_wait(unit0 + stage_off);
                     const uint4 wv0 = lds128(unit), wv1 = lds128(unit + 512);
@@ -607,9 +621,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                     stage_off += (uint32_t)stage_bytes; bar_off += 8;
                     if (++slot == p.n_stages) { slot = 0; phase ^= 1; stage_off = 0; bar_off = 0; }
                 }
+                // the next record is 16 further in the same linear order: it has left the tile (that is why the run ended,
+                // unless the stages ran out); a tile narrower than a stage may be skipped altogether
+                while (kbi >= kb) { kbi -= kb; ++q; }
+            }
+        }
+        // ---- the last stage of the range: chunks cb..ce-1 of one record per step ----
+        while (u < u1 && alive) {
+            {
+                const unsigned rho = walk_record(wk, n_full * kStageRecs + (u >> 2));
+                const int T = (int)(((unsigned long long)rho * it.kb_magic) >> 32);
+                const int kbi = (int)(rho - (unsigned)T * (unsigned)kb);
+                flush_to(walk_part_of_tile(wk, T));
                 if (!alive) break;
-            } else if (in_tail) {
-                // ---- the last stage of the range: chunks cb..ce-1 of one record ----
                 if (!tail_open) {
                     if (!wait_bar(&full_bar[slot], phase, &abort_flag, spin)) { alive = false; break; }
                     tail_open = true;
@@ -648,10 +672,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                     acc[cg][1] = fmaf(sv, rec[cg][1], acc[cg][1]);
                 }
                 u += ce - cb;
-            } else {
-                break;   // every part has been handed over
             }
         }
+        flush_to(wk.P);   // every part has been handed over
         if (!alive) break;
         if (n_tail) {   // every warp takes part in the tail stage's hand-shake, with or without chunks of its own
             if (!tail_open && !wait_bar(&full_bar[slot], phase, &abort_flag, spin)) { alive = false; break; }
