@@ -50,6 +50,10 @@ struct Item {
     unsigned long long kb_magic;             // ceil(2^32 / k_blocks): record number -> tile by multiply and shift (exact while units * k_blocks < 2^32)
     unsigned int units;                      // n_tiles * k_blocks
     int n_tiles, k_blocks, k_in, n_out, m, y_dtype, depends;
+    int xsrc;                                // earlier item whose output this item's x lies in (read from that item's tagged copy), or -1
+    unsigned int xoff;                       // first 64-bit word of x inside that copy
+    int tag_out;                             // a later item reads this item's output: keep the tagged copy
+    int pad_;
 };
 struct Params {
     Item item[kSeqMaxItems];
@@ -58,9 +62,12 @@ struct Params {
     int* done;       // [n_items] CTAs that have finished each linear; zero on entry, left zero
     unsigned* epoch; // launches this scratch buffer has seen: tags the posted parts (zero-filled scratch carries no valid tag)
     uint2* parts;    // [n_items][G][2][32 lanes x 2 NG] posted partial sums, each value in one 64-bit word with its tag
+    uint2* tags;     // [n_items][kTagWords] tagged copies of bf16 outputs: [token][16 n_tiles / 2] words of (two values, tag)
 };
 
 constexpr int kPartWords = 128;              // 64-bit (value, tag) words of one posted part: 16 rows x 8 tokens
+constexpr int kTagWords = 4 * (kMaxKBlocks * kBlockK / 2);   // per item: four tokens of the widest input a linear can take
+constexpr int kXBatch = 3;                   // 16-byte activation chunks a lane holds while it polls their tags
 
 // ---- small helpers ---------------------------------------------------------------------------------
 template <int WB> struct IntTables;
@@ -152,8 +159,10 @@ struct Walk {
 };
 __device__ __forceinline__ Walk make_walk(const Item& it, int cta, int G) {
     Walk w;
-    w.a = (unsigned)((unsigned long long)it.units * (unsigned)cta / (unsigned)G);
-    w.b = (unsigned)((unsigned long long)it.units * (unsigned)(cta + 1) / (unsigned)G);
+    // floor(units c / G) = c (units / G) + floor(c (units % G) / G): 32-bit arithmetic (c (units % G) < G^2)
+    const unsigned uq = it.units / (unsigned)G, ur = it.units % (unsigned)G;
+    w.a = (unsigned)cta * uq + (unsigned)cta * ur / (unsigned)G;
+    w.b = (unsigned)(cta + 1) * uq + (unsigned)(cta + 1) * ur / (unsigned)G;
     w.L = w.b - w.a;
     w.L1 = 0; w.s1 = 0; w.Ta = 0; w.Tb = 0; w.P = 0; w.rot = false;
     if (w.L) {
@@ -169,11 +178,6 @@ __device__ __forceinline__ Walk make_walk(const Item& it, int cta, int G) {
 __device__ __forceinline__ unsigned walk_record(const Walk& w, unsigned j) { return j < w.L1 ? w.s1 + j : w.a + (j - w.L1); }
 __device__ __forceinline__ int walk_part_of_tile(const Walk& w, int T) { return w.rot ? (T == w.Tb ? 0 : 1 + T - w.Ta) : T - w.Ta; }
 __device__ __forceinline__ int walk_tile_of_part(const Walk& w, int q) { return w.rot ? (q == 0 ? w.Tb : w.Ta + q - 1) : w.Ta + q; }
-
-// CTA that owns record r of a linear with `units` records split over G CTAs
-__device__ __forceinline__ int owner_of(unsigned long long r, unsigned units, int G) {
-    return (int)(((r + 1) * (unsigned)G - 1) / units);
-}
 
 // ---- hand-over of one tile part (kept out of line) ------------------------------------------------------
 // A consumer warp parks its sums of part number sq (counted per CTA over the whole chain) in reduction slot sq % kTileSlots
@@ -331,54 +335,48 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                     __syncwarp();
                     if (abort_flag) { ok = false; break; }
                 }
-                const int kb = it.k_blocks;
+                // The control warp is alone on the critical path between the last arithmetic of a tile and the SMs that wait
+                // for its outputs, and a lone warp runs at instruction latency: whatever does not need the sums (which tile, who
+                // finishes it, every address) is worked out BEFORE the wait for the part, and nothing on the far side divides.
+                const unsigned kb = (unsigned)it.k_blocks;
+                const unsigned uq = it.units / (unsigned)G, ur = it.units % (unsigned)G;   // range boundaries step by uq (+1) from CTA to CTA
+                const unsigned rem_a = ((unsigned)cta * ur) % (unsigned)G;
+                const int tok0 = lane & 3;
+                const size_t tstride4 = (size_t)4 * (it.n_tiles * 8), ystride4 = (size_t)4 * it.n_out;
+                const bool y32 = it.y_dtype == GOQ_F32;
+                bool tokv[NG];
+#pragma unroll
+                for (int cg = 0; cg < NG; ++cg) tokv[cg] = cg * 4 + tok0 < it.m;
+                const bool tagw = it.tag_out && (lane & 4) == 0;
                 for (int q = 0; q < wk.P; ++q) {
                     const unsigned sq = seq + (unsigned)q;
                     const int rs = (int)(sq % kTileSlots);
-                    if (!wait_bar(&part_bar[rs], (sq / kTileSlots) & 1u, &abort_flag, spin)) { ok = false; break; }
-                    const float* rall = red + (size_t)rs * kNW * (NG * 64);
-                    float out[NG][2];
-#pragma unroll
-                    for (int cg = 0; cg < NG; ++cg)
-#pragma unroll
-                        for (int hh = 0; hh < 2; ++hh) {
-                            float v[kNW];
-#pragma unroll
-                            for (int w2 = 0; w2 < kNW; ++w2) v[w2] = rall[(size_t)w2 * (NG * 64) + cg * 64 + hh * 32 + lane];
-                            float sum = 0.f;
-#pragma unroll
-                            for (int w2 = 0; w2 < kNW; ++w2) sum += v[w2];   // warp order
-                            out[cg][hh] = sum;
-                        }
-                    __syncwarp();
-                    if (lane == 0) done_gen[rs] = (int)(sq + 1);   // the slot may be parked in again
                     const int T = walk_tile_of_part(wk, q);
-                    const unsigned long long r_lo = (unsigned long long)T * (unsigned)kb, r_hi = r_lo + (unsigned)kb;
-                    bool store = r_lo >= wk.a && r_hi <= wk.b;
-                    if (!store) {
-                        const int c_first = owner_of(r_lo, it.units, G), c_last = owner_of(r_hi - 1, it.units, G);
-                        // The CTA that holds the end of the tile finishes it; the others post their part and go on. A posted
-                        // value travels in one 64-bit word with the launch's tag, so it needs no fence and no counter: the
-                        // finisher reads the words until the tag is there. Every CTA walks its range starting with the tile
-                        // that is open at the range's end, so the posted parts are early, and the finisher waits only on
-                        // lower-numbered CTAs (no cycle).
-                        if (cta != c_last) {
-                            uint2* mine = p.parts + (((size_t)i * G + cta) * 2 + (T == wk.Ta ? 0 : 1)) * kPartWords;
+                    const unsigned r_lo = (unsigned)T * kb, r_hi = r_lo + kb;
+                    const bool whole = r_lo >= wk.a && r_hi <= wk.b;   // every record of the tile is this CTA's
+                    const bool finisher = r_hi <= wk.b;                  // this CTA holds the tile's end
+                    uint2* post = p.parts + (((size_t)i * G + cta) * 2 + (T == wk.Ta ? 0 : 1)) * kPartWords + lane;
+                    uint2* tgp = p.tags + (size_t)i * kTagWords + (size_t)tok0 * (it.n_tiles * 8) + T * 8 + (lane >> 3);
+                    const size_t yoff = (size_t)tok0 * it.n_out + T * 16 + (lane >> 2);
+                    bool rowv[2];
+                    rowv[0] = T * 16 + (lane >> 2) < it.n_out;
+                    rowv[1] = T * 16 + (lane >> 2) + 8 < it.n_out;
+                    const float* rall = red + (size_t)rs * kNW * (NG * 64) + lane;
+                    // A tile this CTA finishes for others: their parts were posted early (every CTA starts with the tile that is
+                    // open at the end of its range), so they are fetched now, before this CTA's own sums are ready - nearest CTA
+                    // first, down to the one that holds the tile's first record.
+                    float below[NG][2];
 #pragma unroll
-                            for (int cg = 0; cg < NG; ++cg)
-#pragma unroll
-                                for (int hh = 0; hh < 2; ++hh)
-                                    asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(mine + (cg * 2 + hh) * 32 + lane),
-                                                 "r"(__float_as_uint(out[cg][hh])), "r"(tag) : "memory");
-                        } else {
-                            float sum[NG][2];
-#pragma unroll
-                            for (int cg = 0; cg < NG; ++cg) sum[cg][0] = sum[cg][1] = 0.f;
-                            bool good = true;
-                            for (int cc = c_first; cc < c_last && good; ++cc) {   // CTA order; this CTA's own part comes last
-                                const unsigned ac = (unsigned)((unsigned long long)it.units * (unsigned)cc / (unsigned)G);
-                                if (ac == (unsigned)((unsigned long long)it.units * (unsigned)(cc + 1) / (unsigned)G)) continue;   // empty range
-                                const uint2* pc = p.parts + (((size_t)i * G + cc) * 2 + ((int)(ac / (unsigned)kb) == T ? 0 : 1)) * kPartWords;
+                    for (int cg = 0; cg < NG; ++cg) below[cg][0] = below[cg][1] = 0.f;
+                    if (!whole && finisher) {
+                        bool good = true;
+                        unsigned bc = wk.a, remc = rem_a;   // upper boundary of CTA cc's range (= lower boundary of CTA cc + 1)
+                        for (int cc = cta - 1; cc >= 0 && bc > r_lo && good; --cc) {
+                            const unsigned borrow = remc < ur ? 1u : 0u;
+                            const unsigned ac = bc - uq - borrow;
+                            remc = remc - ur + (borrow ? (unsigned)G : 0u);
+                            if (ac != bc) {   // CTA cc has records of this tile; they are its first tile's if its range starts inside
+                                const uint2* pc = p.parts + (((size_t)i * G + cc) * 2 + (ac >= r_lo ? 0 : 1)) * kPartWords + lane;
                                 int spins = 0;
                                 for (;;) {
                                     uint2 w[NG][2];
@@ -388,34 +386,72 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
 #pragma unroll
                                         for (int hh = 0; hh < 2; ++hh) {
                                             asm volatile("ld.relaxed.gpu.global.v2.u32 {%0, %1}, [%2];" : "=r"(w[cg][hh].x), "=r"(w[cg][hh].y)
-                                                         : "l"(pc + (cg * 2 + hh) * 32 + lane) : "memory");
+                                                         : "l"(pc + (cg * 2 + hh) * 32) : "memory");
                                             all = all && w[cg][hh].y == tag;
                                         }
                                     if (__all_sync(0xFFFFFFFFu, all)) {
 #pragma unroll
-                                        for (int cg = 0; cg < NG; ++cg) { sum[cg][0] += __uint_as_float(w[cg][0].x); sum[cg][1] += __uint_as_float(w[cg][1].x); }
+                                        for (int cg = 0; cg < NG; ++cg) { below[cg][0] += __uint_as_float(w[cg][0].x); below[cg][1] += __uint_as_float(w[cg][1].x); }
                                         break;
                                     }
-                                    if (abort_flag || ++spins > kGlobalSpin || spins > spin) { abort_flag = 1; good = false; break; }
+                                    ++spins;
+                                    if (__any_sync(0xFFFFFFFFu, abort_flag != 0) || spins > kGlobalSpin || spins > spin) { abort_flag = 1; good = false; break; }
                                 }
                             }
-                            if (!good) { ok = false; break; }
-#pragma unroll
-                            for (int cg = 0; cg < NG; ++cg) { out[cg][0] += sum[cg][0]; out[cg][1] += sum[cg][1]; }
-                            store = true;
+                            bc = ac;
                         }
+                        if (!good) { ok = false; break; }
                     }
-                    if (store) {
+                    if (!wait_bar(&part_bar[rs], (sq / kTileSlots) & 1u, &abort_flag, spin)) { ok = false; break; }
+                    float out[NG][2];
+#pragma unroll
+                    for (int cg = 0; cg < NG; ++cg)
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            float v[kNW];
+#pragma unroll
+                            for (int w2 = 0; w2 < kNW; ++w2) v[w2] = rall[(size_t)w2 * (NG * 64) + cg * 64 + hh * 32];
+#pragma unroll
+                            for (int sft = kNW / 2; sft >= 1; sft >>= 1)   // fixed pairing: deterministic
+#pragma unroll
+                                for (int w2 = 0; w2 < sft; ++w2) v[w2] += v[w2 + sft];
+                            out[cg][hh] = v[0] + below[cg][hh];
+                        }
+                    __syncwarp();
+                    if (lane == 0) done_gen[rs] = (int)(sq + 1);   // every lane has read the slot: it may be parked in again
+                    if (!whole && !finisher) {
+                        // The CTA that holds the end of the tile finishes it; the others post their part and go on. A posted
+                        // value travels in one 64-bit word with the launch's tag, so it needs no fence and no counter: the
+                        // finisher reads the words until the tag is there, and it waits only on lower-numbered CTAs (no cycle).
+#pragma unroll
+                        for (int cg = 0; cg < NG; ++cg)
+#pragma unroll
+                            for (int hh = 0; hh < 2; ++hh)
+                                asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(post + (cg * 2 + hh) * 32),
+                                             "r"(__float_as_uint(out[cg][hh])), "r"(tag) : "memory");
+                    } else {
+                        // A later item reads this output: first the copy it polls. Two neighbouring channels (bf16, as in y)
+                        // and the launch's tag share one 64-bit word, so a reader that sees the tag has the values - no fence
+                        // and no counter between the finisher of a tile and the SMs that wait for it.
+                        uint32_t pair[NG][2];
 #pragma unroll
                         for (int cg = 0; cg < NG; ++cg)
 #pragma unroll
                             for (int hh = 0; hh < 2; ++hh) {
-                                const int row = T * 16 + hh * 8 + (lane >> 2), tok = cg * 4 + (lane & 3);
-                                if (row < it.n_out && tok < it.m) {
-                                    if (it.y_dtype == GOQ_F32) reinterpret_cast<float*>(it.y)[(size_t)tok * it.n_out + row] = out[cg][hh];
-                                    else reinterpret_cast<uint16_t*>(it.y)[(size_t)tok * it.n_out + row] = f32_to_bf16_rne(out[cg][hh]);
-                                }
+                                const float next = __shfl_down_sync(0xFFFFFFFFu, out[cg][hh], 4);   // channel + 1 of the same token
+                                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pair[cg][hh]) : "f"(next), "f"(out[cg][hh]));
+                                if (tagw && tokv[cg])
+                                    asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(tgp + cg * tstride4 + hh * 4), "r"(pair[cg][hh]), "r"(tag) : "memory");
                             }
+#pragma unroll
+                        for (int cg = 0; cg < NG; ++cg)
+#pragma unroll
+                            for (int hh = 0; hh < 2; ++hh)
+                                if (rowv[hh] && tokv[cg]) {
+                                    const size_t o = yoff + cg * ystride4 + hh * 8;
+                                    if (y32) reinterpret_cast<float*>(it.y)[o] = out[cg][hh];
+                                    else reinterpret_cast<uint16_t*>(it.y)[o] = (uint16_t)(pair[cg][hh] & 0xFFFFu);   // the bits the copy carries
+                                }
                     }
                 }
                 if (!ok) break;
@@ -451,6 +487,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
     int x_sel = 0;                    // activation buffer of the current linear
     unsigned seq = 0;                 // tile parts this CTA has opened so far (same in every warp): indexes the reduction slots
     bool alive = true;
+    const unsigned tag = ((*p.epoch + 1u) * 0x9E3779B1u) | 1u;   // as in the control warp: the count changes only when every CTA is done
 
     for (int i = 0; i < p.n_items && alive; ++i) {
         const Item& it = p.item[i];
@@ -460,6 +497,23 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
         if (p.x_double) x_sel ^= 1;
         unsigned char* xb = xq + (size_t)x_sel * p.xbuf_bytes;
         float* xsc = xscale + x_sel * (kMaxKBlocks * 4 * NG);
+
+        // The last stage of the range, n_tail < 16 records: 16 / n_tail warps share each record, each warp a run of its four
+        // 32-wide chunks (the sums are linear in the chunks), so that no warp visits more than one record. Which record, which
+        // chunks, its k-block and tile part are worked out here, ahead of the dependency wait (divisions).
+        const unsigned n_full = wk.L / kStageRecs, n_tail = wk.L - n_full * kStageRecs;
+        unsigned tail_desc = 0;   // [0:4) record of the stage, [4:7) first chunk, [7:10) end chunk, [10:17) k-block, [17:32) tile part
+        if (n_tail) {
+            const unsigned wpr = (unsigned)kNW / n_tail;   // >= 1
+            const unsigned rloc = (unsigned)warp / wpr, sub = (unsigned)warp - rloc * wpr;
+            const unsigned cb = 4u * sub / wpr, ce = 4u * (sub + 1u) / wpr;
+            if (rloc < n_tail && cb < ce) {
+                const unsigned rho = walk_record(wk, n_full * kStageRecs + rloc);
+                const unsigned T = (unsigned)(((unsigned long long)rho * it.kb_magic) >> 32);
+                const unsigned kbi = rho - T * (unsigned)kb;
+                tail_desc = rloc | (cb << 4) | (ce << 7) | (kbi << 10) | ((unsigned)walk_part_of_tile(wk, (int)T) << 17);
+            }
+        }
 
         // ---- start of the linear: wait for the dependency, then every warp converts its slice of the activations ----
         if (it.depends && i > 0) {
@@ -474,12 +528,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
         {
             // 16-byte chunks of 8 bf16; 16 chunks = one k-block of one token: Q = rne(x 2^s), the block's largest magnitude in [2^14, 2^15)
             const int cpt = k_pad / 8, total = cpt * m;
-            for (int c0 = warp * 32; c0 < total; c0 += kNW * 32) {
-                const int c = c0 + lane;
-                const bool in = c < total;
-                const int r = in ? c / cpt : 0, k0 = in ? (c - r * cpt) * 8 : 0;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (in && k0 < it.k_in) v = __ldcg(reinterpret_cast<const uint4*>(it.x + (size_t)r * it.k_in + k0));   // L2: written by other SMs
+            auto convert = [&](const uint4 v, const bool in, const int r, const int k0) {
                 const uint32_t in32[4] = {v.x, v.y, v.z, v.w};
                 uint32_t amax = 0;
 #pragma unroll
@@ -506,6 +555,66 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                     // 2^-s, and 2^-emax for the integer weights
                     if ((lane & 15) == 0) xsc[(k0 >> 7) * (4 * NG) + r] = __uint_as_float((uint32_t)(254 - sfield) << 23) * (1.0f / (float)(1 << ((1 << (WB - 1)) - 1)));
                 }
+            };
+            if (it.xsrc < 0) {   // activations from outside the chain, or ordered by the counter wait above
+                for (int c0 = warp * 32; c0 < total; c0 += kNW * 32) {
+                    const int c = c0 + lane;
+                    const bool in = c < total;
+                    const int r = in ? c / cpt : 0, k0 = in ? (c - r * cpt) * 8 : 0;
+                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                    if (in && k0 < it.k_in) v = __ldcg(reinterpret_cast<const uint4*>(it.x + (size_t)r * it.k_in + k0));   // L2: written by other SMs
+                    convert(v, in, r, k0);
+                }
+            } else {
+                // Activations that an earlier linear of this launch produces: read from its tagged copy, word by word,
+                // until every word carries this launch's tag. That is the whole dependency wait: a chunk is converted as soon
+                // as the tiles it comes from are finished, wherever they were finished.
+                const uint2* tg = p.tags + (size_t)it.xsrc * kTagWords + it.xoff;
+                const int tstride = p.item[it.xsrc].n_tiles * 8;
+                const int bound = spin < kGlobalSpin ? spin : kGlobalSpin;
+                for (int cb = warp * 32; cb < total && alive; cb += kNW * 32 * kXBatch) {
+                    uint4 v[kXBatch];
+                    bool need[kXBatch];
+#pragma unroll
+                    for (int u = 0; u < kXBatch; ++u) {
+                        const int c = cb + u * (kNW * 32) + lane;
+                        const int r = c < total ? c / cpt : 0, k0 = c < total ? (c - r * cpt) * 8 : 0;
+                        need[u] = c < total && k0 < it.k_in;
+                        v[u] = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                    int spins = 0;
+                    for (;;) {
+                        bool ok = true;
+#pragma unroll
+                        for (int u = 0; u < kXBatch; ++u)
+                            if (need[u]) {
+                                const int c = cb + u * (kNW * 32) + lane;
+                                const int r = c / cpt, k0 = (c - r * cpt) * 8;
+                                const uint2* src = tg + (size_t)r * tstride + (k0 >> 1);
+                                unsigned long long w0, w1, w2, w3;
+                                asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(src) : "memory");
+                                asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(w2), "=l"(w3) : "l"(src + 2) : "memory");
+                                if ((unsigned)(w0 >> 32) == tag && (unsigned)(w1 >> 32) == tag && (unsigned)(w2 >> 32) == tag && (unsigned)(w3 >> 32) == tag) {
+                                    v[u] = make_uint4((unsigned)w0, (unsigned)w1, (unsigned)w2, (unsigned)w3);
+                                    need[u] = false;
+                                } else {
+                                    ok = false;
+                                }
+                            }
+                        if (__all_sync(0xFFFFFFFFu, ok)) break;
+                        ++spins;
+                        if (__any_sync(0xFFFFFFFFu, abort_flag != 0) || spins > bound) { abort_flag = 1; alive = false; break; }   // the whole warp or nobody
+                    }
+                    if (!alive) break;
+#pragma unroll
+                    for (int u = 0; u < kXBatch; ++u) {
+                        const int c = cb + u * (kNW * 32) + lane;
+                        const bool in = c < total;
+                        const int r = in ? c / cpt : 0, k0 = in ? (c - r * cpt) * 8 : 0;
+                        if (cb + u * (kNW * 32) < total) convert(v[u], in, r, k0);   // warp-uniform: the conversion shuffles
+                    }
+                }
+                if (!alive) break;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(x_bar);
@@ -528,9 +637,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
         float acc[NG][2];
 #pragma unroll
         for (int cg = 0; cg < NG; ++cg) acc[cg][0] = acc[cg][1] = 0.f;
-        const unsigned n_full = wk.L / kStageRecs, n_tail = wk.L - n_full * kStageRecs;
-        const unsigned u1 = (unsigned)(warp + 1) * 4u * n_tail / kNW;
-        unsigned u = (unsigned)warp * 4u * n_tail / kNW;                                     // next chunk of the tail stage
         bool tail_open = false;
         // hand over the parts this warp has passed (or never touched: zeros) up to part qn
         auto flush_to = [&](int qn) {
@@ -626,52 +732,53 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 while (kbi >= kb) { kbi -= kb; ++q; }
             }
         }
-        // ---- the last stage of the range: chunks cb..ce-1 of one record per step ----
-        while (u < u1 && alive) {
-            {
-                const unsigned rho = walk_record(wk, n_full * kStageRecs + (u >> 2));
-                const int T = (int)(((unsigned long long)rho * it.kb_magic) >> 32);
-                const int kbi = (int)(rho - (unsigned)T * (unsigned)kb);
-                flush_to(walk_part_of_tile(wk, T));
-                if (!alive) break;
-                if (!tail_open) {
-                    if (!wait_bar(&full_bar[slot], phase, &abort_flag, spin)) { alive = false; break; }
+        // ---- the last stage of the range: this warp's chunks of its record, if it has any ----
+        if (n_tail && alive) {
+            const unsigned rloc = tail_desc & 15u, cb = (tail_desc >> 4) & 7u, ce = (tail_desc >> 7) & 7u;
+            if (cb < ce) {
+                const int kbi = (int)((tail_desc >> 10) & 127u);
+                flush_to((int)(tail_desc >> 17));
+                if (alive && !wait_bar(&full_bar[slot], phase, &abort_flag, spin)) alive = false;
+                if (alive) {
                     tail_open = true;
-                }
-                const unsigned rloc = u >> 2, cb = u & 3u, ce = min(4u, cb + (u1 - u));
-                const uint32_t unit = order_after_wait(ring_addr + slot * stage_bytes + rloc * unit_bytes + lane * 16);
-                const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
-                int s1[NG][4], s2[NG][4], s3[NG][4];
-                float rec[NG][2];
-#pragma unroll
-                for (int cg = 0; cg < NG; ++cg) {
-                    rec[cg][0] = rec[cg][1] = 0.f;
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) s1[cg][r] = s2[cg][r] = s3[cg][r] = 0;
-                }
-                for (unsigned c = cb; c < ce; ++c) {
-                    uint32_t pa0, pb0, qa0, qb0, fa0, fb0, pa1, pb1, qa1, qb1, fa1, fb1;
-                    decode_word<WB, K1>(lds32(unit + c * 4), lut_lane, pa0, pb0, qa0, qb0, fa0, fb0);
-                    decode_word<WB, K1>(lds32(unit + 512 + c * 4), lut_lane, pa1, pb1, qa1, qb1, fa1, fb1);
+                    const uint32_t unit = order_after_wait(ring_addr + slot * stage_bytes + rloc * unit_bytes + lane * 16);
+                    const uint4 wv0 = lds128(unit), wv1 = lds128(unit + 512);
+                    const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
+                    const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
+                    int s1[NG][4], s2[NG][4], s3[NG][4];
+                    float rec[NG][2];
 #pragma unroll
                     for (int cg = 0; cg < NG; ++cg) {
-                        const uint2 xf = lds64(xrow[cg] + (uint32_t)kbi * kBlockK + c * 32);
-                        mma_s8(s1[cg], pa0, pa1, pb0, pb1, xf.x, xf.y);
-                        if constexpr (!K1) {
-                            mma_s8(s2[cg], qa0, qa1, qb0, qb1, xf.x, xf.y);
-                            mma_s8(s3[cg], fa0, fa1, fb0, fb1, xf.x, xf.y);
+                        rec[cg][0] = rec[cg][1] = 0.f;
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) s1[cg][r] = s2[cg][r] = s3[cg][r] = 0;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        if ((unsigned)c >= cb && (unsigned)c < ce) {   // warp-uniform
+                            uint32_t pa0, pb0, qa0, qb0, fa0, fb0, pa1, pb1, qa1, qb1, fa1, fb1;
+                            decode_word<WB, K1>(w0[c], lut_lane, pa0, pb0, qa0, qb0, fa0, fb0);
+                            decode_word<WB, K1>(w1[c], lut_lane, pa1, pb1, qa1, qb1, fa1, fb1);
+#pragma unroll
+                            for (int cg = 0; cg < NG; ++cg) {
+                                const uint2 xf = lds64(xrow[cg] + (uint32_t)kbi * kBlockK + c * 32);
+                                mma_s8(s1[cg], pa0, pa1, pb0, pb1, xf.x, xf.y);
+                                if constexpr (!K1) {
+                                    mma_s8(s2[cg], qa0, qa1, qb0, qb1, xf.x, xf.y);
+                                    mma_s8(s3[cg], fa0, fa1, fb0, fb1, xf.x, xf.y);
+                                }
+                            }
+                            if (((c + 1) % CPG) == 0 || (unsigned)(c + 1) == ce)   // end of a macro-block, or of this warp's share of it
+                                group_end<NG, K1>(s1, s2, s3, lds32(coef_addr + (c / CPG) * 64), lds32(coef_addr + (c / CPG) * 64 + 32), rec);
                         }
                     }
-                    if (((c + 1) % CPG) == 0 || c + 1 == ce)   // end of a macro-block, or of this warp's share of it (the sums are linear)
-                        group_end<NG, K1>(s1, s2, s3, lds32(coef_addr + (c / CPG) * 64), lds32(coef_addr + (c / CPG) * 64 + 32), rec);
-                }
 #pragma unroll
-                for (int cg = 0; cg < NG; ++cg) {
-                    const float sv = lds_f32(xs_tok[cg] + kbi * (16 * NG));
-                    acc[cg][0] = fmaf(sv, rec[cg][0], acc[cg][0]);
-                    acc[cg][1] = fmaf(sv, rec[cg][1], acc[cg][1]);
+                    for (int cg = 0; cg < NG; ++cg) {
+                        const float sv = lds_f32(xs_tok[cg] + kbi * (16 * NG));
+                        acc[cg][0] = fmaf(sv, rec[cg][0], acc[cg][0]);
+                        acc[cg][1] = fmaf(sv, rec[cg][1], acc[cg][1]);
+                    }
                 }
-                u += ce - cb;
             }
         }
         flush_to(wk.P);   // every part has been handed over
@@ -712,6 +819,7 @@ static size_t chain_xbuf_bytes(int m, int k_pad) { return ((size_t)2 * m * (k_pa
 bool gemv_seq_supported(const Geometry& g, int m) {
     if (!(g.group >= 32 && g.wbits <= 3 && m >= 1 && m <= 8 && g.k_blocks <= chain::kMaxKBlocks)) return false;
     if ((unsigned long long)g.n_units * (unsigned)g.k_blocks >= (1ull << 32)) return false;   // record -> tile by multiply and shift
+    if (g.n_tiles > (1 << 21)) return false;   // tile parts per CTA stay far below 2^15 (packed beside the tail stage's chunk range)
     // at least two ring stages beside one activation buffer
     return chain_fixed_smem(m <= 4 ? 1 : 2) + chain_xbuf_bytes(m, g.k_pad) + (size_t)2 * chain::kStageRecs * g.unit_bytes <= kChainSmemMax;
 }
@@ -724,9 +832,13 @@ size_t gemv_seq_zeroed_prefix(int n_items) {
     const size_t z = kWsStatusBytes + align_up(n * sizeof(int), 256);
     return z > kWsScratchOff ? z : kWsScratchOff;
 }
+static size_t chain_parts_bytes(int n_items) {
+    return (size_t)(n_items > 0 ? n_items : 0) * (size_t)chain_sm_count() * 2 * chain::kPartWords * sizeof(uint2);
+}
 size_t gemv_seq_workspace(int n_items) {
-    const size_t n = (size_t)(n_items > 0 ? n_items : 0), G = (size_t)chain_sm_count();
-    return gemv_seq_zeroed_prefix(n_items) + n * G * 2 * chain::kPartWords * sizeof(uint2);
+    // a single linear feeds nobody: no tagged copies
+    const size_t tags = n_items > 1 ? (size_t)n_items * chain::kTagWords * sizeof(uint2) : 0;
+    return gemv_seq_zeroed_prefix(n_items) + chain_parts_bytes(n_items) + tags;
 }
 
 template <int WB, int CPG, int NG, bool K1>
@@ -768,6 +880,7 @@ cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, i
     p.done = (int*)(wsb + 256);
     p.epoch = (unsigned*)(wsb + 4);
     p.parts = (uint2*)(wsb + gemv_seq_zeroed_prefix(n));
+    p.tags = (uint2*)(wsb + gemv_seq_zeroed_prefix(n) + chain_parts_bytes(n));
     int m_max = 1;
     bool k1 = true;
     size_t x_need = 0;
@@ -786,10 +899,51 @@ cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, i
         it.m = calls[i].m;
         it.y_dtype = calls[i].y_dtype;
         it.depends = calls[i].depends;
+        it.xsrc = -1; it.xoff = 0; it.tag_out = 0; it.pad_ = 0;
         if (calls[i].m > m_max) m_max = calls[i].m;
         k1 = k1 && g.k1;
         const size_t b = chain_xbuf_bytes(calls[i].m, g.k_pad);
         if (b > x_need) x_need = b;
+    }
+    // Ordering between the items of one launch, from the address ranges. An item flagged `depends` waits for every earlier
+    // item (counter wait). An unflagged item whose activations lie inside ONE earlier bf16 output reads that output's tagged
+    // copy and waits word by word; any other overlap with what earlier items read or write falls back to the counter wait.
+    auto overlaps = [](const void* a, size_t an, const void* b, size_t bn) {
+        const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+        return a0 < b0 + bn && b0 < a0 + an;
+    };
+    auto x_bytes = [&](int i) { return (size_t)calls[i].m * calls[i].g.k_in * 2; };
+    auto y_bytes = [&](int i) { return (size_t)calls[i].m * calls[i].g.n_out * (calls[i].y_dtype == GOQ_F32 ? 4 : 2); };
+    for (int j = 1; j < n; ++j) {
+        chain::Item& it = p.item[j];
+        if (it.depends) continue;
+        int src = -1, hits = 0;
+        bool clash = false;
+        for (int i = 0; i < j; ++i) {
+            if (overlaps(calls[j].x, x_bytes(j), calls[i].y, y_bytes(i))) { src = i; ++hits; }
+            if (overlaps(calls[j].y, y_bytes(j), calls[i].y, y_bytes(i)) || overlaps(calls[j].y, y_bytes(j), calls[i].x, x_bytes(i))) clash = true;
+        }
+        if (!clash && hits == 0) continue;   // independent of everything before it
+        bool tagged = false;
+        if (!clash && hits == 1 && calls[src].y_dtype == GOQ_BF16) {
+            const Geometry& gs = calls[src].g;
+            const Geometry& gj = calls[j].g;
+            const int ms = calls[src].m, mj = calls[j].m;
+            const uintptr_t x0 = (uintptr_t)calls[j].x, y0 = (uintptr_t)calls[src].y;
+            const size_t stride = (size_t)gs.n_tiles * 8;   // words per token of the copy
+            if (x0 >= y0 && (x0 - y0) % 2 == 0 && (size_t)ms * stride <= (size_t)chain::kTagWords && gj.k_in % 8 == 0) {
+                const size_t e = (x0 - y0) / 2, tok0 = e / (size_t)gs.n_out, off = e % (size_t)gs.n_out;
+                const bool rows_ok = (mj == 1) ? (off + (size_t)gj.k_in <= (size_t)gs.n_out)
+                                               : (off == 0 && gj.k_in == gs.n_out && tok0 + (size_t)mj <= (size_t)ms);
+                if (off % 8 == 0 && rows_ok && tok0 < (size_t)ms) {
+                    it.xsrc = src;
+                    it.xoff = (unsigned)(tok0 * stride + off / 2);
+                    p.item[src].tag_out = 1;
+                    tagged = true;
+                }
+            }
+        }
+        if (!tagged) it.depends = 1;
     }
     const int cpg = group / 32;
 #define GOQ_CHAIN(WB_, NG_, K1_)                                                                             \

@@ -41,18 +41,19 @@ def form(goq):
     goq.set_gemv_variant(prev)
 
 
-def test_chain_with_real_dependencies_matches_oracle_stage_by_stage(goq, form):
+@pytest.mark.parametrize("flagged,batch", [(True, 3), (False, 3), (False, 1), (False, 4), (False, 6)])
+def test_chain_with_real_dependencies_matches_oracle_stage_by_stage(goq, form, flagged, batch):
     """y0 = W0 x0 (bf16 out) feeds W1, whose bf16 output feeds W2: every stage is checked against the oracle
-    evaluated on the bits the previous stage actually produced."""
+    evaluated on the bits the previous stage actually produced. Flagged items wait for the completion counter;
+    unflagged ones are ordered by the library from the address ranges (they poll the producer's tagged copy)."""
     from tests.gpu_util import dev
-    batch = 3
     shapes = [(256, 384), (512, 256), (130, 512)]   # (n_out, k_in): n_out of one = k_in of the next
     layers = [_layer(goq, n, k, 64, 3, seed=40 + i) for i, (n, k) in enumerate(shapes)]
     x0 = si.bf16_activations(batch, shapes[0][1], seed=5)
     bufs = [dev(x0)] + [torch.zeros((batch, n), dtype=torch.bfloat16, device="cuda") for n, _ in shapes[:-1]]
     y_last = torch.zeros((batch, shapes[-1][0]), dtype=torch.float32, device="cuda")
     outs = bufs[1:] + [y_last]
-    items = [(L["d"], L["packed"], bufs[i], batch, outs[i], goq.BF16 if i < 2 else goq.F32, i > 0)
+    items = [(L["d"], L["packed"], bufs[i], batch, outs[i], goq.BF16 if i < 2 else goq.F32, flagged and i > 0)
              for i, L in enumerate(layers)]
     seq = goq.make_sequence(items)
     ws = _ws(goq, len(items))
@@ -71,6 +72,120 @@ def test_chain_with_real_dependencies_matches_oracle_stage_by_stage(goq, form):
                 check_bf16_output(got, y_ref, 1e-4, "stage %d" % i)
             if i < 2:
                 x_bits = outs[i].view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def _check_item(L, x_bits, out, bf16_out, what):
+    """One item against the oracle evaluated on the activation bits it was given."""
+    from tests.gpu_util import check_bf16_output
+    y_ref = O.linear_f64(L["codes"], L["meta"], L["coef"], si.bf16_bits_to_f64(x_bits), L["g"], L["b"])
+    got = out.float().cpu().numpy().astype(np.float64)
+    if bf16_out:
+        check_bf16_output(got, y_ref, 1e-4, what)
+    else:
+        assert O.normwise_rel_err(got, y_ref) <= TIGHT, (what, O.normwise_rel_err(got, y_ref))
+
+
+def _bits(t):
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def test_data_flow_slices_fan_out_and_a_producer_two_items_back(goq, form):
+    """Unflagged items ordered by address ranges alone (batch 1): item 1 and item 2 read two different slices of item
+    0's bf16 output (channel counts that are no multiple of a tile), item 3 reads item 1's output although item 2 lies
+    between them, item 4 reads all of item 2's. Run twice on one scratch buffer, with a producer wide enough to be
+    spread over every SM, so that readers really wait for tiles finished elsewhere."""
+    from tests.gpu_util import dev
+    L0 = _layer(goq, 4104, 512, 32, 3, seed=700)       # 256.5 tiles: the last one is half empty
+    L1 = _layer(goq, 416, 2048, 32, 3, seed=701)        # reads y0[0:2048]
+    L2 = _layer(goq, 544, 1024, 32, 3, seed=702)        # reads y0[3072:4096]
+    L3 = _layer(goq, 100, 416, 32, 3, seed=703)         # reads y1 (416 channels: k padded to 512)
+    L4 = _layer(goq, 64, 544, 32, 3, seed=704)          # reads y2
+    x0 = si.bf16_activations(1, 512, seed=70)
+    y0 = torch.zeros((1, 4104), dtype=torch.bfloat16, device="cuda")
+    y1 = torch.zeros((1, 416), dtype=torch.bfloat16, device="cuda")
+    y2 = torch.zeros((1, 544), dtype=torch.bfloat16, device="cuda")
+    y3 = torch.zeros((1, 100), dtype=torch.float32, device="cuda")
+    y4 = torch.zeros((1, 64), dtype=torch.bfloat16, device="cuda")
+    items = [(L0["d"], L0["packed"], dev(x0), 1, y0, goq.BF16, False),
+             (L1["d"], L1["packed"], y0[:, 0:2048], 1, y1, goq.BF16, False),
+             (L2["d"], L2["packed"], y0[:, 3072:4096], 1, y2, goq.BF16, False),
+             (L3["d"], L3["packed"], y1, 1, y3, goq.F32, False),
+             (L4["d"], L4["packed"], y2, 1, y4, goq.BF16, False)]
+    keep = [t[2] for t in items]
+    seq = goq.make_sequence(items)
+    ws = _ws(goq, len(items))
+    for rep in range(2):
+        for y in (y0, y1, y2, y3, y4):
+            y.zero_()
+        goq.gemv_sequence(seq, ws)
+        torch.cuda.synchronize()
+        assert goq.workspace_status(ws) == goq.OK
+        b0 = _bits(y0)
+        _check_item(L0, x0, y0, True, "item 0")
+        _check_item(L1, b0[:, 0:2048], y1, True, "item 1")
+        _check_item(L2, b0[:, 3072:4096], y2, True, "item 2")
+        _check_item(L3, _bits(y1), y3, False, "item 3")
+        _check_item(L4, _bits(y2), y4, True, "item 4")
+    del keep
+
+
+def test_overlaps_the_tagged_copy_cannot_serve_fall_back_to_the_counter_wait(goq, form):
+    """Unflagged items whose buffers overlap earlier ones in ways the word-by-word wait does not cover are still ordered
+    correctly: item 2 reads one buffer that items 0 and 1 each wrote half of (two producers), item 3 writes where item 0
+    wrote after item 2 has read it (an output buffer used twice)."""
+    from tests.gpu_util import dev
+    La = _layer(goq, 512, 256, 64, 3, seed=710)
+    Lb = _layer(goq, 512, 256, 64, 3, seed=711)
+    Lc = _layer(goq, 256, 1024, 64, 3, seed=712)
+    Ld = _layer(goq, 512, 256, 64, 3, seed=713)
+    x0 = si.bf16_activations(1, 256, seed=71)
+    xd = dev(x0)
+    P = torch.zeros((1, 1024), dtype=torch.bfloat16, device="cuda")
+    B = torch.zeros((1, 256), dtype=torch.bfloat16, device="cuda")
+    items = [(La["d"], La["packed"], xd, 1, P[:, 0:512], goq.BF16, False),
+             (Lb["d"], Lb["packed"], xd, 1, P[:, 512:1024], goq.BF16, False),
+             (Lc["d"], Lc["packed"], P, 1, B, goq.BF16, False),
+             (Ld["d"], Ld["packed"], B, 1, P[:, 0:512], goq.BF16, False)]
+    keep = [t[4] for t in items]
+    ws = _ws(goq, len(items))
+    goq.gemv_sequence(goq.make_sequence(items), ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    # P[0:512] now holds item 3's result; item 0's is recomputed on its own (the kernel is deterministic)
+    P0 = torch.zeros((1, 512), dtype=torch.bfloat16, device="cuda")
+    goq.gemv_sequence(goq.make_sequence([(La["d"], La["packed"], xd, 1, P0, goq.BF16, False)]), _ws(goq, 1))
+    torch.cuda.synchronize()
+    _check_item(La, x0, P0, True, "item 0")
+    _check_item(Lb, x0, P[:, 512:1024].contiguous(), True, "item 1")
+    p_bits = np.concatenate([_bits(P0), _bits(P[:, 512:1024].contiguous())], axis=1)
+    _check_item(Lc, p_bits, B, True, "item 2")
+    _check_item(Ld, _bits(B), P[:, 0:512].contiguous(), True, "item 3")
+    del keep
+
+
+def test_a_data_flow_wait_that_runs_out_reports_timeout(goq):
+    """The word-by-word wait is bounded like every other: with a bound of one poll a reader gives up before the producer's
+    tiles are there, the launch ends by itself with GOQ_ERR_TIMEOUT, and after a zero-fill the chain runs correctly."""
+    from tests.gpu_util import dev
+    La, Lb = _layer(goq, 2048, 2048, 128, 3, seed=601), _layer(goq, 512, 2048, 128, 3, seed=602)
+    xa = si.bf16_activations(1, 2048, seed=31)
+    mid = torch.zeros((1, 2048), dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros((1, 512), dtype=torch.float32, device="cuda")
+    xd = dev(xa)
+    seq = goq.make_sequence([(La["d"], La["packed"], xd, 1, mid, goq.BF16, False), (Lb["d"], Lb["packed"], mid, 1, y, goq.F32, False)])
+    ws = _ws(goq, 2)
+    prev = goq.set_wait_limit(1)
+    try:
+        goq.gemv_sequence(seq, ws)
+        torch.cuda.synchronize()
+        assert goq.workspace_status(ws) == goq.ERR_TIMEOUT
+    finally:
+        goq.set_wait_limit(prev)
+    goq.workspace_init(ws)
+    goq.gemv_sequence(seq, ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    _check_item(Lb, _bits(mid), y, False, "second linear")
 
 
 @pytest.mark.parametrize("g,b", [(128, 3), (32, 2)])
