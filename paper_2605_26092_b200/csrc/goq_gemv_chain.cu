@@ -53,17 +53,34 @@ struct Item {
     int xsrc;                                // earlier item whose output this item's x lies in (read from that item's tagged copy), or -1
     unsigned int xoff;                       // first 64-bit word of x inside that copy
     int tag_out;                             // a later item reads this item's output: keep the tagged copy
-    int pad_;
+    unsigned int uq, ur;                     // units / G and units % G for the launch's G CTAs (the kernel never divides)
 };
 struct Params {
     Item item[kSeqMaxItems];
     int n_items, unit_bytes, n_stages, x_double, xbuf_bytes, spin_limit;
+    unsigned long long g_magic;   // ceil(2^32 / G): n / G for n < G^2 by multiply and shift
     int* status;
     int* done;       // [n_items] CTAs that have finished each linear; zero on entry, left zero
     unsigned* epoch; // launches this scratch buffer has seen: tags the posted parts (zero-filled scratch carries no valid tag)
     uint2* parts;    // [n_items][G][2][32 lanes x 2 NG] posted partial sums, each value in one 64-bit word with its tag
     uint2* tags;     // [n_items][kTagWords] tagged copies of bf16 outputs: [token][16 n_tiles / 2] words of (two values, tag)
 };
+
+// Split of a last stage of n < 16 records over the 16 consumer warps: 16 / n warps share a record, each a run of its four chunks.
+struct TailShare { unsigned short v[16][16]; };
+constexpr TailShare make_tail_share() {
+    TailShare t{};
+    for (int n = 1; n < 16; ++n) {
+        const int wpr = 16 / n;
+        for (int w = 0; w < 16; ++w) {
+            const int rloc = w / wpr, sub = w - rloc * wpr;
+            const int cb = 4 * sub / wpr, ce = 4 * (sub + 1) / wpr;
+            t.v[n][w] = (unsigned short)(rloc < n ? (rloc | (cb << 4) | (ce << 7)) : 15);   // 15: no share (first chunk = end chunk = 0)
+        }
+    }
+    return t;
+}
+__constant__ TailShare c_tail_share = make_tail_share();
 
 constexpr int kPartWords = 128;              // 64-bit (value, tag) words of one posted part: 16 rows x 8 tokens
 constexpr int kTagWords = 4 * (kMaxKBlocks * kBlockK / 2);   // per item: four tokens of the widest input a linear can take
@@ -157,20 +174,21 @@ struct Walk {
     int Ta, Tb, P;           // first and last tile touched, number of tile parts
     bool rot;
 };
-__device__ __forceinline__ Walk make_walk(const Item& it, int cta, int G) {
+// No division anywhere: every warp works this out at the start of every linear, on the critical path of a chain of small ones.
+__device__ __forceinline__ unsigned mul_shift32(unsigned n, unsigned long long magic) { return (unsigned)(((unsigned long long)n * magic) >> 32); }
+__device__ __forceinline__ Walk make_walk(const Item& it, int cta, unsigned long long g_magic) {
     Walk w;
-    // floor(units c / G) = c (units / G) + floor(c (units % G) / G): 32-bit arithmetic (c (units % G) < G^2)
-    const unsigned uq = it.units / (unsigned)G, ur = it.units % (unsigned)G;
-    w.a = (unsigned)cta * uq + (unsigned)cta * ur / (unsigned)G;
-    w.b = (unsigned)(cta + 1) * uq + (unsigned)(cta + 1) * ur / (unsigned)G;
+    // floor(units c / G) = c (units / G) + floor(c (units % G) / G)
+    w.a = (unsigned)cta * it.uq + mul_shift32((unsigned)cta * it.ur, g_magic);
+    w.b = (unsigned)(cta + 1) * it.uq + mul_shift32((unsigned)(cta + 1) * it.ur, g_magic);
     w.L = w.b - w.a;
     w.L1 = 0; w.s1 = 0; w.Ta = 0; w.Tb = 0; w.P = 0; w.rot = false;
     if (w.L) {
         const unsigned kb = (unsigned)it.k_blocks;
-        w.Ta = (int)(w.a / kb);
-        w.Tb = (int)((w.b - 1) / kb);
+        w.Ta = (int)mul_shift32(w.a, it.kb_magic);
+        w.Tb = (int)mul_shift32(w.b - 1, it.kb_magic);
         w.P = w.Tb - w.Ta + 1;
-        w.rot = w.Tb > w.Ta && (w.b % kb) != 0;
+        w.rot = w.Tb > w.Ta && w.b != mul_shift32(w.b, it.kb_magic) * kb;
         if (w.rot) { w.s1 = (unsigned)w.Tb * kb; w.L1 = w.b - w.s1; }
     }
     return w;
@@ -281,7 +299,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
             bool ok = true;
             for (int i = 0; i < p.n_items && ok; ++i) {
                 const Item& it = p.item[i];
-                const Walk wk = make_walk(it, cta, G);
+                const Walk wk = make_walk(it, cta, p.g_magic);
                 for (unsigned j0 = 0; j0 < wk.L; j0 += kStageRecs) {
                     if (round > 0 && !wait_bar(&empty_bar[slot], (round - 1) & 1, &abort_flag, spin)) { ok = false; break; }
                     const unsigned n = min((unsigned)kStageRecs, wk.L - j0);
@@ -323,7 +341,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
         const unsigned epoch = *p.epoch, tag = ((epoch + 1u) * 0x9E3779B1u) | 1u;
         for (int i = 0; i < p.n_items && ok; ++i) {
             const Item& it = p.item[i];
-            const Walk wk = make_walk(it, cta, G);
+            const Walk wk = make_walk(it, cta, p.g_magic);
             if (wk.L) {
                 if (it.depends && i > 0) {
                     if (lane == 0) {
@@ -339,8 +357,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 // for its outputs, and a lone warp runs at instruction latency: whatever does not need the sums (which tile, who
                 // finishes it, every address) is worked out BEFORE the wait for the part, and nothing on the far side divides.
                 const unsigned kb = (unsigned)it.k_blocks;
-                const unsigned uq = it.units / (unsigned)G, ur = it.units % (unsigned)G;   // range boundaries step by uq (+1) from CTA to CTA
-                const unsigned rem_a = ((unsigned)cta * ur) % (unsigned)G;
+                const unsigned uq = it.uq, ur = it.ur;   // range boundaries step by uq (+1) from CTA to CTA
+                const unsigned rem_a = (unsigned)cta * ur - (unsigned)G * mul_shift32((unsigned)cta * ur, p.g_magic);
                 const int tok0 = lane & 3;
                 const size_t tstride4 = (size_t)4 * (it.n_tiles * 8), ystride4 = (size_t)4 * it.n_out;
                 const bool y32 = it.y_dtype == GOQ_F32;
@@ -491,7 +509,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
 
     for (int i = 0; i < p.n_items && alive; ++i) {
         const Item& it = p.item[i];
-        const Walk wk = make_walk(it, cta, G);
+        const Walk wk = make_walk(it, cta, p.g_magic);
         if (wk.L == 0) continue;   // nothing of this linear belongs to this CTA (the control warp reports it finished)
         const int kb = it.k_blocks, k_pad = kb * kBlockK, plane = k_pad + kXPad, m = it.m;
         if (p.x_double) x_sel ^= 1;
@@ -504,12 +522,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
         const unsigned n_full = wk.L / kStageRecs, n_tail = wk.L - n_full * kStageRecs;
         unsigned tail_desc = 0;   // [0:4) record of the stage, [4:7) first chunk, [7:10) end chunk, [10:17) k-block, [17:32) tile part
         if (n_tail) {
-            const unsigned wpr = (unsigned)kNW / n_tail;   // >= 1
-            const unsigned rloc = (unsigned)warp / wpr, sub = (unsigned)warp - rloc * wpr;
-            const unsigned cb = 4u * sub / wpr, ce = 4u * (sub + 1u) / wpr;
+            const unsigned share = c_tail_share.v[n_tail][warp];   // record, first and end chunk of this warp
+            const unsigned rloc = share & 15u, cb = (share >> 4) & 7u, ce = (share >> 7) & 7u;
             if (rloc < n_tail && cb < ce) {
                 const unsigned rho = walk_record(wk, n_full * kStageRecs + rloc);
-                const unsigned T = (unsigned)(((unsigned long long)rho * it.kb_magic) >> 32);
+                const unsigned T = mul_shift32(rho, it.kb_magic);
                 const unsigned kbi = rho - T * (unsigned)kb;
                 tail_desc = rloc | (cb << 4) | (ce << 7) | (kbi << 10) | ((unsigned)walk_part_of_tile(wk, (int)T) << 17);
             }
@@ -560,7 +577,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 for (int c0 = warp * 32; c0 < total; c0 += kNW * 32) {
                     const int c = c0 + lane;
                     const bool in = c < total;
-                    const int r = in ? c / cpt : 0, k0 = in ? (c - r * cpt) * 8 : 0;
+                    const int r = in ? (int)mul_shift32((unsigned)c >> 4, it.kb_magic) : 0, k0 = in ? (c - r * cpt) * 8 : 0;   // cpt = 16 k_blocks
                     uint4 v = make_uint4(0u, 0u, 0u, 0u);
                     if (in && k0 < it.k_in) v = __ldcg(reinterpret_cast<const uint4*>(it.x + (size_t)r * it.k_in + k0));   // L2: written by other SMs
                     convert(v, in, r, k0);
@@ -578,7 +595,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
 #pragma unroll
                     for (int u = 0; u < kXBatch; ++u) {
                         const int c = cb + u * (kNW * 32) + lane;
-                        const int r = c < total ? c / cpt : 0, k0 = c < total ? (c - r * cpt) * 8 : 0;
+                        const int r = c < total ? (int)mul_shift32((unsigned)c >> 4, it.kb_magic) : 0, k0 = c < total ? (c - r * cpt) * 8 : 0;
                         need[u] = c < total && k0 < it.k_in;
                         v[u] = make_uint4(0u, 0u, 0u, 0u);
                     }
@@ -589,7 +606,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                         for (int u = 0; u < kXBatch; ++u)
                             if (need[u]) {
                                 const int c = cb + u * (kNW * 32) + lane;
-                                const int r = c / cpt, k0 = (c - r * cpt) * 8;
+                                const int r = (int)mul_shift32((unsigned)c >> 4, it.kb_magic), k0 = (c - r * cpt) * 8;
                                 const uint2* src = tg + (size_t)r * tstride + (k0 >> 1);
                                 unsigned long long w0, w1, w2, w3;
                                 asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(src) : "memory");
@@ -610,7 +627,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                     for (int u = 0; u < kXBatch; ++u) {
                         const int c = cb + u * (kNW * 32) + lane;
                         const bool in = c < total;
-                        const int r = in ? c / cpt : 0, k0 = in ? (c - r * cpt) * 8 : 0;
+                        const int r = in ? (int)mul_shift32((unsigned)c >> 4, it.kb_magic) : 0, k0 = in ? (c - r * cpt) * 8 : 0;
                         if (cb + u * (kNW * 32) < total) convert(v[u], in, r, k0);   // warp-uniform: the conversion shuffles
                     }
                 }
@@ -658,7 +675,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
             while (st < n_full && alive) {
                 if (locate) {
                     const unsigned rho = walk_record(wk, j);
-                    const int T = (int)(((unsigned long long)rho * it.kb_magic) >> 32);
+                    const int T = (int)mul_shift32(rho, it.kb_magic);
                     kbi = (int)(rho - (unsigned)T * (unsigned)kb);
                     q = walk_part_of_tile(wk, T);
                     locate = false;
@@ -881,6 +898,8 @@ cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, i
     p.epoch = (unsigned*)(wsb + 4);
     p.parts = (uint2*)(wsb + gemv_seq_zeroed_prefix(n));
     p.tags = (uint2*)(wsb + gemv_seq_zeroed_prefix(n) + chain_parts_bytes(n));
+    const int G = chain_sm_count();   // the grid
+    p.g_magic = ((1ull << 32) + (unsigned)G - 1) / (unsigned)G;
     int m_max = 1;
     bool k1 = true;
     size_t x_need = 0;
@@ -899,7 +918,9 @@ cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, i
         it.m = calls[i].m;
         it.y_dtype = calls[i].y_dtype;
         it.depends = calls[i].depends;
-        it.xsrc = -1; it.xoff = 0; it.tag_out = 0; it.pad_ = 0;
+        it.xsrc = -1; it.xoff = 0; it.tag_out = 0;
+        it.uq = it.units / (unsigned)G;
+        it.ur = it.units % (unsigned)G;
         if (calls[i].m > m_max) m_max = calls[i].m;
         k1 = k1 && g.k1;
         const size_t b = chain_xbuf_bytes(calls[i].m, g.k_pad);
