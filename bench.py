@@ -192,16 +192,34 @@ def build_stack(goq, torch, layers, seed0, batch):
             d = goq.desc(n, k, GROUP, WBITS)
             codes = torch.randint(0, 1 << WBITS, (n, k), dtype=torch.uint8, device="cuda", generator=gen)
             meta = torch.randint(0, 64, (n, k // 8), dtype=torch.uint8, device="cuda", generator=gen)
-            coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * 0.03).to(torch.float16)
+            # coefficient scale for unit gain: with uniform codes E[b^2] = 0.33 per basis, so |W x| ~ |x| when the two
+            # coefficients have standard deviation 1 / sqrt(0.66 k); a chain fed its own outputs then neither dies out nor overflows
+            coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * (0.66 * k) ** -0.5).to(torch.float16)
             packed = torch.empty(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
             goq.pack(d, codes, meta, coef, packed)
             x = torch.randn((batch, k), device="cuda", generator=gen).to(torch.bfloat16)
             y = torch.empty((batch, n), dtype=torch.float32, device="cuda")
-            stack.append({"d": d, "packed": packed, "x": x, "y": y, "n": n, "k": k})
+            stack.append({"d": d, "packed": packed, "x": x, "y": y, "n": n, "k": k,
+                          "yb": torch.zeros((batch, n), dtype=torch.bfloat16, device="cuda")})
             build_stack.ws_bytes = max(getattr(build_stack, "ws_bytes", 256), goq.workspace_bytes(d, goq.OP_GEMV, 16))
             del codes, meta, coef
     torch.cuda.synchronize()
     return stack
+
+
+def flow_items(goq, stack, x0=None, outs=None):
+    """The decode step as a true chain: linear j reads the first k_j channels of linear j-1's bf16 output (the first one
+    reads x0). No item is flagged: the library finds the dependencies from the address ranges."""
+    items = []
+    for j, s in enumerate(stack):
+        y = outs[j] if outs is not None else s["yb"]
+        if j == 0:
+            x = x0 if x0 is not None else s["x"]
+        else:
+            prev = outs[j - 1] if outs is not None else stack[j - 1]["yb"]
+            x = prev[:, :s["k"]]
+        items.append((s["d"], s["packed"], x, 1, y, goq.BF16, False))
+    return items
 
 
 def capture(torch, fn):
@@ -305,8 +323,8 @@ def run_cuda(args):
     goq.workspace_init(ws)
 
     if args.launch == "sequence":
-        # the whole step is one persistent kernel; every linear waits for all earlier ones (stream-order semantics)
-        seq = goq.make_sequence([(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, True) for s in stack])
+        # the whole step is one persistent kernel and a true chain: every linear reads the previous linear's output
+        seq = goq.make_sequence(flow_items(goq, stack))
         ws_seq = torch.empty(goq.sequence_workspace_bytes(n_lin), dtype=torch.uint8, device="cuda")
         goq.workspace_init(ws_seq)
         kernels_per_step = (n_lin + 255) // 256
@@ -351,22 +369,20 @@ def run_cuda(args):
 
     # ---- end to end: host buffers in, host buffers out, through the C ABI's host entry points ---------
     if args.launch == "sequence":
-        # one pinned host block with every linear's activations, one with every output; goq_gemv_sequence_host
+        # one pinned host block with the step's input activations, one with every linear's output; goq_gemv_sequence_host
         # copies the first in, runs the sequence kernel on views of the device blocks, copies the second out
-        x_off, y_off, xo, yo = [], [], 0, 0
+        y_off, yo = [], 0
         for s in stack:
-            x_off.append(xo); xo += (s["k"] * 2 + 255) // 256 * 256
-            y_off.append(yo); yo += (s["n"] * 4 + 255) // 256 * 256
+            y_off.append(yo); yo += (s["n"] * 2 + 255) // 256 * 256
+        xo = (stack[0]["k"] * 2 + 255) // 256 * 256
         x_stage = torch.zeros(xo, dtype=torch.uint8, device="cuda")
         y_stage = torch.zeros(yo, dtype=torch.uint8, device="cuda")
         x_host = torch.zeros(xo, dtype=torch.uint8).pin_memory()
         y_host = torch.zeros(yo, dtype=torch.uint8).pin_memory()
-        views = []
-        for s, a, b in zip(stack, x_off, y_off):
-            x_host[a:a + s["k"] * 2] = s["x"].view(torch.uint8).flatten().cpu()
-            views.append((x_stage[a:a + s["k"] * 2].view(torch.bfloat16).view(1, s["k"]),
-                          y_stage[b:b + s["n"] * 4].view(torch.float32).view(1, s["n"])))
-        seq_e2e = goq.make_sequence([(s["d"], s["packed"], xv, 1, yv, goq.F32, True) for s, (xv, yv) in zip(stack, views)])
+        x_host[:stack[0]["k"] * 2] = stack[0]["x"].view(torch.uint8).flatten().cpu()
+        x0v = x_stage[:stack[0]["k"] * 2].view(torch.bfloat16).view(1, stack[0]["k"])
+        outs = [y_stage[b:b + s["n"] * 2].view(torch.bfloat16).view(1, s["n"]) for s, b in zip(stack, y_off)]
+        seq_e2e = goq.make_sequence(flow_items(goq, stack, x0v, outs))
         e2e_desc = "one CUDA graph holding one goq_gemv_sequence_host call (one pinned H2D block, the sequence kernel, one D2H block)"
 
         def step_e2e():
@@ -414,7 +430,8 @@ def run_cuda(args):
     achieved = launch_bytes / (launch_ms * 1e-3) / 1e9
     if args.launch == "sequence":
         kernel_name = "gemv_chain_kernel<3,4,1>"
-        launch_desc = "one CUDA graph holding one goq_gemv_sequence call (%d linears, each waits for all earlier ones)" % n_lin
+        launch_desc = ("one CUDA graph holding one goq_gemv_sequence call: %d linears in a true chain, each reads the previous "
+                       "one's bf16 output (its first k channels)" % n_lin)
         ratio, ratio_src = NCU_TRAFFIC_RATIO_SEQ, "ncu dram bytes of a 14-linear chain launch (profiles/gemv_chain_llama7b_2layers_batch1.md) scaled by algorithmic bytes"
         if int(goq.workspace_status(ws_seq)) != 0:
             raise RuntimeError("sequence kernel reported a device-side timeout")
@@ -491,16 +508,33 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
     ms = time_graph(torch, g, 20, 3)
     out["gemv_graph_of_launches_gbs"] = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack) / (ms * 1e-3) / 1e9
     del g
-    # ... and as a sequence whose dependencies follow a transformer layer (k, v and up need not wait)
-    names = [nm for nm, _, _ in si.LLAMA2_7B_LINEARS]
-    seq = goq.make_sequence([(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, names[j % 7] not in ("k_proj", "v_proj", "up_proj"))
-                             for j, s in enumerate(stack)])
+    # ... as a sequence of flagged items over independent buffers: every linear waits until all SMs have finished the previous
+    # one (the completion-counter barrier; the timed path orders by data flow instead)
+    seq = goq.make_sequence([(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, j > 0) for j, s in enumerate(stack)])
     ws_seq = torch.empty(goq.sequence_workspace_bytes(len(stack)), dtype=torch.uint8, device="cuda")
     goq.workspace_init(ws_seq)
     g = capture(torch, lambda: goq.gemv_sequence(seq, ws_seq))
     ms = time_graph(torch, g, 20, 3)
-    out["gemv_sequence_layer_groups_gbs"] = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack) / (ms * 1e-3) / 1e9
+    out["gemv_sequence_barrier_chain_gbs"] = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack) / (ms * 1e-3) / 1e9
     del g
+    # ... and with the data flow of a transformer layer: q, k and v read the previous layer's down output, o reads v's,
+    # gate and up read o's, down reads up's (bf16 outputs, dependencies found from the address ranges)
+    src = {"q_proj": ("down_proj", -1), "k_proj": ("down_proj", -1), "v_proj": ("down_proj", -1), "o_proj": ("v_proj", 0),
+           "gate_proj": ("o_proj", 0), "up_proj": ("o_proj", 0), "down_proj": ("up_proj", 0)}
+    names = [nm for nm, _, _ in si.LLAMA2_7B_LINEARS]
+    items = []
+    for j, s in enumerate(stack):
+        layer, nm = divmod(j, 7)[0], names[j % 7]
+        pn, dl = src[nm]
+        pj = (layer + dl) * 7 + names.index(pn)
+        x = s["x"] if pj < 0 else stack[pj]["yb"][:, :s["k"]]
+        items.append((s["d"], s["packed"], x, 1, s["yb"], goq.BF16, False))
+    seq = goq.make_sequence(items)
+    goq.workspace_init(ws_seq)
+    g = capture(torch, lambda: goq.gemv_sequence(seq, ws_seq))
+    ms = time_graph(torch, g, 20, 3)
+    out["gemv_sequence_layer_groups_gbs"] = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in stack) / (ms * 1e-3) / 1e9
+    del g, items
     # ... and with the usual serving fusions: q, k, v share their input and become one 12288 x 4096 linear, gate and up
     # one 22016 x 4096 (row-wise quantization groups make the concatenation exact): 4 dependent linears per layer, same bytes
     fused_shapes = [(3 * 4096, 4096), (4096, 4096), (2 * 11008, 4096), (4096, 11008)]
@@ -512,20 +546,29 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
             d = goq.desc(n, k, GROUP, WBITS)
             codes = torch.randint(0, 1 << WBITS, (n, k), dtype=torch.uint8, device="cuda", generator=gen)
             meta = torch.randint(0, 64, (n, k // 8), dtype=torch.uint8, device="cuda", generator=gen)
-            coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * 0.03).to(torch.float16)
+            coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * (0.66 * k) ** -0.5).to(torch.float16)
             packed = torch.empty(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
             goq.pack(d, codes, meta, coef, packed)
             x = torch.randn((1, k), device="cuda", generator=gen).to(torch.bfloat16)
-            y = torch.empty((1, n), dtype=torch.float32, device="cuda")
+            y = torch.zeros((1, n), dtype=torch.bfloat16, device="cuda")
             fused.append({"d": d, "packed": packed, "x": x, "y": y, "n": n, "k": k})
             del codes, meta, coef
-    seq_f = goq.make_sequence([(s["d"], s["packed"], s["x"], 1, s["y"], goq.F32, j > 0) for j, s in enumerate(fused)])
+    # data flow: o reads the v third of q|k|v, gate|up reads o, down reads the up half of gate|up, the next q|k|v reads down
+    items = []
+    for j, s in enumerate(fused):
+        if j == 0:
+            x = s["x"]
+        else:
+            prev = fused[j - 1]
+            x = prev["y"][:, prev["n"] - s["k"]:]
+        items.append((s["d"], s["packed"], x, 1, s["y"], goq.BF16, False))
+    seq_f = goq.make_sequence(items)
     ws_f = torch.empty(goq.sequence_workspace_bytes(len(fused)), dtype=torch.uint8, device="cuda")
     goq.workspace_init(ws_f)
     g = capture(torch, lambda: goq.gemv_sequence(seq_f, ws_f))
     ms = time_graph(torch, g, 20, 3)
     out["gemv_sequence_fused_qkv_gateup_gbs"] = sum(algorithmic_bytes(s["n"], s["k"], 1) for s in fused) / (ms * 1e-3) / 1e9
-    del g, fused, seq_f
+    del g, fused, seq_f, items
     # per-shape batch-1 time (rotating over the layers' copies of that shape, so each launch reads cold weights)
     shapes = {}
     for idx, (name, n, k) in enumerate(si.LLAMA2_7B_LINEARS):

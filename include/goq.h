@@ -242,10 +242,18 @@ goq_status goq_gemv_static_status(void* stream, int* status_out);
  * not propagated (they saturate).
  *   items    HOST array of n_items entries (read during the call, not kept):
  *            desc, packed, x_bf16 [batch][k_in], y [batch][n_out], y_dtype as in goq_gemv, all device pointers;
- *            depends != 0 : this item's x (or y) may alias outputs of EARLIER items of the sequence - the kernel
- *                           then waits until every earlier item is complete before it reads x;
- *            depends == 0 : x and y are independent of every earlier item (their buffers must not overlap the
- *                           outputs of earlier items).
+ *            depends != 0 : the kernel waits until every earlier item of the sequence is complete (all SMs) before it
+ *                           reads this item's x - a full barrier, whatever the buffers;
+ *            depends == 0 : the library orders the item from the address ranges alone. Activations that lie inside
+ *                           ONE earlier item's bf16 output (the whole output with the same batch, or for batch 1 any
+ *                           slice of it that starts at a multiple of 8 channels) are taken as soon as the producer's
+ *                           16-channel tiles that hold them are finished, wherever on the GPU that happened: the
+ *                           fastest way to chain linears. Any other overlap of this item's x or y with the x or y of
+ *                           earlier items (an fp32 producer, an input that spans two outputs, an output buffer used
+ *                           twice) is detected too and handled as if depends were set. Items that overlap nothing
+ *                           run without waiting.
+ *            Give every item of a chain its own output buffer: writing an earlier item's output (or input) buffer
+ *            again forces the full barrier.
  *   Constraints (else GOQ_ERR_UNSUPPORTED): every item has the same wbits (2 or 3) and group (32, 64, 128),
  *   batch <= 8, k_in <= 12288, and the staged activations (2 * batch * (round_up(k_in, 128) + 32) bytes) fit in
  *   shared memory beside two 16-record stages of the weight stream (about 180 KB: batch 8 up to k_in = 11008).

@@ -305,7 +305,7 @@ goq_status goq_gemv_sequence_host(const goq_gemv_item* items, int n_items, const
         const size_t yb = (size_t)it.batch * it.desc.n_out * (it.y_dtype == GOQ_F32 ? 4 : 2);
         const uintptr_t x = (uintptr_t)it.x_bf16, y = (uintptr_t)it.y;
         const bool x_in_x = x >= xs && x + xb <= xs + x_bytes, x_in_y = x >= ys && x + xb <= ys + y_bytes;
-        if (!(x_in_x || (x_in_y && i > 0 && it.depends)) || !(y >= ys && y + yb <= ys + y_bytes)) return GOQ_ERR_INVALID_ARG;
+        if (!(x_in_x || (x_in_y && i > 0)) || !(y >= ys && y + yb <= ys + y_bytes)) return GOQ_ERR_INVALID_ARG;
     }
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemcpyAsync(x_stage, x_host, x_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return from_cuda(cudaGetLastError());

@@ -4,18 +4,29 @@
 // are numbered tile by tile, k-block by k-block, which is also their order in the packed buffer. CTA c of G takes
 // the contiguous range [U c / G, U (c+1) / G) of the U records of every linear: equal bytes per SM whatever the
 // shape. A range is consumed 16 records at a time (one ring stage = one bulk copy), record w of a stage by
-// consumer warp w; a last stage of n < 16 records is split at the granularity of a 32-wide k-chunk so that the
-// 4n chunks are spread evenly over the 16 warps.
+// consumer warp w; a last stage of n < 16 records is shared out so that 16 / n warps take a run of 32-wide k-chunks
+// of the same record each (no warp visits more than one).
 //
 // Roles. 16 consumer warps do the arithmetic and touch global memory only to read activations. One producer
 // thread keeps the weight stream going, across the boundaries between linears too (weights do not depend on
 // results). One control warp does everything else that waits on global memory: per 16-row tile part it adds the
-// 16 partial sums the consumer warps parked in shared memory (warp order) and stores the outputs; a tile whose
+// 16 partial sums the consumer warps parked in shared memory (fixed pairing) and stores the outputs; a tile whose
 // records fall into several CTAs is finished by the CTA that holds its end, the others post their part in scratch
 // (each value in one 64-bit word together with a per-launch tag: no fence, no counter), and the finisher adds the
-// parts in CTA order - deterministic. A range that ends inside a tile is walked starting with that open tile, so
-// the posted parts are early and a finisher waits only on lower-numbered CTAs. The control warp then reports the
-// linear finished on a device-wide counter and, before a linear flagged `depends`, waits until every CTA has.
+// parts in a fixed order - deterministic. A range that ends inside a tile is walked starting with that open tile, so
+// the posted parts are early and a finisher waits only on lower-numbered CTAs.
+//
+// Order between linears. (a) Data flow: a linear whose activations lie inside an earlier linear's bf16 output reads
+// them from a copy of that output in scratch, in which two values share a 64-bit word with the launch's tag. The
+// finisher of a tile writes those words with plain relaxed stores; a reader polls exactly the words it converts until
+// they carry the tag. That is the whole hand-over: no fence, no counter, and a reader waits for the tiles it needs, not
+// for the linear. (b) Counter: the control warp reports every linear finished on a device-wide counter (release), and
+// before a linear flagged `depends` (or whose buffers overlap earlier ones in a way (a) does not cover) waits until
+// every CTA has. The host decides between the two from the address ranges of the items.
+//
+// A lone warp runs at instruction latency, and at the start and the end of a small linear every warp is alone on the
+// critical path. So the kernel never divides (quotients and reciprocals come from the host), the control warp works
+// out every address before it waits for a part and fetches the lower CTAs' parts ahead of its own.
 //
 // Math per record (Eq. 4 of the paper, integer operands): every PoT state times 2^emax is a small integer, so b1
 // is one byte-table lookup per four weights; b2 = the same bytes routed by "partner i XOR s" (Section 3.3) with
