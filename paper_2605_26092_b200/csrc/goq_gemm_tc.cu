@@ -294,6 +294,9 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bid = blockIdx.x;
+    // a kernel launched as a programmatic dependent of this one (the next call's pre-pass) may be scheduled once every CTA
+    // of this grid is running; it waits for this grid's completion before it touches memory
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int unit_id = bid / p.n_split, split = bid - unit_id * p.n_split;   // n_split > 1 only when every tile is one half
     const int tile = unit_id < p.n_full ? unit_id : p.n_full + (unit_id - p.n_full) / p.halves_per_tile;
     const int n_half = unit_id < p.n_full ? 2 : 1;   // token halves (of 256) this CTA computes
@@ -323,13 +326,16 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
         const uint32_t* e = c_lut.v[slot];
         *reinterpret_cast<uint4*>(lut + (size_t)i * 16) = make_uint4(e[0], e[1], e[2], e[3]);
     }
-    for (int i = tid; i < kTileM; i += kThreads) inv_s[i] = (tok0 + i < p.m_total) ? __ldg(&p.inv_scale[tok0 + i]) : 1.0f;
+    if (warp == 1) tmem_alloc_512(&tmem_base_slot);
+    // Everything above needs nothing from the activation pre-pass, which may still be running (programmatic dependent
+    // launch: this grid is scheduled as soon as the pre-pass lets it); what follows reads what the pre-pass wrote.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (int i = tid; i < kTileM; i += kThreads) inv_s[i] = (tok0 + i < p.m_total) ? __ldcg(&p.inv_scale[tok0 + i]) : 1.0f;
     for (int i = tid; i < kTileN; i += kThreads) {
         const bool in = T0 * kTileRows + i < p.n_tiles * kTileRows;
-        row_s[i] = in ? __ldg(&p.row_scale[T0 * kTileRows + i]) : 0x3C003C00u;   // 1.0
-        row_i[i] = in ? __ldg(&p.row_inv[T0 * kTileRows + i]) : 1.0f;
+        row_s[i] = in ? __ldcg(&p.row_scale[T0 * kTileRows + i]) : 0x3C003C00u;   // 1.0
+        row_i[i] = in ? __ldcg(&p.row_inv[T0 * kTileRows + i]) : 1.0f;
     }
-    if (warp == 1) tmem_alloc_512(&tmem_base_slot);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -582,6 +588,10 @@ __global__ void __launch_bounds__(kPrepThreads) x_to_f16_kernel(const uint16_t* 
                                                                 const uint8_t* __restrict__ packed, int unit_bytes, int k_blocks,
                                                                 int groups_per_block, uint32_t* __restrict__ row_scale,
                                                                 float* __restrict__ row_inv) {
+    // Launched as a programmatic dependent of whatever precedes it in the stream: it may be scheduled before that kernel's
+    // memory is visible, so nothing is read or written before this wait (which returns once the predecessor has completed).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the GEMM's CTAs may set themselves up meanwhile
     if ((int)blockIdx.x >= m_total) {
         __shared__ uint32_t part_max[kPrepThreads / 16][16];
         const int T = (int)blockIdx.x - m_total, r = threadIdx.x & 15, part = threadIdx.x >> 4;
@@ -690,8 +700,20 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return cudaErrorNotSupported;
     if (g.k_in % 8 != 0) return cudaErrorInvalidValue;
-    x_to_f16_kernel<<<m + g.n_tiles, kPrepThreads, 0, st>>>((const uint16_t*)x, g.k_in, xh, inv_scale, m, (const uint8_t*)packed,
-                                                           g.unit_bytes, g.k_blocks, g.groups_per_block, row_scale, row_inv);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(m + g.n_tiles);
+        cfg.blockDim = dim3(kPrepThreads);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaError_t e = cudaLaunchKernelEx(&cfg, x_to_f16_kernel, (const uint16_t*)x, g.k_in, xh, inv_scale, m, (const uint8_t*)packed,
+                                               g.unit_bytes, g.k_blocks, g.groups_per_block, row_scale, row_inv))
+            return e;
+    }
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)g.k_in, (cuuint64_t)m};
     const cuuint64_t strides[1] = {(cuuint64_t)g.k_in * 2};
@@ -733,8 +755,19 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
     p.partial = partial;
     p.tile_counter = tile_counter;
     const int n_ctas = (m <= 256) ? tiles * p.n_split : p.n_full + 2 * split;
-    gemm_tc_kernel<WB><<<n_ctas, kThreads, smem, st>>>(p, map);
-    return cudaGetLastError();
+    // Programmatic dependent launch on the pre-pass just enqueued: the CTAs fill their tables, allocate tensor memory
+    // and initialise their barriers while it runs, and wait (griddepcontrol.wait) before the first read of its outputs.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_ctas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<WB>, p, map);
 }
 
 }  // namespace tc
