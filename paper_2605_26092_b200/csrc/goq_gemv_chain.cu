@@ -566,16 +566,23 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 int sfield = 268 - (int)(amax >> 7);
                 sfield = sfield < 1 ? 1 : (sfield > 253 ? 253 : sfield);
                 const float mult = __uint_as_float((uint32_t)sfield << 23);
-                uint32_t q0[2] = {0u, 0u}, q1[2] = {0u, 0u};
+                // Q = rne(x 2^s) without a convert: adding 1.5 * 2^23 leaves the integer in the low mantissa bits. With 128 more in
+                // the constant the low 16 bits are 256 hi + (lo + 128) for the split Q = 256 hi + lo, lo in [-128, 127]: the high
+                // byte is hi as it stands and the low byte is lo with its top bit flipped. Clamped as raw bits (monotonic):
+                // Q = 32640 (all-ones mantissa at the block's top exponent) would need hi = 128; inf and nan saturate.
+                uint32_t v16[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const uint32_t bits = (j & 1) ? (in32[j >> 1] & 0xFFFF0000u) : (in32[j >> 1] << 16);
-                    // rne to an integer without a convert: adding 1.5 * 2^23 leaves it in the low mantissa bits
-                    int Q = __float_as_int(fmaf(__uint_as_float(bits), mult, 12582912.0f)) - 0x4B400000;
-                    Q = max(-32639, min(32639, Q));
-                    const int lo = ((Q + 128) & 255) - 128, hi = (Q - lo) >> 8;   // Q = 256 hi + lo, both int8
-                    q0[j >> 2] |= (uint32_t)(hi & 255) << (8 * (j & 3));
-                    q1[j >> 2] |= (uint32_t)(lo & 255) << (8 * (j & 3));
+                    const int raw = __float_as_int(fmaf(__uint_as_float(bits), mult, 12582912.0f + 128.0f));
+                    v16[j] = (uint32_t)max(0x4B400000 + 128 - 32640, min(0x4B400000 + 128 + 32639, raw));
+                }
+                uint32_t q0[2], q1[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t t01 = prmt_b32(v16[4 * h], v16[4 * h + 1], 0x5410u), t23 = prmt_b32(v16[4 * h + 2], v16[4 * h + 3], 0x5410u);
+                    q0[h] = prmt_b32(t01, t23, 0x7531u);                   // the four high bytes
+                    q1[h] = prmt_b32(t01, t23, 0x6420u) ^ 0x80808080u;     // the four low bytes, as signed
                 }
                 if (in) {
                     *reinterpret_cast<uint2*>(xb + (size_t)(2 * r) * plane + k0) = make_uint2(q0[0], q0[1]);
