@@ -790,6 +790,34 @@ def run_probe_steady(args):
                       "gbs": nbytes / (best * 1e-3) / 1e9, "status": int(goq.workspace_status(ws))}))
 
 
+def run_probe_gemm(args):
+    """`--probe gemm`: one 4096 x 4096 W3 g128 linear at M = 2048 tokens through goq_gemm (activation pre-pass + tcgen05
+    GEMM), a few times. Small enough for a profiler capture of one launch; prints one JSON line."""
+    import torch
+    from paper_2605_26092_b200 import build
+    build.build()
+    from paper_2605_26092_b200 import goq
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(8100)
+    n, k, m = 4096, 4096, 2048
+    d = goq.desc(n, k, GROUP, WBITS)
+    codes = torch.randint(0, 1 << WBITS, (n, k), dtype=torch.uint8, device="cuda", generator=gen)
+    meta = torch.randint(0, 64, (n, k // 8), dtype=torch.uint8, device="cuda", generator=gen)
+    coef = (torch.randn((n, k // GROUP, 2), device="cuda", generator=gen) * 0.02).to(torch.float16)
+    pk = torch.empty(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
+    goq.pack(d, codes, meta, coef, pk)
+    x = torch.randn((m, k), device="cuda", generator=gen).to(torch.bfloat16)
+    y = torch.empty((m, n), dtype=torch.float32, device="cuda")
+    ws = goq.new_workspace(d, goq.OP_GEMM, m)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    best = float("inf")
+    for _ in range(max(args.steps, 1) + max(args.warmup, 1)):
+        e0.record(); goq.gemm(d, pk, x, m, goq.BF16, y=y, y_dtype=goq.F32, ws=ws); e1.record(); torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    print(json.dumps({"probe": "gemm", "shape": [n, k], "tokens": m, "best_ms": best,
+                      "tflops": 2.0 * m * n * k / (best * 1e-3) / 1e12, "status": int(goq.workspace_status(ws))}))
+
+
 def launch_command(n_gpus, argv, port=None):
     """The command that starts one rank per GPU on this node for `bench.py --gpus N` (N > 1) when no launcher has."""
     port = port or (29500 + os.getpid() % 2000)
@@ -812,13 +840,17 @@ def main():
                     help="force a kernel variant (goq_set_gemv_variant): 0 automatic, 3 streaming, 4 tcgen05 tensor-memory GEMV, ...")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="dram bytes per launch of the dominant kernel from an ncu capture (reported as-is)")
-    ap.add_argument("--probe", choices=("steady",), default=None, help="run one small case only (for profiler captures)")
+    ap.add_argument("--probe", choices=("steady", "gemm"), default=None, help="run one small case only (for profiler captures)")
     ap.add_argument("--copies", type=int, default=2, help="--probe steady: number of 28672 x 8192 linears in the chain")
     args = ap.parse_args()
     if args.probe == "steady":
         if args.steps == 200:
             args.steps = 3
         return run_probe_steady(args)
+    if args.probe == "gemm":
+        if args.steps == 200:
+            args.steps = 3
+        return run_probe_gemm(args)
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # asked for N GPUs without a launcher: start the N ranks (replicas, one per GPU) ourselves
         os.execv(sys.executable, launch_command(args.gpus, sys.argv[1:]))

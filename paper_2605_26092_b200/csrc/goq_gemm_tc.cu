@@ -294,9 +294,6 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap x_map) {
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bid = blockIdx.x;
-    // a kernel launched as a programmatic dependent of this one (the next call's pre-pass) may be scheduled once every CTA
-    // of this grid is running; it waits for this grid's completion before it touches memory
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int unit_id = bid / p.n_split, split = bid - unit_id * p.n_split;   // n_split > 1 only when every tile is one half
     const int tile = unit_id < p.n_full ? unit_id : p.n_full + (unit_id - p.n_full) / p.halves_per_tile;
     const int n_half = unit_id < p.n_full ? 2 : 1;   // token halves (of 256) this CTA computes
@@ -588,9 +585,6 @@ __global__ void __launch_bounds__(kPrepThreads) x_to_f16_kernel(const uint16_t* 
                                                                 const uint8_t* __restrict__ packed, int unit_bytes, int k_blocks,
                                                                 int groups_per_block, uint32_t* __restrict__ row_scale,
                                                                 float* __restrict__ row_inv) {
-    // Launched as a programmatic dependent of whatever precedes it in the stream: it may be scheduled before that kernel's
-    // memory is visible, so nothing is read or written before this wait (which returns once the predecessor has completed).
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the GEMM's CTAs may set themselves up meanwhile
     if ((int)blockIdx.x >= m_total) {
         __shared__ uint32_t part_max[kPrepThreads / 16][16];
@@ -700,20 +694,8 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return cudaErrorNotSupported;
     if (g.k_in % 8 != 0) return cudaErrorInvalidValue;
-    {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(m + g.n_tiles);
-        cfg.blockDim = dim3(kPrepThreads);
-        cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        if (cudaError_t e = cudaLaunchKernelEx(&cfg, x_to_f16_kernel, (const uint16_t*)x, g.k_in, xh, inv_scale, m, (const uint8_t*)packed,
-                                               g.unit_bytes, g.k_blocks, g.groups_per_block, row_scale, row_inv))
-            return e;
-    }
+    x_to_f16_kernel<<<m + g.n_tiles, kPrepThreads, 0, st>>>((const uint16_t*)x, g.k_in, xh, inv_scale, m, (const uint8_t*)packed,
+                                                           g.unit_bytes, g.k_blocks, g.groups_per_block, row_scale, row_inv);
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)g.k_in, (cuuint64_t)m};
     const cuuint64_t strides[1] = {(cuuint64_t)g.k_in * 2};
@@ -766,7 +748,7 @@ static cudaError_t launch_wb(const Geometry& g, const void* packed, const void* 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = (m > 256) ? 1 : 0;   // measured: with at most 256 tokens (two waves of split-K CTAs) the early launch costs ~5 us
     return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<WB>, p, map);
 }
 
