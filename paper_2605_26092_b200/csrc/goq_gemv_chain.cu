@@ -282,6 +282,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
     unsigned char* xq = reinterpret_cast<unsigned char*>(part_bar + kTileSlots);                 // [2][2 m][k_pad + kXPad] int8 planes
     __shared__ volatile int abort_flag;
     __shared__ volatile int done_gen[kTileSlots];
+    __shared__ unsigned tag_s;   // the launch's tag, for the consumer warps (one register less across the record loop)
 
     // the broadcast tells the compiler that the warp index (and everything derived from it) is uniform across the warp
     const int tid = threadIdx.x, warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0), lane = tid & 31;
@@ -290,6 +291,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
 
     if (tid == 0) {
         abort_flag = 0;
+        tag_s = ((*p.epoch + 1u) * 0x9E3779B1u) | 1u;   // nobody changes the count before every CTA has finished the last linear
         for (int i = 0; i < kTileSlots; ++i) { done_gen[i] = 0; mbar_init(&part_bar[i], kNW); }
         for (int s = 0; s < p.n_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kNW); }
         mbar_init(dep_bar, 1);
@@ -512,46 +514,31 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
     int slot = 0, phase = 0;          // position in the stage ring ...
     uint32_t stage_off = 0, bar_off = 0;   // ... and the same as byte offsets of the stage and of its barriers
     const uint32_t unit0 = ring_addr + (uint32_t)warp * unit_bytes + (uint32_t)lane * 16;
-    uint32_t dep_phase = 0, x_phase = 0, free_phase = 0;
-    int x_sel = 0;                    // activation buffer of the current linear
+    uint32_t phases = 0;              // bit 0: dependency barrier, bit 1: activation barrier, bit 2: buffer hand-shake, bit 3: activation buffer in use
     unsigned seq = 0;                 // tile parts this CTA has opened so far (same in every warp): indexes the reduction slots
     bool alive = true;
-    const unsigned tag = ((*p.epoch + 1u) * 0x9E3779B1u) | 1u;   // as in the control warp: the count changes only when every CTA is done
 
     for (int i = 0; i < p.n_items && alive; ++i) {
         const Item& it = p.item[i];
         const Walk wk = make_walk(it, cta, p.g_magic);
         if (wk.L == 0) continue;   // nothing of this linear belongs to this CTA (the control warp reports it finished)
         const int kb = it.k_blocks, k_pad = kb * kBlockK, plane = k_pad + kXPad, m = it.m;
-        if (p.x_double) x_sel ^= 1;
+        if (p.x_double) phases ^= 8u;
+        const int x_sel = (int)((phases >> 3) & 1u);
         unsigned char* xb = xq + (size_t)x_sel * p.xbuf_bytes;
         float* xsc = xscale + x_sel * (kMaxKBlocks * 4 * NG);
 
-        // The last stage of the range, n_tail < 16 records: 16 / n_tail warps share each record, each warp a run of its four
-        // 32-wide chunks (the sums are linear in the chunks), so that no warp visits more than one record. Which record, which
-        // chunks, its k-block and tile part are worked out here, ahead of the dependency wait (divisions).
         const unsigned n_full = wk.L / kStageRecs, n_tail = wk.L - n_full * kStageRecs;
-        unsigned tail_desc = 0;   // [0:4) record of the stage, [4:7) first chunk, [7:10) end chunk, [10:17) k-block, [17:32) tile part
-        if (n_tail) {
-            const unsigned share = c_tail_share.v[n_tail][warp];   // record, first and end chunk of this warp
-            const unsigned rloc = share & 15u, cb = (share >> 4) & 7u, ce = (share >> 7) & 7u;
-            if (rloc < n_tail && cb < ce) {
-                const unsigned rho = walk_record(wk, n_full * kStageRecs + rloc);
-                const unsigned T = mul_shift32(rho, it.kb_magic);
-                const unsigned kbi = rho - T * (unsigned)kb;
-                tail_desc = rloc | (cb << 4) | (ce << 7) | (kbi << 10) | ((unsigned)walk_part_of_tile(wk, (int)T) << 17);
-            }
-        }
 
         // ---- start of the linear: wait for the dependency, then every warp converts its slice of the activations ----
         if (it.depends && i > 0) {
-            if (!wait_bar(dep_bar, dep_phase, &abort_flag, spin)) { alive = false; break; }
-            dep_phase ^= 1u;
+            if (!wait_bar(dep_bar, phases & 1u, &abort_flag, spin)) { alive = false; break; }
+            phases ^= 1u;
         } else if (!p.x_double) {   // one buffer: every warp must have left the previous linear
             __syncwarp();
             if (lane == 0) mbar_arrive(free_bar);
-            if (!wait_bar(free_bar, free_phase, &abort_flag, spin)) { alive = false; break; }
-            free_phase ^= 1u;
+            if (!wait_bar(free_bar, (phases >> 2) & 1u, &abort_flag, spin)) { alive = false; break; }
+            phases ^= 4u;
         }
         {
             // 16-byte chunks of 8 bf16; 16 chunks = one k-block of one token: Q = rne(x 2^s), the block's largest magnitude in [2^14, 2^15)
@@ -604,6 +591,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 // Activations that an earlier linear of this launch produces: read from its tagged copy, word by word,
                 // until every word carries this launch's tag. That is the whole dependency wait: a chunk is converted as soon
                 // as the tiles it comes from are finished, wherever they were finished.
+                const unsigned tag = tag_s;
                 const uint2* tg = p.tags + (size_t)it.xsrc * kTagWords + it.xoff;
                 const int tstride = p.item[it.xsrc].n_tiles * 8;
                 const int bound = spin < kGlobalSpin ? spin : kGlobalSpin;
@@ -653,8 +641,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(x_bar);
-            if (!wait_bar(x_bar, x_phase, &abort_flag, spin)) { alive = false; break; }
-            x_phase ^= 1u;
+            if (!wait_bar(x_bar, (phases >> 1) & 1u, &abort_flag, spin)) { alive = false; break; }
+            phases ^= 2u;
         }
         // B fragment of lane (g, t): column g of column group cg = plane 8 cg + g (token 4 cg + g/2, slice g&1), k bytes t*8..t*8+7 of a chunk.
         // Planes of tokens that do not exist alias the last real plane: an output column depends on its own B column only.
@@ -767,12 +755,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 while (kbi >= kb) { kbi -= kb; ++q; }
             }
         }
-        // ---- the last stage of the range: this warp's chunks of its record, if it has any ----
+        // ---- the last stage of the range, n_tail < 16 records: 16 / n_tail warps share each record, each warp a run of its four
+        //      32-wide chunks (the sums are linear in the chunks), so that no warp visits more than one record; the shares come
+        //      from a constant table and nothing here divides ----
         if (n_tail && alive) {
-            const unsigned rloc = tail_desc & 15u, cb = (tail_desc >> 4) & 7u, ce = (tail_desc >> 7) & 7u;
-            if (cb < ce) {
-                const int kbi = (int)((tail_desc >> 10) & 127u);
-                flush_to((int)(tail_desc >> 17));
+            const unsigned share = c_tail_share.v[n_tail][warp];   // record, first and end chunk of this warp
+            const unsigned rloc = share & 15u, cb = (share >> 4) & 7u, ce = (share >> 7) & 7u;
+            if (rloc < n_tail && cb < ce) {
+                const unsigned rho = walk_record(wk, n_full * kStageRecs + rloc);
+                const unsigned T = mul_shift32(rho, it.kb_magic);
+                const int kbi = (int)(rho - T * (unsigned)kb);
+                flush_to(walk_part_of_tile(wk, (int)T));
                 if (alive && !wait_bar(&full_bar[slot], phase, &abort_flag, spin)) alive = false;
                 if (alive) {
                     tail_open = true;
