@@ -751,7 +751,7 @@ def run_extras(torch, goq, stack, layers, tf_peak, ws):
 
 
 NCU_TRAFFIC_RATIO = 8.96 / 8.39
-NCU_TRAFFIC_RATIO_SEQ = (215.2 + 4.2) / 202.9   # ncu: 215.2 MB read + 4.2 MB written for the 202.9 MB (algorithmic) of a 14-linear launch
+NCU_TRAFFIC_RATIO_SEQ = (215.8 + 4.4) / 202.9   # ncu: 215.2 MB read + 4.2 MB written for the 202.9 MB (algorithmic) of a 14-linear launch
 
 
 def run_probe_steady(args):
