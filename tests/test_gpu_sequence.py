@@ -300,6 +300,49 @@ def test_one_7b_shaped_layer_sampled_rows(goq, form):
         check_parity(y.cpu().numpy().astype(np.float64)[:, rows], y_ref, TIGHT, 1e-4)
 
 
+def test_two_7b_shaped_layers_as_a_true_chain_sampled_rows(goq, form):
+    """The launch configuration the benchmark times, at full size: 14 linears of the 7B shapes, each reading the first
+    k channels of the previous linear's bf16 output (no item flagged: ordered by data flow), run three times on one
+    scratch buffer. Every linear is checked on sampled rows against the oracle evaluated on the bits its producer
+    actually wrote; repeated launches must reproduce the same bits (fixed summation order)."""
+    from tests.gpu_util import dev, pack_weights, check_bf16_output
+    layers, outs, items = [], [], []
+    x0 = si.bf16_activations(1, 4096, seed=900)
+    for j in range(14):
+        name, n, k = si.LLAMA2_7B_LINEARS[j % 7]
+        codes, meta, coef = si.random_quantized(n, k, 128, 3, seed=910 + j)
+        coef = (coef.astype(np.float64) * (0.02 / 0.03) * (4096.0 / k) ** 0.5).astype(np.float16)   # about unit gain along the chain
+        rows = si.sample_rows(n, 24, seed=j)
+        d, packed = pack_weights(n, k, 128, 3, codes, meta, coef)
+        y = torch.zeros((1, n), dtype=torch.bfloat16, device="cuda")
+        x = dev(x0) if j == 0 else outs[j - 1][:, :k]
+        items.append((d, packed, x, 1, y, goq.BF16, False))
+        outs.append(y)
+        layers.append((codes, meta, coef, rows, k))
+    keep = [t[2] for t in items]
+    seq = goq.make_sequence(items)
+    ws = _ws(goq, len(items))
+    first = None
+    for rep in range(3):
+        for y in outs:
+            y.zero_()
+        goq.gemv_sequence(seq, ws)
+        torch.cuda.synchronize()
+        assert goq.workspace_status(ws) == goq.OK
+        bits = [_bits(y) for y in outs]
+        if first is None:
+            first = bits
+            for j, (codes, meta, coef, rows, k) in enumerate(layers):
+                x_bits = x0 if j == 0 else bits[j - 1][:, :k]
+                y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(x_bits), 128, 3, rows=rows)
+                check_bf16_output(si.bf16_bits_to_f64(bits[j])[:, rows], y_ref, 1e-4, "linear %d" % j)
+            assert np.isfinite(si.bf16_bits_to_f64(bits[-1])).all() and np.abs(si.bf16_bits_to_f64(bits[-1])).max() > 0
+        else:
+            for j in range(14):
+                assert np.array_equal(bits[j], first[j]), (rep, j)
+    del keep
+
+
 def test_unsupported_and_invalid_sequences_return_a_status(goq):
     from tests.gpu_util import dev
     L = _layer(goq, 64, 256, 64, 3, seed=1)
