@@ -276,6 +276,16 @@ typedef struct {
 size_t goq_sequence_workspace_bytes(int n_items);
 goq_status goq_gemv_sequence(const goq_gemv_item* items, int n_items, void* ws, size_t ws_bytes, void* stream);
 
+/* goq_sequence_order: how goq_gemv_sequence will order each item of `items` (host only: nothing is launched, no pointer
+ * is dereferenced; the paper has no counterpart). kind_out[i] receives GOQ_ORDER_NONE (the item waits for nothing),
+ * GOQ_ORDER_DATA (it reads an earlier item's bf16 output as that item's 16-channel tiles are finished; source_out[i], if
+ * given, receives that item's index, else -1) or GOQ_ORDER_BARRIER (it waits until every earlier item is complete).
+ * Item 0 and the first item of every further GOQ_SEQUENCE_MAX_ITEMS items (a new launch) are GOQ_ORDER_NONE. */
+#define GOQ_ORDER_NONE 0
+#define GOQ_ORDER_DATA 1
+#define GOQ_ORDER_BARRIER 2
+goq_status goq_sequence_order(const goq_gemv_item* items, int n_items, int32_t* kind_out, int32_t* source_out);
+
 /* goq_gemv_sequence_host: goq_gemv_sequence for callers whose activations and results live in HOST memory.
  * All activations of the sequence sit in one host block and all outputs in another; the call enqueues, on `stream`,
  *   one copy x_host -> x_stage (x_bytes), the sequence kernel, one copy y_stage -> y_host (y_bytes).

@@ -293,6 +293,29 @@ goq_status goq_gemv_sequence(const goq_gemv_item* items, int n_items, void* ws, 
     return GOQ_OK;
 }
 
+goq_status goq_sequence_order(const goq_gemv_item* items, int n_items, int32_t* kind_out, int32_t* source_out) {
+    if (!items || n_items < 1 || !kind_out) return GOQ_ERR_INVALID_ARG;
+    std::vector<goq::SeqCall> calls((size_t)n_items);
+    for (int i = 0; i < n_items; ++i) {
+        const goq_gemv_item& it = items[i];
+        goq::SeqCall& c = calls[(size_t)i];
+        if (!goq::make_geometry(&it.desc, &c.g) || !it.x_bf16 || !it.y || it.batch < 1) return GOQ_ERR_INVALID_ARG;
+        if (it.y_dtype != GOQ_BF16 && it.y_dtype != GOQ_F32) return GOQ_ERR_INVALID_ARG;
+        c.packed = it.packed; c.x = it.x_bf16; c.y = it.y; c.m = it.batch; c.y_dtype = it.y_dtype; c.depends = it.depends ? 1 : 0;
+    }
+    std::vector<goq::SeqOrder> order((size_t)n_items);
+    // a launch holds at most kSeqMaxItems items: a later chunk starts after the earlier ones have completed
+    for (int i0 = 0; i0 < n_items; i0 += goq::kSeqMaxItems) {
+        const int n = (n_items - i0 < goq::kSeqMaxItems) ? (n_items - i0) : goq::kSeqMaxItems;
+        goq::plan_sequence(&calls[(size_t)i0], n, &order[(size_t)i0]);
+        for (int j = 0; j < n; ++j) {
+            kind_out[i0 + j] = order[(size_t)(i0 + j)].kind;
+            if (source_out) source_out[i0 + j] = order[(size_t)(i0 + j)].source < 0 ? -1 : i0 + order[(size_t)(i0 + j)].source;
+        }
+    }
+    return GOQ_OK;
+}
+
 goq_status goq_gemv_sequence_host(const goq_gemv_item* items, int n_items, const void* x_host, void* x_stage,
                                   size_t x_bytes, void* y_host, void* y_stage, size_t y_bytes, void* ws,
                                   size_t ws_bytes, void* stream) {

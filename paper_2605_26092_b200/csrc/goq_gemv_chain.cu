@@ -39,6 +39,7 @@
 // copies in flight are drained and GOQ_ERR_TIMEOUT is written to the status word.
 #include "goq_stream_core.cuh"
 #include "goq_internal.h"
+#include <vector>
 
 namespace goq {
 namespace chain {
@@ -898,6 +899,49 @@ static cudaError_t launch_chain_cfg(chain::Params& p, size_t x_need, cudaStream_
     return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
+// How the items of one launch are ordered (host only, no CUDA call). An item flagged `depends` waits for every earlier
+// item (counter wait). An unflagged item whose activations lie inside ONE earlier bf16 output reads that output's tagged
+// copy and waits word by word; any other overlap with what earlier items read or write falls back to the counter wait;
+// an item that overlaps nothing does not wait.
+void plan_sequence(const SeqCall* calls, int n, SeqOrder* out) {
+    auto overlaps = [](const void* a, size_t an, const void* b, size_t bn) {
+        const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+        return a0 < b0 + bn && b0 < a0 + an;
+    };
+    auto x_bytes = [&](int i) { return (size_t)calls[i].m * calls[i].g.k_in * 2; };
+    auto y_bytes = [&](int i) { return (size_t)calls[i].m * calls[i].g.n_out * (calls[i].y_dtype == GOQ_F32 ? 4 : 2); };
+    for (int j = 0; j < n; ++j) {
+        out[j].kind = kSeqOrderNone; out[j].source = -1; out[j].word_offset = 0;
+        if (j == 0) continue;
+        if (calls[j].depends) { out[j].kind = kSeqOrderBarrier; continue; }
+        int src = -1, hits = 0;
+        bool clash = false;
+        for (int i = 0; i < j; ++i) {
+            if (overlaps(calls[j].x, x_bytes(j), calls[i].y, y_bytes(i))) { src = i; ++hits; }
+            if (overlaps(calls[j].y, y_bytes(j), calls[i].y, y_bytes(i)) || overlaps(calls[j].y, y_bytes(j), calls[i].x, x_bytes(i))) clash = true;
+        }
+        if (!clash && hits == 0) continue;   // independent of everything before it
+        out[j].kind = kSeqOrderBarrier;
+        if (!clash && hits == 1 && calls[src].y_dtype == GOQ_BF16) {
+            const Geometry& gs = calls[src].g;
+            const Geometry& gj = calls[j].g;
+            const int ms = calls[src].m, mj = calls[j].m;
+            const uintptr_t x0 = (uintptr_t)calls[j].x, y0 = (uintptr_t)calls[src].y;
+            const size_t stride = (size_t)gs.n_tiles * 8;   // words per token of the copy
+            if (x0 >= y0 && (x0 - y0) % 2 == 0 && (size_t)ms * stride <= (size_t)chain::kTagWords && gj.k_in % 8 == 0) {
+                const size_t e = (x0 - y0) / 2, tok0 = e / (size_t)gs.n_out, off = e % (size_t)gs.n_out;
+                const bool rows_ok = (mj == 1) ? (off + (size_t)gj.k_in <= (size_t)gs.n_out)
+                                               : (off == 0 && gj.k_in == gs.n_out && tok0 + (size_t)mj <= (size_t)ms);
+                if (off % 8 == 0 && rows_ok && tok0 < (size_t)ms) {
+                    out[j].kind = kSeqOrderData;
+                    out[j].source = src;
+                    out[j].word_offset = (unsigned)(tok0 * stride + off / 2);
+                }
+            }
+        }
+    }
+}
+
 cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, int unit_bytes, void* ws, int spin_limit, cudaStream_t st) {
     static thread_local chain::Params p;   // ~17 KB: kept off the stack
     auto* wsb = (uint8_t*)ws;
@@ -937,45 +981,21 @@ cudaError_t launch_gemv_seq(const SeqCall* calls, int n, int wbits, int group, i
         const size_t b = chain_xbuf_bytes(calls[i].m, g.k_pad);
         if (b > x_need) x_need = b;
     }
-    // Ordering between the items of one launch, from the address ranges. An item flagged `depends` waits for every earlier
-    // item (counter wait). An unflagged item whose activations lie inside ONE earlier bf16 output reads that output's tagged
-    // copy and waits word by word; any other overlap with what earlier items read or write falls back to the counter wait.
-    auto overlaps = [](const void* a, size_t an, const void* b, size_t bn) {
-        const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
-        return a0 < b0 + bn && b0 < a0 + an;
-    };
-    auto x_bytes = [&](int i) { return (size_t)calls[i].m * calls[i].g.k_in * 2; };
-    auto y_bytes = [&](int i) { return (size_t)calls[i].m * calls[i].g.n_out * (calls[i].y_dtype == GOQ_F32 ? 4 : 2); };
-    for (int j = 1; j < n; ++j) {
-        chain::Item& it = p.item[j];
-        if (it.depends) continue;
-        int src = -1, hits = 0;
-        bool clash = false;
-        for (int i = 0; i < j; ++i) {
-            if (overlaps(calls[j].x, x_bytes(j), calls[i].y, y_bytes(i))) { src = i; ++hits; }
-            if (overlaps(calls[j].y, y_bytes(j), calls[i].y, y_bytes(i)) || overlaps(calls[j].y, y_bytes(j), calls[i].x, x_bytes(i))) clash = true;
-        }
-        if (!clash && hits == 0) continue;   // independent of everything before it
-        bool tagged = false;
-        if (!clash && hits == 1 && calls[src].y_dtype == GOQ_BF16) {
-            const Geometry& gs = calls[src].g;
-            const Geometry& gj = calls[j].g;
-            const int ms = calls[src].m, mj = calls[j].m;
-            const uintptr_t x0 = (uintptr_t)calls[j].x, y0 = (uintptr_t)calls[src].y;
-            const size_t stride = (size_t)gs.n_tiles * 8;   // words per token of the copy
-            if (x0 >= y0 && (x0 - y0) % 2 == 0 && (size_t)ms * stride <= (size_t)chain::kTagWords && gj.k_in % 8 == 0) {
-                const size_t e = (x0 - y0) / 2, tok0 = e / (size_t)gs.n_out, off = e % (size_t)gs.n_out;
-                const bool rows_ok = (mj == 1) ? (off + (size_t)gj.k_in <= (size_t)gs.n_out)
-                                               : (off == 0 && gj.k_in == gs.n_out && tok0 + (size_t)mj <= (size_t)ms);
-                if (off % 8 == 0 && rows_ok && tok0 < (size_t)ms) {
-                    it.xsrc = src;
-                    it.xoff = (unsigned)(tok0 * stride + off / 2);
-                    p.item[src].tag_out = 1;
-                    tagged = true;
-                }
+    // Ordering between the items of one launch, from the address ranges (plan_sequence).
+    {
+        static thread_local std::vector<SeqOrder> order;
+        order.resize((size_t)n);
+        plan_sequence(calls, n, order.data());
+        for (int j = 0; j < n; ++j) {
+            chain::Item& it = p.item[j];
+            if (order[(size_t)j].kind == kSeqOrderBarrier) it.depends = 1;
+            else it.depends = 0;
+            if (order[(size_t)j].kind == kSeqOrderData) {
+                it.xsrc = order[(size_t)j].source;
+                it.xoff = order[(size_t)j].word_offset;
+                p.item[it.xsrc].tag_out = 1;
             }
         }
-        if (!tagged) it.depends = 1;
     }
     const int cpg = group / 32;
 #define GOQ_CHAIN(WB_, NG_, K1_)                                                                             \

@@ -57,6 +57,14 @@ struct SeqCall {
     void* y;
     int m, y_dtype, depends;
 };
+// Ordering of one item of a sequence launch, decided on the host from the address ranges
+enum { kSeqOrderNone = 0, kSeqOrderData = 1, kSeqOrderBarrier = 2 };
+struct SeqOrder {
+    int kind;               // kSeqOrder...
+    int source;             // kSeqOrderData: the earlier item whose output holds this item's activations
+    unsigned word_offset;   // ... and where they start in that item's tagged copy (64-bit words)
+};
+void plan_sequence(const SeqCall* calls, int n, SeqOrder* out);
 bool gemv_seq_supported(const Geometry& g, int m);
 size_t gemv_seq_workspace(int n_items);
 size_t gemv_seq_zeroed_prefix(int n_items);

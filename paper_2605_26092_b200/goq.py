@@ -22,7 +22,7 @@ LAYOUT_TILE16_K1 = 2
 
 EXPORTS = (
     "goq_status_string", "goq_packed_bytes", "goq_algorithmic_bytes", "goq_workspace_bytes", "goq_pack",
-    "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant", "goq_workspace_init",
+    "goq_unpack", "goq_gemv", "goq_gemm", "goq_gemv_host", "goq_set_gemv_variant", "goq_sequence_order", "goq_workspace_init",
     "goq_workspace_status", "goq_gemv_static", "goq_last_cuda_error", "goq_sequence_workspace_bytes",
     "goq_gemv_sequence", "goq_gemv_sequence_host", "goq_set_wait_limit", "goq_gemv_static_status", "goq_quantize_activations", "goq_gemm_i8_requant",
     "goq_quantize_geo", "goq_solve_ref",
@@ -98,6 +98,8 @@ def lib() -> ctypes.CDLL:
         L.goq_sequence_workspace_bytes.argtypes = [c_int]
         L.goq_gemv_sequence.restype = c_int
         L.goq_gemv_sequence.argtypes = [POINTER(GemvItem), c_int, c_void_p, ctypes.c_size_t, c_void_p]
+        L.goq_sequence_order.restype = c_int
+        L.goq_sequence_order.argtypes = [POINTER(GemvItem), c_int, POINTER(c_int32), POINTER(c_int32)]
         L.goq_gemv_sequence_host.restype = c_int
         L.goq_gemv_sequence_host.argtypes = [POINTER(GemvItem), c_int, c_void_p, c_void_p, ctypes.c_size_t, c_void_p,
                                              c_void_p, ctypes.c_size_t, c_void_p, ctypes.c_size_t, c_void_p]
@@ -239,6 +241,17 @@ def make_sequence(items):
         a.packed, a.x_bf16, a.y = _ptr(packed), _ptr(x), _ptr(y)
         a.batch, a.y_dtype, a.depends = batch, y_dtype, 1 if depends else 0
     return arr
+
+
+ORDER_NONE, ORDER_DATA, ORDER_BARRIER = 0, 1, 2
+
+
+def sequence_order(seq):
+    """goq_sequence_order: (kinds, sources) - how goq_gemv_sequence will order each item of `seq` (host only)."""
+    n = len(seq)
+    kinds, sources = (c_int32 * n)(), (c_int32 * n)()
+    _check(lib().goq_sequence_order(seq, n, kinds, sources), "goq_sequence_order")
+    return list(kinds), list(sources)
 
 
 def gemv_sequence(seq, ws, stream=None):

@@ -60,3 +60,50 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(g, "_LIB_PATH", "/nonexistent/libgoq.so")
     with pytest.raises(ImportError):
         g.lib()
+
+
+class _FakeBuffer:
+    """Stands in for a device tensor in make_sequence: goq_sequence_order only compares addresses."""
+    def __init__(self, addr):
+        self.addr = addr
+
+    def data_ptr(self):
+        return self.addr
+
+
+def test_sequence_order_is_decided_from_the_address_ranges(goq):
+    """goq_sequence_order runs on the host and dereferences nothing: items are described with made-up addresses.
+    Cases: nothing shared; the whole bf16 output of the previous item; a slice of it (batch 1) at a multiple of 8
+    channels and at an odd start; an fp32 producer; an input that spans two outputs; an output buffer written twice; a
+    flagged item; batch 2 reading all of a batch-2 output and reading a slice of it."""
+    d44 = goq.desc(4096, 4096, 128, 3)
+    d_half = goq.desc(256, 2048, 128, 3)     # reads 2048 channels
+    d_two = goq.desc(256, 8192, 128, 3)      # reads 8192 channels
+    B = 1 << 20
+    X0, Y0, Y1, Y2, Y3, Y4 = (_FakeBuffer(0x10000000 + i * B) for i in range(6))
+    pk = _FakeBuffer(0x70000000)
+    def order(items):
+        kinds, sources = goq.sequence_order(goq.make_sequence(items))
+        return list(zip(kinds, sources))
+    N, D, Bar = goq.ORDER_NONE, goq.ORDER_DATA, goq.ORDER_BARRIER
+    # independent items
+    assert order([(d44, pk, X0, 1, Y0, goq.BF16, False), (d44, pk, X0, 1, Y1, goq.BF16, False)]) == [(N, -1), (N, -1)]
+    # a chain through whole outputs, then an fp32 producer, then a flagged item
+    got = order([(d44, pk, X0, 1, Y0, goq.BF16, False), (d44, pk, Y0, 1, Y1, goq.BF16, False),
+                 (d44, pk, Y1, 1, Y2, goq.F32, False), (d44, pk, Y2, 1, Y3, goq.BF16, False),
+                 (d44, pk, X0, 1, Y4, goq.BF16, True)])
+    assert got == [(N, -1), (D, 0), (D, 1), (Bar, -1), (Bar, -1)]
+    # slices of a batch-1 output: channel 2048 (a multiple of 8) is data flow, channel 2052 is not
+    s_ok, s_odd = _FakeBuffer(Y0.addr + 2048 * 2), _FakeBuffer(Y0.addr + 2052 * 2)
+    got = order([(d44, pk, X0, 1, Y0, goq.BF16, False), (d_half, pk, s_ok, 1, Y1, goq.BF16, False),
+                 (d_half, pk, s_odd, 1, Y2, goq.BF16, False)])
+    assert got == [(N, -1), (D, 0), (Bar, -1)]
+    # one input spanning two outputs that lie side by side; then an output buffer written a second time
+    y_lo, y_hi = _FakeBuffer(Y0.addr), _FakeBuffer(Y0.addr + 4096 * 2)
+    got = order([(d44, pk, X0, 1, y_lo, goq.BF16, False), (d44, pk, X0, 1, y_hi, goq.BF16, False),
+                 (d_two, pk, y_lo, 1, Y1, goq.BF16, False), (d44, pk, X0, 1, y_lo, goq.BF16, False)])
+    assert got == [(N, -1), (N, -1), (Bar, -1), (Bar, -1)]
+    # batch 2: the whole output is data flow, a narrower view of it is not
+    got = order([(d44, pk, X0, 2, Y0, goq.BF16, False), (d44, pk, Y0, 2, Y1, goq.BF16, False),
+                 (d_half, pk, Y0, 2, Y2, goq.BF16, False)])
+    assert got == [(N, -1), (D, 0), (Bar, -1)]
