@@ -673,13 +673,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 for (int cg = 0; cg < NG; ++cg) acc[cg][0] = acc[cg][1] = 0.f;
             }
         };
-        // ---- full stages: record st*16 + warp of the walk. Its tile, k-block and part are found once and then carried
-        //      along (16 records further each stage); only the turn of the walk needs them found again ----
+        // ---- full stages: record st*16 + warp of the walk, one per pass of ONE loop. Its k-block and tile part are carried
+        //      along (16 records further each stage: a compare and a subtract), found afresh only at the turn of the walk ----
         {
-            unsigned st = 0, j = (unsigned)warp;
+            unsigned j = (unsigned)warp;
             int kbi = 0, q = 0;
             bool locate = true;
-            while (st < n_full && alive) {
+            for (unsigned st = 0; st < n_full && alive; ++st) {
                 if (locate) {
                     const unsigned rho = walk_record(wk, j);
                     const int T = (int)mul_shift32(rho, it.kb_magic);
@@ -687,73 +687,62 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                     q = walk_part_of_tile(wk, T);
                     locate = false;
                 }
-                if (cur_q < q) flush_to(q);
-                if (!alive) break;
-                // stages in a row in which this warp's record stays inside its tile and on this side of the turn of the walk
-                unsigned run = ((unsigned)(kb - kbi) + kStageRecs - 1) / kStageRecs;
-                const bool before_turn = j < wk.L1;
-                if (before_turn) run = min(run, (wk.L1 - j + kStageRecs - 1) / kStageRecs);
-                run = min(run, n_full - st);
-                st += run;
-                j += run * kStageRecs;
-                if (before_turn && j >= wk.L1) locate = true;   // the next record lies beyond the turn
-                // ================= the hot loop: one record per iteration =================
-                uint32_t koff = (uint32_t)kbi * kBlockK, ksc = (uint32_t)kbi * (16 * NG);
-                kbi += (int)run * kStageRecs;
-                for (; run; --run, koff += kStageRecs * kBlockK, ksc += kStageRecs * 16 * NG) {
-                    {   // bounded wait for the stage, written out so that the record loop contains no call
-                        int polls = 0;
-                        while (!try_wait_a(full_addr + bar_off, phase)) {
-                            if (++polls >= spin || ((polls & 255) == 0 && abort_flag)) {
-                                abort_flag = 1;
-                                alive = false;   // give up after this iteration (whatever it computes is never stored)
-                                run = 1;
-                                break;
-                            }
+                if (cur_q < q) { flush_to(q); if (!alive) break; }
+                const uint32_t koff = (uint32_t)kbi * kBlockK, ksc = (uint32_t)kbi * (16 * NG);
+                {   // bounded wait for the stage, written out so that the record loop contains no call
+                    int polls = 0;
+                    while (!try_wait_a(full_addr + bar_off, phase)) {
+                        if (++polls >= spin || ((polls & 255) == 0 && abort_flag)) {
+                            abort_flag = 1;
+                            alive = false;   // give up after this iteration (whatever it computes is never stored)
+                            break;
                         }
                     }
-                    const uint32_t unit = order_after_wait(unit0 + stage_off);
-                    const uint4 wv0 = lds128(unit), wv1 = lds128(unit + 512);
-                    const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
-                    const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
-                    int s1[NG][4], s2[NG][4], s3[NG][4];
-                    float rec[NG][2];
-#pragma unroll
-                    for (int cg = 0; cg < NG; ++cg) {
-                        rec[cg][0] = rec[cg][1] = 0.f;
-#pragma unroll
-                        for (int r = 0; r < 4; ++r) s1[cg][r] = s2[cg][r] = s3[cg][r] = 0;
-                    }
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t pa0, pb0, qa0, qb0, fa0, fb0, pa1, pb1, qa1, qb1, fa1, fb1;
-                        decode_word<WB, K1>(w0[c], lut_lane, pa0, pb0, qa0, qb0, fa0, fb0);
-                        decode_word<WB, K1>(w1[c], lut_lane, pa1, pb1, qa1, qb1, fa1, fb1);
-#pragma unroll
-                        for (int cg = 0; cg < NG; ++cg) {
-                            const uint2 xf = lds64(xrow[cg] + koff + c * 32);
-                            mma_s8(s1[cg], pa0, pa1, pb0, pb1, xf.x, xf.y);
-                            if constexpr (!K1) {
-                                mma_s8(s2[cg], qa0, qa1, qb0, qb1, xf.x, xf.y);
-                                mma_s8(s3[cg], fa0, fa1, fb0, fb1, xf.x, xf.y);
-                            }
-                        }
-                        if (((c + 1) % CPG) == 0) group_end<NG, K1>(s1, s2, s3, lds32(coef_addr + (c / CPG) * 64), lds32(coef_addr + (c / CPG) * 64 + 32), rec);
-                    }
-#pragma unroll
-                    for (int cg = 0; cg < NG; ++cg) {
-                        const float sv = lds_f32(xs_tok[cg] + ksc);   // undo the activation scale of this k-block
-                        acc[cg][0] = fmaf(sv, rec[cg][0], acc[cg][0]);
-                        acc[cg][1] = fmaf(sv, rec[cg][1], acc[cg][1]);
-                    }
-                    __syncwarp();
-                    if (lane == 0) arrive_a(empty_addr + bar_off);
-                    stage_off += (uint32_t)stage_bytes; bar_off += 8;
-                    if (++slot == p.n_stages) { slot = 0; phase ^= 1; stage_off = 0; bar_off = 0; }
                 }
-                // the next record is 16 further in the same linear order: it has left the tile (that is why the run ended,
-                // unless the stages ran out); a tile narrower than a stage may be skipped altogether
-                while (kbi >= kb) { kbi -= kb; ++q; }
+                const uint32_t unit = order_after_wait(unit0 + stage_off);
+                const uint4 wv0 = lds128(unit), wv1 = lds128(unit + 512);
+                const uint32_t coef_addr = unit - lane * 16 + kCodeBytesPerUnit + g * 4;
+                const uint32_t w0[4] = {wv0.x, wv0.y, wv0.z, wv0.w}, w1[4] = {wv1.x, wv1.y, wv1.z, wv1.w};
+                int s1[NG][4], s2[NG][4], s3[NG][4];
+                float rec[NG][2];
+#pragma unroll
+                for (int cg = 0; cg < NG; ++cg) {
+                    rec[cg][0] = rec[cg][1] = 0.f;
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) s1[cg][r] = s2[cg][r] = s3[cg][r] = 0;
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pa0, pb0, qa0, qb0, fa0, fb0, pa1, pb1, qa1, qb1, fa1, fb1;
+                    decode_word<WB, K1>(w0[c], lut_lane, pa0, pb0, qa0, qb0, fa0, fb0);
+                    decode_word<WB, K1>(w1[c], lut_lane, pa1, pb1, qa1, qb1, fa1, fb1);
+#pragma unroll
+                    for (int cg = 0; cg < NG; ++cg) {
+                        const uint2 xf = lds64(xrow[cg] + koff + c * 32);
+                        mma_s8(s1[cg], pa0, pa1, pb0, pb1, xf.x, xf.y);
+                        if constexpr (!K1) {
+                            mma_s8(s2[cg], qa0, qa1, qb0, qb1, xf.x, xf.y);
+                            mma_s8(s3[cg], fa0, fa1, fb0, fb1, xf.x, xf.y);
+                        }
+                    }
+                    if (((c + 1) % CPG) == 0) group_end<NG, K1>(s1, s2, s3, lds32(coef_addr + (c / CPG) * 64), lds32(coef_addr + (c / CPG) * 64 + 32), rec);
+                }
+#pragma unroll
+                for (int cg = 0; cg < NG; ++cg) {
+                    const float sv = lds_f32(xs_tok[cg] + ksc);   // undo the activation scale of this k-block
+                    acc[cg][0] = fmaf(sv, rec[cg][0], acc[cg][0]);
+                    acc[cg][1] = fmaf(sv, rec[cg][1], acc[cg][1]);
+                }
+                __syncwarp();
+                if (lane == 0) arrive_a(empty_addr + bar_off);
+                stage_off += (uint32_t)stage_bytes; bar_off += 8;
+                if (++slot == p.n_stages) { slot = 0; phase ^= 1; stage_off = 0; bar_off = 0; }
+                // the next record is 16 further in the same linear order, unless the walk turns in between
+                const bool before_turn = j < wk.L1;
+                j += kStageRecs;
+                kbi += kStageRecs;
+                while (kbi >= kb) { kbi -= kb; ++q; }   // it has left the tile; a tile narrower than a stage may be skipped altogether
+                if (before_turn && j >= wk.L1) locate = true;
             }
         }
         // ---- the last stage of the range, n_tail < 16 records: 16 / n_tail warps share each record, each warp a run of its four
