@@ -546,3 +546,52 @@ def test_host_buffer_entry_point(goq):
     torch.cuda.synchronize()
     y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(xb), 64, 3)
     assert O.normwise_rel_err(yh.numpy().astype(np.float64), y_ref) <= TIGHT
+
+
+def test_weights_packed_just_before_the_call_on_the_same_stream(goq):
+    """Stream order without a synchronise in between: goq_pack writes the packed image, and the very next calls on the same
+    stream are goq_gemv (batch 1, the chain kernel), goq_gemm at 300 tokens (tcgen05 kernel, launched as a programmatic
+    dependent of its pre-pass) and goq_gemv_sequence. Each must give the bits of the same call made after a synchronise:
+    none of these kernels reads the weights before the preceding work on the stream is complete. (The streaming kernel
+    behind goq_gemv at batch 5..16 prefetches weights ahead of its dependency wait; its rule is stated in goq.h.)"""
+    from tests.gpu_util import dev
+    n, k, g, b, m = 2048, 1024, 128, 3, 300
+    codes, meta, coef = si.random_quantized(n, k, g, b, seed=77)
+    d = goq.desc(n, k, g, b)
+    x1, xm = dev(si.bf16_activations(1, k, seed=78)), dev(si.bf16_activations(m, k, seed=79))
+    cd, md, fd = dev(codes), dev(meta), dev(coef)
+    ws_v, ws_m = goq.new_workspace(d, goq.OP_GEMV, 1), goq.new_workspace(d, goq.OP_GEMM, m)
+    ws_s = torch.empty(goq.sequence_workspace_bytes(2), dtype=torch.uint8, device="cuda")
+    goq.workspace_init(ws_s)
+    torch.cuda.synchronize()
+
+    def run(sync_between):
+        packed = torch.full((goq.packed_bytes(d),), 0x5A, dtype=torch.uint8, device="cuda")   # stale contents
+        y1 = torch.zeros((1, n), dtype=torch.float32, device="cuda")
+        ym = torch.zeros((m, n), dtype=torch.float32, device="cuda")
+        ya = torch.zeros((1, n), dtype=torch.bfloat16, device="cuda")
+        yb = torch.zeros((1, n), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        goq.pack(d, cd, md, fd, packed)
+        if sync_between:
+            torch.cuda.synchronize()
+        goq.gemv(d, packed, x1, 1, y1, goq.F32, ws=ws_v)
+        if sync_between:
+            torch.cuda.synchronize()
+        goq.gemm(d, packed, xm, m, goq.BF16, y=ym, y_dtype=goq.F32, ws=ws_m)
+        if sync_between:
+            torch.cuda.synchronize()
+        seq = goq.make_sequence([(d, packed, x1, 1, ya, goq.BF16, False), (d, packed, ya[:, :k], 1, yb, goq.F32, False)])
+        goq.gemv_sequence(seq, ws_s)
+        torch.cuda.synchronize()
+        for w in (ws_v, ws_m, ws_s):
+            assert goq.workspace_status(w) == goq.OK
+        return y1.clone(), ym.clone(), ya.clone(), yb.clone()
+
+    ref = run(True)
+    for rep in range(3):
+        got = run(False)
+        for a, r in zip(got, ref):
+            assert torch.equal(a, r), rep
+    y_ref = O.linear_f64(codes, meta, coef, si.bf16_bits_to_f64(x1.view(torch.int16).cpu().numpy().view(np.uint16)), g, b)
+    assert O.normwise_rel_err(ref[0].cpu().numpy().astype(np.float64), y_ref) <= TIGHT
