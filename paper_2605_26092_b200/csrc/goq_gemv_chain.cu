@@ -145,6 +145,15 @@ __device__ __noinline__ bool wait_slow_a(uint32_t bar, uint32_t parity, volatile
     *abort_flag = 1;
     return false;
 }
+// the same bounded wait, inlined (start-of-linear waits: a call would sit on the critical path)
+__device__ __forceinline__ bool wait_a(uint32_t bar, uint32_t parity, volatile int* abort_flag, int limit) {
+    for (int it = 0; it < limit; ++it) {
+        if (try_wait_a(bar, parity)) return true;
+        if ((it & 63) == 63 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
 __device__ __forceinline__ float lds_f32(uint32_t addr) {
     float v;
     asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
@@ -214,13 +223,16 @@ __device__ __forceinline__ int walk_tile_of_part(const Walk& w, int q) { return 
 // and arrives on the slot's mbarrier; the control warp adds the 16 partials, stores or passes on the result and then
 // frees the slot. Returns false after a give-up.
 struct FlushCtx {
-    float* red;
-    uint64_t* part_bar;
+    uint32_t red_addr;        // shared-window addresses: no 64-bit pointers are kept alive across the record loop
+    uint32_t part_bar_addr;
     volatile int* done_gen;
     volatile int* abort_flag;
     int spin;
 };
 struct Sums4 { float v[4]; };   // by value: the accumulators never have their address taken, so they stay in registers
+__device__ __forceinline__ void sts_f32(uint32_t addr, float v) {
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
 template <int NG>
 __device__ __forceinline__ bool flush_part(const FlushCtx& c, unsigned sq, Sums4 sums) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
@@ -233,14 +245,14 @@ __device__ __forceinline__ bool flush_part(const FlushCtx& c, unsigned sq, Sums4
             __nanosleep(20);
         }
     }
-    float* rb = c.red + ((size_t)rs * kNW + warp) * (NG * 64);
+    const uint32_t rb = c.red_addr + (uint32_t)(((rs * kNW + warp) * (NG * 64) + g * 4 + t) * 4);
 #pragma unroll
     for (int cg = 0; cg < NG; ++cg) {
-        rb[cg * 64 + g * 4 + t] = sums.v[2 * cg];
-        rb[cg * 64 + (g + 8) * 4 + t] = sums.v[2 * cg + 1];
+        sts_f32(rb + (cg * 64) * 4, sums.v[2 * cg]);
+        sts_f32(rb + (cg * 64 + 32) * 4, sums.v[2 * cg + 1]);
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(&c.part_bar[rs]);   // releases the warp's stores (ordered before it by the barrier above)
+    if (lane == 0) arrive_a(c.part_bar_addr + rs * 8);   // releases the warp's stores (ordered before it by the barrier above)
     return true;
 }
 
@@ -512,6 +524,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
     const uint32_t lut_lane = smem_u32(lut) + (lane & (kLutCopies - 1)) * 16;
     const uint32_t ring_addr = smem_u32(ring), unit_bytes = (uint32_t)p.unit_bytes;
     const uint32_t full_addr = smem_u32(full_bar), empty_addr = smem_u32(empty_bar);
+    const uint32_t dep_addr = smem_u32(dep_bar), xbar_addr = smem_u32(x_bar), free_addr = smem_u32(free_bar);
     int slot = 0, phase = 0;          // position in the stage ring ...
     uint32_t stage_off = 0, bar_off = 0;   // ... and the same as byte offsets of the stage and of its barriers
     const uint32_t unit0 = ring_addr + (uint32_t)warp * unit_bytes + (uint32_t)lane * 16;
@@ -533,12 +546,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
 
         // ---- start of the linear: wait for the dependency, then every warp converts its slice of the activations ----
         if (it.depends && i > 0) {
-            if (!wait_bar(dep_bar, phases & 1u, &abort_flag, spin)) { alive = false; break; }
+            if (!wait_a(dep_addr, phases & 1u, &abort_flag, spin)) { alive = false; break; }
             phases ^= 1u;
         } else if (!p.x_double) {   // one buffer: every warp must have left the previous linear
             __syncwarp();
-            if (lane == 0) mbar_arrive(free_bar);
-            if (!wait_bar(free_bar, (phases >> 2) & 1u, &abort_flag, spin)) { alive = false; break; }
+            if (lane == 0) arrive_a(free_addr);
+            if (!wait_a(free_addr, (phases >> 2) & 1u, &abort_flag, spin)) { alive = false; break; }
             phases ^= 4u;
         }
         {
@@ -641,8 +654,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 if (!alive) break;
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(x_bar);
-            if (!wait_bar(x_bar, (phases >> 1) & 1u, &abort_flag, spin)) { alive = false; break; }
+            if (lane == 0) arrive_a(xbar_addr);
+            if (!wait_a(xbar_addr, (phases >> 1) & 1u, &abort_flag, spin)) { alive = false; break; }
             phases ^= 2u;
         }
         // B fragment of lane (g, t): column g of column group cg = plane 8 cg + g (token 4 cg + g/2, slice g&1), k bytes t*8..t*8+7 of a chunk.
@@ -655,7 +668,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
             xs_tok[cg] = smem_u32(xsc + min(cg * 4 + t, m - 1));
         }
         FlushCtx fc;
-        fc.red = red; fc.part_bar = part_bar; fc.done_gen = done_gen; fc.abort_flag = &abort_flag; fc.spin = spin;
+        fc.red_addr = smem_u32(red); fc.part_bar_addr = smem_u32(part_bar); fc.done_gen = done_gen; fc.abort_flag = &abort_flag; fc.spin = spin;
 
         int cur_q = 0;                         // tile part this warp is accumulating
         float acc[NG][2];
@@ -756,7 +769,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
                 const unsigned T = mul_shift32(rho, it.kb_magic);
                 const int kbi = (int)(rho - T * (unsigned)kb);
                 flush_to(walk_part_of_tile(wk, (int)T));
-                if (alive && !wait_bar(&full_bar[slot], phase, &abort_flag, spin)) alive = false;
+                if (alive && !wait_a(full_addr + bar_off, phase, &abort_flag, spin)) alive = false;
                 if (alive) {
                     tail_open = true;
                     const uint32_t unit = order_after_wait(ring_addr + slot * stage_bytes + rloc * unit_bytes + lane * 16);
@@ -802,9 +815,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_chain_kernel(const __grid_co
         flush_to(wk.P);   // every part has been handed over
         if (!alive) break;
         if (n_tail) {   // every warp takes part in the tail stage's hand-shake, with or without chunks of its own
-            if (!tail_open && !wait_bar(&full_bar[slot], phase, &abort_flag, spin)) { alive = false; break; }
+            if (!tail_open && !wait_a(full_addr + bar_off, phase, &abort_flag, spin)) { alive = false; break; }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[slot]);
+            if (lane == 0) arrive_a(empty_addr + bar_off);
             stage_off += (uint32_t)stage_bytes; bar_off += 8;
             if (++slot == p.n_stages) { slot = 0; phase ^= 1; stage_off = 0; bar_off = 0; }
         }
