@@ -451,3 +451,85 @@ def test_long_sequence_is_split_into_launches_and_small_grids_work(goq, form):
         ref = ref_a if i % 2 == 0 else ref_b
         assert O.normwise_rel_err(y.cpu().numpy().astype(np.float64), ref) <= TIGHT, i
     assert torch.equal(ys[0], ys[298]) and torch.equal(ys[1], ys[299])
+
+
+@pytest.mark.parametrize("g,b,k1,batch", [(32, 2, False, 1), (64, 2, False, 5), (128, 3, True, 1), (64, 3, True, 4), (32, 3, False, 8)])
+def test_data_flow_chain_over_widths_groups_single_basis_and_batches(goq, form, g, b, k1, batch):
+    """A four-linear true chain (no item flagged) for every template form of the chain kernel that the headline case does
+    not reach: W2, the three group sizes, the single-basis layout (no second operand), one and two column groups of
+    tokens. Every linear against the oracle on the bits its producer wrote."""
+    from tests.gpu_util import dev
+    layout = goq.LAYOUT_TILE16_K1 if k1 else goq.LAYOUT_TILE16
+    if batch > 1:   # the whole output of the producer (batch 1 reads slices, below)
+        return _whole_output_chain(goq, g, b, layout, batch)
+    shapes = [(1040, 384), (640, 1040 - 16), (2064, 640), (96, 2064 - 16)]   # channel counts that are no multiple of 16 or 128
+    shapes = [(n, (k // g) * g) for n, k in shapes]                            # ... but whole macro-blocks along k
+    layers, outs, items = [], [], []
+    x0 = si.bf16_activations(batch, shapes[0][1], seed=950 + g)
+    for j, (n, k) in enumerate(shapes):
+        codes, meta, coef = si.random_quantized(n, k, g, b, seed=960 + j + g + b)
+        d = goq.desc(n, k, g, b, layout)
+        packed = torch.zeros(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
+        goq.pack(d, dev(codes), dev(meta), dev(coef), packed)
+        last = j == len(shapes) - 1
+        y = torch.zeros((batch, n), dtype=torch.float32 if last else torch.bfloat16, device="cuda")
+        x = dev(x0) if j == 0 else outs[j - 1][:, :k]   # a slice of the producer's row
+        items.append((d, packed, x, batch, y, goq.F32 if last else goq.BF16, False))
+        outs.append(y)
+        layers.append((codes, meta, coef, n, k))
+    torch.cuda.synchronize()
+    kinds, _ = goq.sequence_order(goq.make_sequence(items))
+    assert kinds == [goq.ORDER_NONE] + [goq.ORDER_DATA] * 3
+    ws = _ws(goq, len(items))
+    goq.gemv_sequence(goq.make_sequence(items), ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    x_bits = x0
+    for j, (codes, meta, coef, n, k) in enumerate(layers):
+        c, mt, cf = (codes, np.zeros_like(meta), np.stack([coef[..., 0], np.zeros_like(coef[..., 1])], axis=-1)) if k1 else (codes, meta, coef)
+        y_ref = O.linear_f64(c, mt, cf, si.bf16_bits_to_f64(x_bits[:, :k]), g, b)
+        got = outs[j].float().cpu().numpy().astype(np.float64)
+        if j == len(layers) - 1:
+            assert O.normwise_rel_err(got, y_ref) <= TIGHT, (j, O.normwise_rel_err(got, y_ref))
+        else:
+            from tests.gpu_util import check_bf16_output
+            check_bf16_output(got, y_ref, 1e-4, "linear %d" % j)
+            x_bits = _bits(outs[j])
+
+
+def _whole_output_chain(goq, g, b, layout, batch):
+    """batch > 1: each linear reads the whole bf16 output of the previous one (k_j = n_{j-1})."""
+    from tests.gpu_util import dev, check_bf16_output
+    k1 = layout == goq.LAYOUT_TILE16_K1
+    widths = [384, 1024, 640, 2048, 96]
+    widths = [max(g, (w // g) * g) for w in widths]
+    layers, outs, items = [], [], []
+    x0 = si.bf16_activations(batch, widths[0], seed=970 + g)
+    for j in range(4):
+        n, k = widths[j + 1], widths[j]
+        codes, meta, coef = si.random_quantized(n, k, g, b, seed=980 + j + g + b)
+        d = goq.desc(n, k, g, b, layout)
+        packed = torch.zeros(goq.packed_bytes(d), dtype=torch.uint8, device="cuda")
+        goq.pack(d, dev(codes), dev(meta), dev(coef), packed)
+        last = j == 3
+        y = torch.zeros((batch, n), dtype=torch.float32 if last else torch.bfloat16, device="cuda")
+        x = dev(x0) if j == 0 else outs[j - 1]
+        items.append((d, packed, x, batch, y, goq.F32 if last else goq.BF16, False))
+        outs.append(y)
+        layers.append((codes, meta, coef, n, k))
+    kinds, sources = goq.sequence_order(goq.make_sequence(items))
+    assert kinds == [goq.ORDER_NONE] + [goq.ORDER_DATA] * 3 and sources == [-1, 0, 1, 2]
+    ws = _ws(goq, len(items))
+    goq.gemv_sequence(goq.make_sequence(items), ws)
+    torch.cuda.synchronize()
+    assert goq.workspace_status(ws) == goq.OK
+    x_bits = x0
+    for j, (codes, meta, coef, n, k) in enumerate(layers):
+        c, mt, cf = (codes, np.zeros_like(meta), np.stack([coef[..., 0], np.zeros_like(coef[..., 1])], axis=-1)) if k1 else (codes, meta, coef)
+        y_ref = O.linear_f64(c, mt, cf, si.bf16_bits_to_f64(x_bits), g, b)
+        got = outs[j].float().cpu().numpy().astype(np.float64)
+        if j == 3:
+            assert O.normwise_rel_err(got, y_ref) <= TIGHT, (j, O.normwise_rel_err(got, y_ref))
+        else:
+            check_bf16_output(got, y_ref, 1e-4, "linear %d" % j)
+            x_bits = _bits(outs[j])
