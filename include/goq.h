@@ -257,7 +257,8 @@ goq_status goq_gemv_static_status(void* stream, int* status_out);
  *   Constraints (else GOQ_ERR_UNSUPPORTED): every item has the same wbits (2 or 3) and group (32, 64, 128),
  *   batch <= 8, k_in <= 12288, and the staged activations (2 * batch * (round_up(k_in, 128) + 32) bytes) fit in
  *   shared memory beside two 16-record stages of the weight stream (about 180 KB: batch 8 up to k_in = 11008).
- *   ws       goq_sequence_workspace_bytes(n_items) bytes, 256-byte aligned, zero-filled once with
+ *   ws       goq_sequence_workspace_bytes(n_items) bytes (about 0.5 MB per item: the parts of tiles shared between SMs
+ *            and the copies of bf16 outputs that later items read), 256-byte aligned, zero-filled once with
  *            goq_workspace_init; every call leaves it ready for the next one. Its first word is the status word
  *            (goq_workspace_status): after GOQ_ERR_TIMEOUT the outputs are undefined and the buffer must be
  *            zero-filled again before it is reused.
